@@ -1,0 +1,155 @@
+/*
+ * ecco.h -- C ABI of the B200-native Ecco 4x block codec (decompression hot path).
+ *
+ * Format (Ecco, Sec. 3.1-3.2): a tensor is cut into groups of 128 fp16 values; every group is
+ * stored in one 64-byte block holding an FP8 group scale (the group's signed abs-max under a
+ * per-tensor power-of-two factor T = 2^e), a 2-bit choice ID_HF among H = 4 Huffman codebooks,
+ * the Huffman-coded index ID_KP of one of S <= 64 shared 15-centroid k-means patterns, and 128
+ * Huffman-coded 4-bit indices (code lengths 2..8; index 15 = the abs-max itself).  A stream
+ * longer than the block is clipped; a shorter one is padded with 15-bit outliers (7-bit
+ * location + FP8 value) for the next-largest values (Sec. 3.2, Fig. 4 step 9).
+ *
+ * Bit order inside a block (the paper's block drawing is not part of its text; this is the
+ * library's definition): stream bit k is bit (k & 7) of byte (k >> 3).  Fixed-width fields are
+ * least-significant bit first; codewords are first-code-bit first (canonical codes: symbols
+ * ordered by (length, id), consecutive values).  Stream order: [0,8) scale byte (OCP E4M3),
+ * [8,10) ID_HF, [10, ..) ID_KP codeword, then the codewords of positions 0..127, zero fill,
+ * and pads in 15-bit slots growing down from bit 511: pad j occupies [512-15(j+1), 512-15j),
+ * low 7 bits location, high 8 bits E4M3 value; at most 16 pads.
+ *
+ * Conventions: every function returns ECCO_OK (0) or a negative error code and never throws.
+ * "host" pointers are ordinary CPU memory; "device" pointers (d_*) are CUDA device memory
+ * owned by the caller, who also owns the stream.  Device calls are asynchronous on `stream`
+ * (a cudaStream_t passed as void*, NULL = the legacy default stream), never synchronise and
+ * never allocate.  fp16 values travel as raw uint16_t / void*.  d_blocks, d_out, d_x, d_q and
+ * d_meta must be 16-byte aligned.  The library refuses to run on a device that is not
+ * compute capability 10.x (ECCO_ERR_UNSUPPORTED_ARCH); there is no CPU fallback.
+ */
+#ifndef ECCO_H_
+#define ECCO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define ECCO_GROUP 128          /* values per group  (Sec. 3.1) */
+#define ECCO_BLOCK_BYTES 64     /* bytes per block   (Sec. 3.1) */
+#define ECCO_MAX_PATTERNS 64    /* S                 (Sec. 3.2) */
+#define ECCO_CODEBOOKS 4        /* H                 (Sec. 3.2) */
+#define ECCO_CENTROIDS 15       /* per pattern       (Sec. 3.2) */
+#define ECCO_MAX_BATCH 8        /* ecco_gemv rows of x */
+
+enum {
+    ECCO_OK = 0,
+    ECCO_ERR_INVALID_ARG = -1,
+    ECCO_ERR_ALIGNMENT = -2,
+    ECCO_ERR_NONFINITE_INPUT = -3,
+    ECCO_ERR_BAD_META = -4,
+    ECCO_ERR_UNSUPPORTED_ARCH = -5,
+    ECCO_ERR_CUDA = -6,             /* see ecco_last_cuda_error() */
+    ECCO_ERR_WORKSPACE = -7,        /* workspace too small */
+    ECCO_ERR_DEVICE_TIMEOUT = -8    /* a bounded device-side wait gave up (ecco_device_status) */
+};
+
+/* flags of ecco_encode_host / ecco_params.select */
+#define ECCO_SELECT_MSE 0u        /* Fig. 4 step 5: pattern with the least squared error (weights) */
+#define ECCO_SELECT_MINMAX 1u     /* Sec. 4.3: min/max fitness (online KV path) */
+#define ECCO_KEEP_EXPONENT 2u     /* keep the metadata's exponent e instead of refitting it */
+
+typedef struct ecco_meta ecco_meta;   /* opaque per-tensor metadata (Sec. 4.2: "tensor-wise metadata") */
+
+typedef struct {
+    int32_t S;                  /* shared patterns, 2..64 */
+    int32_t H;                  /* must be 4 */
+    uint64_t seed;              /* seeds the k-means initialisations */
+    uint32_t select;            /* ECCO_SELECT_MSE or ECCO_SELECT_MINMAX for step 5 of calibration */
+    int32_t kmeans_iters;       /* iteration cap of every Lloyd loop (0 = 25) */
+    uint64_t max_groups;        /* calibrate on at most this many groups, evenly strided (0 = all) */
+    int32_t threads;            /* worker threads (0 = all available cores) */
+} ecco_params;
+
+typedef struct {
+    uint64_t n_groups;
+    uint64_t clipped_groups;    /* groups that lost at least one value to clipping */
+    uint64_t clipped_values;
+    uint64_t padded_groups;
+    uint64_t padded_values;
+    uint64_t total_bits;        /* header + stored codewords, summed over groups */
+    uint64_t kp_usage[ECCO_MAX_PATTERNS];
+    uint64_t hf_usage[ECCO_CODEBOOKS];
+    uint64_t sym_count[16];
+} ecco_stats;
+
+/* ---------------------------------------------------------------- host, blocking */
+
+/* Fig. 4 steps 1-7 on a calibration tensor of n_groups*128 fp16 values (host): per-group
+ * 15-means patterns, S shared patterns, H codebooks per pattern (lengths 2..8, Sec. 4.2) and the
+ * ID_KP code.  elem_weights_or_null: 128 non-negative weights applied to every group in step 3
+ * ("activation-aware"), or NULL.  *out_meta is owned by the caller (ecco_meta_free). */
+int ecco_calibrate_host(const uint16_t* calib_fp16, uint64_t n_groups, const float* elem_weights_or_null,
+                        const ecco_params* params, ecco_meta** out_meta);
+
+/* Metadata from explicit tables (host arrays): patterns [S][15] fp16 ascending, cb_len [S][4][16]
+ * in 2..8 with Kraft sum 1, kp_len [S] in 1..12 with Kraft sum 1, exponent e in [-32, 16].
+ * Returns ECCO_ERR_BAD_META if any table is inconsistent. */
+int ecco_meta_create(int32_t S, int32_t e, const uint16_t* patterns, const uint8_t* cb_len, const uint8_t* kp_len,
+                     ecco_meta** out_meta);
+/* Copies the tables out (any output pointer may be NULL). */
+int ecco_meta_get(const ecco_meta* meta, int32_t* S, int32_t* e, uint16_t* patterns, uint8_t* cb_len, uint8_t* kp_len);
+void ecco_meta_free(ecco_meta* meta);
+
+/* Fig. 4 steps 2, 5, 8, 9 (and Sec. 4.3 for ECCO_SELECT_MINMAX): encodes n_groups*128 fp16 host
+ * values into n_groups*64 bytes at dst_blocks (host, caller-owned).  Unless ECCO_KEEP_EXPONENT is
+ * set, first refits meta's exponent e to this tensor (smallest e with max|x| <= 448*2^e).
+ * Non-finite input gives ECCO_ERR_NONFINITE_INPUT.  Runs on all available cores. */
+int ecco_encode_host(ecco_meta* meta, const uint16_t* src_fp16, uint64_t n_groups, uint32_t flags,
+                     uint8_t* dst_blocks, ecco_stats* stats_or_null);
+
+/* Device image of the metadata (Sec. 4.2: loaded once before the compressed loads): header,
+ * patterns, and the prebuilt decode tables.  The caller copies `bytes` bytes from host_staging to
+ * 16-byte aligned device memory and passes that pointer as d_meta. */
+size_t ecco_meta_device_bytes(const ecco_meta* meta);
+int ecco_meta_serialize_device(const ecco_meta* meta, void* host_staging, size_t bytes);
+
+/* ---------------------------------------------------------------- device, asynchronous */
+
+/* Sec. 4.2 (pattern retriever, Huffman decode, outlier handling, mapper): n_groups blocks at
+ * d_blocks -> n_groups*128 fp16 at d_out_fp16.  Value = fp16_rn(fp32(centroid) * fp32(scale));
+ * clipped positions read +0.  n_groups == 0 is a no-op. */
+int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out_fp16, void* stream);
+
+/* Decode-phase GEMV on compressed weights (Sec. 2.1: M = 1 matrix-vector products; Sec. 4.2
+ * decode): y[b][n] = sum_k W~[n][k] * x[b][k], fp32 accumulation.  W is row-major [n_out][k],
+ * groups along k, block of (n, kblock) at byte 64*(n*(k/128) + kblock).  x is fp16 [batch][k],
+ * y is fp32 [batch][n_out], batch in 1..8, k a multiple of 128.  d_workspace: device scratch of
+ * at least ecco_gemv_workspace_bytes(n_out, k, batch) bytes, 16-byte aligned, contents
+ * irrelevant before and undefined after; calls sharing a workspace must not overlap. */
+size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch);
+int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x_fp16,
+              int32_t batch, float* d_y, void* d_workspace, size_t workspace_bytes, void* stream);
+
+/* Fused attention scores over a compressed K cache (Eq. 3: Q K^T / sqrt(d_k), without the
+ * softmax): scores[b][hq][t] = scale * sum_d q[b][hq][d] * K~[b][hq / q_per_kv][t][d].  One group
+ * is the 128-wide head vector of one token; blocks are ordered [batch][n_kv_heads][seq]; q is
+ * fp16 [batch][n_kv_heads*q_per_kv][128]; scores fp32 [batch][n_kv_heads*q_per_kv][seq];
+ * q_per_kv in 1..8. */
+int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
+                     int32_t q_per_kv, const void* d_q_fp16, float scale, float* d_scores, void* stream);
+
+/* ---------------------------------------------------------------- diagnostics */
+const char* ecco_error_string(int code);
+int ecco_last_cuda_error(void);        /* cudaError_t of the last ECCO_ERR_CUDA on this thread */
+/* Synchronises the device and reads the library's device-side status word: 0, or
+ * ECCO_ERR_DEVICE_TIMEOUT if a kernel's bounded wait on a bulk copy expired (its output is then
+ * undefined).  Clears the word. */
+int ecco_device_status(void);
+/* Number of kernels the library has launched in this process (diagnostic counter). */
+uint64_t ecco_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ECCO_H_ */

@@ -1,0 +1,45 @@
+"""Builds the C-ABI shared library (CUDA kernels for sm_100a + host encoder) in-tree with nvcc."""
+from __future__ import annotations
+
+import os
+import shutil
+import subprocess
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+CSRC = os.path.join(HERE, "csrc")
+LIB = os.path.join(HERE, "libecco_b200.so")
+SOURCES = [os.path.join(CSRC, "ecco_kernels.cu"), os.path.join(CSRC, "ecco_host.cpp")]
+HEADERS = [os.path.join(CSRC, "ecco_format.h"), os.path.join(os.path.dirname(HERE), "include", "ecco.h")]
+
+
+def nvcc_path() -> str:
+    for cand in (shutil.which("nvcc"), "/usr/local/cuda/bin/nvcc"):
+        if cand and os.path.exists(cand):
+            return cand
+    raise RuntimeError("nvcc not found: the library has no CPU fallback and cannot be built without the CUDA toolkit")
+
+
+def is_stale() -> bool:
+    if not os.path.exists(LIB):
+        return True
+    t = os.path.getmtime(LIB)
+    return any(os.path.getmtime(f) > t for f in SOURCES + HEADERS)
+
+
+def build_library(force: bool = False, verbose: bool = False) -> str:
+    """nvcc -gencode arch=compute_100a,code=sm_100a ... -> libecco_b200.so next to this file."""
+    if not force and not is_stale():
+        return LIB
+    cmd = [
+        nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+        "-Xcompiler", "-fPIC,-ffp-contract=off,-Wall,-pthread", "-shared", "-o", LIB, *SOURCES,
+    ]
+    if verbose:
+        cmd.insert(1, "-Xptxas")
+        cmd.insert(2, "-v")
+    subprocess.check_call(cmd)
+    return LIB
+
+
+if __name__ == "__main__":
+    print(build_library(force=True, verbose=True))

@@ -1,0 +1,46 @@
+// ecco_format.h -- constants of the 64-byte block and of the device metadata image, shared by
+// the host encoder and the CUDA kernels of this library (never by the test oracle).
+#pragma once
+#include <cstdint>
+
+namespace ecco {
+
+constexpr int kGroup = 128;        // values per group (Sec. 3.1)
+constexpr int kBlockBytes = 64;    // bytes per block (Sec. 3.1)
+constexpr int kBlockBits = 512;
+constexpr int kCentroids = 15;     // Sec. 3.2
+constexpr int kSymbols = 16;       // 15 centroid indices + index 15 = the abs-max
+constexpr int kMaxPatterns = 64;   // S
+constexpr int kCodebooks = 4;      // H
+constexpr int kMinLen = 2, kMaxLen = 8;   // Sec. 4.2
+constexpr int kKpMaxLen = 12;      // limit of the ID_KP code
+constexpr int kPadBits = 15;       // 7-bit location + FP8 value (Sec. 3.2)
+constexpr int kMaxPads = 16;       // the sorter's top 16 (Sec. 4.3)
+constexpr int kHeaderBits = 10;    // scale byte + ID_HF
+constexpr int kExpMin = -32, kExpMax = 16;
+
+// Device image of the per-tensor metadata.  The tables follow the 64-byte header back to back
+// so that one bulk copy brings them into shared memory.
+constexpr uint32_t kDevMagic = 0x4F434345u;  // "ECCO"
+constexpr uint32_t kDevVersion = 1;
+struct DevHeader {
+    uint32_t magic, version;
+    int32_t S, H, e;
+    float T;                 // 2^e
+    uint32_t total_bytes;
+    uint32_t reserved[9];
+};
+static_assert(sizeof(DevHeader) == 64, "header is 64 bytes");
+
+constexpr uint32_t kOffPattern = 64;                                  // [64][16] fp16, entry 15 = 0
+constexpr uint32_t kPatternBytes = kMaxPatterns * 16 * 2;
+constexpr uint32_t kOffKpLut = kOffPattern + kPatternBytes;           // [4096] u16: kp | len << 8
+constexpr uint32_t kKpLutBytes = (1u << kKpMaxLen) * 2;
+constexpr uint32_t kOffSymLut = kOffKpLut + kKpLutBytes;              // [S*H = 256][256] u8: len << 4 | sym
+constexpr uint32_t kSymLutBytes = kMaxPatterns * kCodebooks * 256;
+constexpr uint32_t kDevBytes = kOffSymLut + kSymLutBytes;             // 75840
+constexpr uint32_t kTableBytes = kDevBytes - kOffPattern;             // 75776, a multiple of 16
+// Both lookup tables are indexed by the next stream bits with the first stream bit in bit 0,
+// i.e. by the bit-reversed codeword followed by whatever comes next.
+
+}  // namespace ecco

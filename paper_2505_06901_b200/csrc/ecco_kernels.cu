@@ -1,0 +1,701 @@
+// ecco_kernels.cu -- sm_100a kernels and the device half of the C ABI.
+//
+// One thread owns one group: a 64-byte block is independent of every other block (Sec. 3.2,
+// "all group-wise information ... compressed to a fixed compressed block size"), so the decoder
+// runs the serial Huffman chain (Sec. 4.2) once per thread and takes its parallelism across
+// groups, not inside a group.  The lanes of a warp advance symbol by symbol in lock step, which
+// keeps every per-symbol index (output position, activation element) uniform across the warp.
+//
+// Shared memory per CTA:
+//   tables   pattern[64][16] fp16 | ID_KP table [4096] u16 | symbol tables [256][256] u8,
+//            brought in by one bulk copy (cp.async.bulk + mbarrier)
+//   per warp bits[18][32] u32   the warp's 32 blocks, word-transposed: lane L's word w at
+//                               [w][L] -> bank L whatever w is (conflict-free refills);
+//                               rows 16 and 17 stay zero (stream bits past 512 read as 0)
+//            tab[16][32]  u32   per-lane dequantised centroids (entry 15 = the abs-max)
+//            syms[16][32] u32   (fused kernels) decoded indices, 8 nibbles per word, for the
+//                               outlier fix-up
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <cstdio>
+
+#include "../../include/ecco.h"
+#include "ecco_format.h"
+
+using namespace ecco;
+
+namespace {
+
+__device__ int g_device_status = 0;            // sticky: ECCO_ERR_DEVICE_TIMEOUT if a bounded wait expired
+thread_local int t_last_cuda_error = 0;
+std::atomic<uint64_t> g_launches{0};
+
+constexpr uint32_t kSmemPattern = 0;
+constexpr uint32_t kSmemKpLut = kPatternBytes;
+constexpr uint32_t kSmemSymLut = kPatternBytes + kKpLutBytes;        // 10240: 256-aligned
+constexpr uint32_t kSmemWarpBase = kTableBytes;                      // 75776: 1024-aligned
+constexpr uint32_t kBitsRows = 18;
+constexpr uint32_t kBitsBytes = kBitsRows * 32 * 4;                  // 2304
+constexpr uint32_t kTabBytes = 16 * 32 * 4;                          // 2048
+constexpr uint32_t kSymsBytes = 16 * 32 * 4;                         // 2048
+constexpr int kWaitLimit = 1 << 22;                                  // bounded mbarrier polling
+
+// ---------------------------------------------------------------------------------------------
+// small PTX helpers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// 1-D bulk copy global -> shared (TMA engine, no tensor map, no multicast); both addresses and
+// the size are multiples of 16 bytes
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
+__device__ __forceinline__ uint4 ldg_nc_v4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void stg_v8(void* p, const uint32_t (&r)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
+                 "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+// OCP E4M3 byte -> fp32, arithmetically (the all-ones exponent/mantissa code reads as 480)
+__device__ __forceinline__ float fp8_to_float(uint32_t b)
+{
+    uint32_t ex = (b >> 3) & 15u, man = b & 7u;
+    float mag = ex ? __uint_as_float(((ex + 120u) << 23) | (man << 20)) : static_cast<float>(man) * 0.001953125f;
+    return (b & 0x80u) ? -mag : mag;
+}
+__device__ __forceinline__ uint32_t f2h_bits(float f) { return static_cast<uint32_t>(__half_as_ushort(__float2half_rn(f))); }
+
+// ---------------------------------------------------------------------------------------------
+// table staging (Sec. 4.2: metadata "loaded once" before the compressed loads)
+// ---------------------------------------------------------------------------------------------
+// Returns false (CTA-uniform) if the bounded wait expired; the caller must then return.
+__device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+{
+    const uint32_t bar = smem_u32(bar_storage);
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        mbar_expect_tx(bar, kTableBytes);
+        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kTableBytes, bar);
+    }
+    bool done = false;
+    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+    if (!done)                                   // second, bounded chance for the copy in flight
+        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+    const bool all = __syncthreads_and(done);
+    if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
+    return all;
+}
+
+// ---------------------------------------------------------------------------------------------
+// the per-group decoder
+// ---------------------------------------------------------------------------------------------
+struct WarpSmem {
+    uint32_t bits;      // shared address of bits[0][lane]
+    uint32_t tab;       // shared address of tab[0][lane]
+    uint32_t syms;      // shared address of syms[0][lane] (fused kernels only)
+};
+
+struct GroupHeader {
+    uint32_t pos;       // first bit of the coded indices
+    uint32_t lut;       // shared address of the symbol table of (ID_KP, ID_HF)
+};
+
+// Pattern retriever (Sec. 4.2): scale byte, ID_HF, Huffman-coded ID_KP; writes the lane's 16
+// dequantised values (fp16 bits, or fp32 bits when kFloatTab) and the transposed bit stream.
+template <bool kFloatTab>
+__device__ __forceinline__ GroupHeader open_group(const uint4 (&blk)[4], uint32_t smem_base, const WarpSmem& ws, float T)
+{
+    const uint32_t w[16] = {blk[0].x, blk[0].y, blk[0].z, blk[0].w, blk[1].x, blk[1].y, blk[1].z, blk[1].w,
+                            blk[2].x, blk[2].y, blk[2].z, blk[2].w, blk[3].x, blk[3].y, blk[3].z, blk[3].w};
+#pragma unroll
+    for (int i = 0; i < 16; ++i) sts_u32(ws.bits + i * 128, w[i]);
+    const uint32_t qs = w[0] & 0xffu, hf = (w[0] >> 8) & 3u;
+    const uint32_t kpw = __funnelshift_r(w[0], w[1], 10) & 0xfffu;
+    uint32_t kpe;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=r"(kpe) : "r"(smem_base + kSmemKpLut + kpw * 2));
+    const uint32_t kp = kpe & 0xffu;
+    GroupHeader h;
+    h.pos = kHeaderBits + (kpe >> 8);
+    h.lut = smem_base + kSmemSymLut + (kp * kCodebooks + hf) * 256;
+    const float top = fp8_to_float(qs) * T;           // FP8 -> FP16 range by the power-of-two factor
+    const float s = fabsf(top);
+    uint4 p0, p1;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(p0.x), "=r"(p0.y), "=r"(p0.z), "=r"(p0.w) : "r"(smem_base + kSmemPattern + kp * 32));
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(p1.x), "=r"(p1.y), "=r"(p1.z), "=r"(p1.w) : "r"(smem_base + kSmemPattern + kp * 32 + 16));
+    const uint32_t pr[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+        const __half c = __ushort_as_half(static_cast<unsigned short>((pr[j >> 1] >> ((j & 1) * 16)) & 0xffffu));
+        // mapper (Sec. 4.2): one fp32 product, one rounding to fp16
+        const __half v = __float2half_rn(j < 15 ? __half2float(c) * s : top);
+        sts_u32(ws.tab + j * 128, kFloatTab ? __float_as_uint(__half2float(v)) : static_cast<uint32_t>(__half_as_ushort(v)));
+    }
+    return h;
+}
+
+// Decodes the 128 indices of the lane's group (Sec. 4.2, Huffman decode) and hands each value to
+// sink(n, value_bits, symbol).  A codeword that would cross bit 512 ends the group: that and all
+// later positions are delivered as zero (clipped).  Returns the end bit if all 128 fitted, else 0.
+template <class Sink>
+__device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const WarpSmem& ws, Sink&& sink)
+{
+    uint32_t pos = h.pos;
+    bool alive = true;
+#pragma unroll 4
+    for (int step = 0; step < 32; ++step) {
+        const uint32_t wi = min(pos >> 5, 16u);
+        const uint32_t lo = lds_u32(ws.bits + wi * 128), hi = lds_u32(ws.bits + wi * 128 + 128);
+        const uint32_t win = __funnelshift_r(lo, hi, pos);           // 32 stream bits from pos
+        const uint32_t limit = kBlockBits - min(pos, static_cast<uint32_t>(kBlockBits));
+        uint32_t acc = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t e = lds_u8(h.lut + ((win >> acc) & 0xffu));
+            acc += e >> 4;
+            alive = alive && (acc <= limit);
+            const uint32_t v = lds_u32(ws.tab + (e & 15u) * 128);
+            sink(step * 4 + j, alive ? v : 0u, e & 15u);
+        }
+        pos += acc;
+    }
+    return alive ? pos : 0u;
+}
+
+// Outlier fields (Sec. 3.2: 7-bit location + FP8 value, quantised with the per-tensor factor):
+// pad j sits at bits [512-15(j+1), 512-15j).
+__device__ __forceinline__ uint32_t read_pad(const WarpSmem& ws, int j)
+{
+    const uint32_t bitpos = kBlockBits - kPadBits * (j + 1);
+    const uint32_t wi = bitpos >> 5;
+    const uint32_t lo = lds_u32(ws.bits + wi * 128), hi = lds_u32(ws.bits + wi * 128 + 128);
+    return __funnelshift_r(lo, hi, bitpos) & 0x7fffu;
+}
+
+// ---------------------------------------------------------------------------------------------
+// K1: ecco_decompress
+// ---------------------------------------------------------------------------------------------
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
+                       uint16_t* __restrict__ d_out)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t smem_base = smem_u32(smem);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * (kBitsBytes + kTabBytes) + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = 0;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+
+    const uint64_t tile = static_cast<uint64_t>(kWarps) * 32u;
+    uint64_t g = blockIdx.x * tile + threadIdx.x;
+    uint4 blk[4];
+    if (g < n_groups) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(d_blocks + g * kBlockBytes + i * 16);
+    }
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    for (; g < n_groups; g += gridDim.x * tile) {
+        const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
+        const uint64_t gn = g + gridDim.x * tile;
+        if (gn < n_groups) {                               // next block in flight while this one decodes
+#pragma unroll
+            for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(d_blocks + gn * kBlockBytes + i * 16);
+        }
+        uint16_t* out = d_out + g * kGroup;
+        uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t) {
+            const int slot = (n & 15) >> 1;
+            if (n & 1) r[slot] |= v << 16; else r[slot] = v;
+            if ((n & 15) == 15) stg_v8(out + (n - 15), r);
+        });
+        if (end) {
+            const int n_pad = min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits));
+            for (int j = 0; j < n_pad; ++j) {
+                const uint32_t f = read_pad(ws, j);
+                // same thread, same address as the vector store above: program order holds
+                out[f & 127u] = static_cast<uint16_t>(f2h_bits(fp8_to_float(f >> 7) * T));
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// K2/K3: fused consumers.  kV = number of dot products per group (batch rows of x, or query
+// heads per KV head).  The vector slice xs[128][kV] fp32 lives in shared memory; every lane reads
+// the same element at the same time (broadcast).
+// ---------------------------------------------------------------------------------------------
+template <int kV>
+struct Accum {
+    float a[kV];
+    __device__ __forceinline__ void clear()
+    {
+#pragma unroll
+        for (int v = 0; v < kV; ++v) a[v] = 0.0f;
+    }
+    __device__ __forceinline__ void fma(float w, uint32_t xs_addr)
+    {
+        if constexpr (kV == 1) {
+            float x;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(xs_addr));
+            a[0] = fmaf(w, x, a[0]);
+        } else if constexpr (kV == 2) {
+            float x0, x1;
+            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(x0), "=f"(x1) : "r"(xs_addr));
+            a[0] = fmaf(w, x0, a[0]);
+            a[1] = fmaf(w, x1, a[1]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < kV / 4; ++q) {
+                float x0, x1, x2, x3;
+                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(xs_addr + q * 16));
+                a[q * 4 + 0] = fmaf(w, x0, a[q * 4 + 0]);
+                a[q * 4 + 1] = fmaf(w, x1, a[q * 4 + 1]);
+                a[q * 4 + 2] = fmaf(w, x2, a[q * 4 + 2]);
+                a[q * 4 + 3] = fmaf(w, x3, a[q * 4 + 3]);
+            }
+        }
+    }
+};
+
+// decode one group and accumulate its kV dot products against xs (shared address of xs[0][0])
+template <int kV>
+__device__ __forceinline__ void fused_group(const uint4 (&blk)[4], uint32_t smem_base, const WarpSmem& ws, float T,
+                                            uint32_t xs, Accum<kV>& acc)
+{
+    const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
+    uint32_t packed = 0;
+    const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym) {
+        acc.fma(__uint_as_float(v), xs + n * (kV * 4));
+        packed |= sym << ((n & 7) * 4);
+        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+    });
+    if (end) {
+        // outliers replace the mapped value at their location: add (outlier - mapped) * x
+        const int n_pad = min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits));
+        uint64_t seen_lo = 0, seen_hi = 0;                  // 128-bit "already replaced" mask
+        for (int j = n_pad - 1; j >= 0; --j) {             // the last pad wins on a duplicate location
+            const uint32_t f = read_pad(ws, j);
+            const uint32_t loc = f & 127u;
+            const uint64_t bit = 1ull << (loc & 63u);
+            const bool upper = loc >= 64u;
+            if ((upper ? seen_hi : seen_lo) & bit) continue;
+            if (upper) seen_hi |= bit; else seen_lo |= bit;
+            const uint32_t word = lds_u32(ws.syms + (loc >> 3) * 128);
+            const uint32_t sym = (word >> ((loc & 7u) * 4)) & 15u;
+            const float mapped = __uint_as_float(lds_u32(ws.tab + sym * 128));
+            const float outlier = __half2float(__float2half_rn(fp8_to_float(f >> 7) * T));
+            acc.fma(outlier - mapped, xs + loc * (kV * 4));
+        }
+    }
+}
+
+// K2: y[b][n] = sum_k W~[n][k] x[b][k].  A CTA owns kWarps*32 rows and a contiguous range of
+// k-blocks; a thread owns one row and walks the range.  Partial sums go to the workspace
+// [ksplit][kV][n_out]; the last CTA of a row tile (ticket counter) adds them in a fixed order,
+// so the result does not depend on scheduling.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                 const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+                 unsigned int* __restrict__ d_tickets, int ksplit)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    __shared__ unsigned int ticket;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t smem_base = smem_u32(smem);
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    constexpr uint32_t kXsBytes = kGroup * kV * 4;
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    float* xs_ptr = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);   // two slices
+    const uint32_t xs_base = smem_u32(xs_ptr);
+
+    const int row_tile = blockIdx.x, split = blockIdx.y;
+    const int row = row_tile * (kWarps * 32) + static_cast<int>(threadIdx.x);
+    const bool row_ok = row < n_out;
+    const int kb_lo = static_cast<int>(static_cast<int64_t>(kblocks) * split / ksplit);
+    const int kb_hi = static_cast<int>(static_cast<int64_t>(kblocks) * (split + 1) / ksplit);
+    const int k = kblocks * kGroup;
+
+    uint4 blk[4];
+    const uint8_t* row_blocks = d_blocks + static_cast<uint64_t>(row_ok ? row : 0) * kblocks * kBlockBytes;
+    if (row_ok && kb_lo < kb_hi) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(row_blocks + static_cast<uint64_t>(kb_lo) * kBlockBytes + i * 16);
+    }
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    Accum<kV> acc;
+    acc.clear();
+    for (int kb = kb_lo; kb < kb_hi; ++kb) {
+        // stage x[b][kb*128 .. +128) as fp32 xs[i][b] (rows beyond `batch` are zero)
+        float* xs = xs_ptr + ((kb - kb_lo) & 1) * (kGroup * kV);
+        for (int i = threadIdx.x; i < kGroup * kV; i += kWarps * 32) {
+            const int b = i % kV, e = i / kV;
+            xs[i] = (b < batch) ? __half2float(d_x[static_cast<size_t>(b) * k + kb * kGroup + e]) : 0.0f;
+        }
+        __syncthreads();                                   // slice visible; the other slice is free again
+        if (row_ok) {
+            uint4 cur[4] = {blk[0], blk[1], blk[2], blk[3]};
+            if (kb + 1 < kb_hi) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(row_blocks + static_cast<uint64_t>(kb + 1) * kBlockBytes + i * 16);
+            }
+            fused_group<kV>(cur, smem_base, ws, T, xs_base + ((kb - kb_lo) & 1) * kXsBytes, acc);
+        }
+    }
+    if (ksplit == 1) {
+        if (row_ok) {
+#pragma unroll
+            for (int b = 0; b < kV; ++b)
+                if (b < batch) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
+        }
+        return;
+    }
+    if (row_ok)
+#pragma unroll
+        for (int b = 0; b < kV; ++b)
+            if (b < batch) d_partial[(static_cast<size_t>(split) * kV + b) * n_out + row] = acc.a[b];
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) ticket = atomicAdd(&d_tickets[row_tile], 1u);
+    __syncthreads();
+    if (ticket != static_cast<unsigned int>(ksplit - 1)) return;
+    __threadfence();
+    if (row_ok)
+        for (int b = 0; b < batch; ++b) {
+            float s = 0.0f;
+            for (int sp = 0; sp < ksplit; ++sp) s += __ldcg(&d_partial[(static_cast<size_t>(sp) * kV + b) * n_out + row]);
+            d_y[static_cast<size_t>(b) * n_out + row] = s;
+        }
+    if (threadIdx.x == 0) d_tickets[row_tile] = 0;         // ready for the next call on this workspace
+}
+
+// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / kV][t].  A CTA owns one (batch, kv head)
+// pair and a run of kWarps*32 tokens per iteration; a thread owns one token.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int seq, int q_per_kv,
+                        const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores, int chunks_per_head)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t smem_base = smem_u32(smem);
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    float* xs = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);
+    const uint32_t xs_addr = smem_u32(xs);
+
+    const int bh = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;   // bh = b * n_kv_heads + h
+    const int tile = kWarps * 32;
+    int t = chunk * tile + static_cast<int>(threadIdx.x);
+    const uint8_t* head_blocks = d_kblocks + static_cast<uint64_t>(bh) * seq * kBlockBytes;
+    uint4 blk[4];
+    if (t < seq) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(head_blocks + static_cast<uint64_t>(t) * kBlockBytes + i * 16);
+    }
+    // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
+    for (int i = threadIdx.x; i < kGroup * kV; i += tile) {
+        const int r = i % kV, d = i / kV;
+        xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
+    }
+    if (!stage_tables(smem, d_meta, &bar)) return;        // also orders the xs writes (barrier inside)
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    for (; t < seq; t += chunks_per_head * tile) {
+        uint4 cur[4] = {blk[0], blk[1], blk[2], blk[3]};
+        const int tn = t + chunks_per_head * tile;
+        if (tn < seq) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(head_blocks + static_cast<uint64_t>(tn) * kBlockBytes + i * 16);
+        }
+        Accum<kV> acc;
+        acc.clear();
+        fused_group<kV>(cur, smem_base, ws, T, xs_addr, acc);
+#pragma unroll
+        for (int r = 0; r < kV; ++r)
+            if (r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = acc.a[r];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host-side launch helpers
+// ---------------------------------------------------------------------------------------------
+struct DeviceInfo {
+    int device = -1, sms = 0, cc_major = 0;
+    bool ok = false;
+};
+
+int device_info(DeviceInfo* out)
+{
+    static thread_local DeviceInfo cache[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return ECCO_ERR_INVALID_ARG;
+    DeviceInfo& c = cache[dev];
+    if (!c.ok) {
+        cudaDeviceProp prop;
+        e = cudaGetDeviceProperties(&prop, dev);
+        if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+        c.device = dev; c.sms = prop.multiProcessorCount; c.cc_major = prop.major; c.ok = true;
+    }
+    *out = c;
+    return c.cc_major == 10 ? ECCO_OK : ECCO_ERR_UNSUPPORTED_ARCH;
+}
+
+template <class K>
+int set_smem(K kernel, size_t bytes)
+{
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    return ECCO_OK;
+}
+
+int check_launch()
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ECCO_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+constexpr int kDecompressWarps = 32;
+constexpr int kFusedWarps = 16;
+
+struct GemvPlan { int row_tiles, ksplit; size_t partial_bytes, ticket_bytes; };
+
+GemvPlan gemv_plan(int n_out, int kblocks, int vpad, int sms)
+{
+    GemvPlan p;
+    const int rows_per_cta = kFusedWarps * 32;
+    p.row_tiles = (n_out + rows_per_cta - 1) / rows_per_cta;
+    // enough k-splits to give every SM a CTA, at most one per k-block
+    int want = (sms + p.row_tiles - 1) / p.row_tiles;
+    p.ksplit = want < 1 ? 1 : (want > kblocks ? kblocks : want);
+    p.partial_bytes = p.ksplit > 1 ? static_cast<size_t>(p.ksplit) * vpad * n_out * sizeof(float) : 0;
+    p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return p;
+}
+
+inline int pad_v(int v) { return v <= 1 ? 1 : v <= 2 ? 2 : v <= 4 ? 4 : 8; }
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+extern "C" int ecco_last_cuda_error(void) { return t_last_cuda_error; }
+extern "C" uint64_t ecco_kernel_launch_count(void) { return g_launches.load(); }
+
+extern "C" int ecco_device_status(void)
+{
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    int st = 0, zero = 0;
+    e = cudaMemcpyFromSymbol(&st, g_device_status, sizeof st);
+    if (e == cudaSuccess && st) e = cudaMemcpyToSymbol(g_device_status, &zero, sizeof zero);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    return st;
+}
+
+extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out, void* stream)
+{
+    if (n_groups == 0) return ECCO_OK;
+    if (!d_meta || !d_blocks || !d_out) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_out)) return ECCO_ERR_ALIGNMENT;
+    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    auto kernel = ecco_decompress_kernel<kDecompressWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kDecompressWarps) * (kBitsBytes + kTabBytes);
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    const uint64_t tile = kDecompressWarps * 32;
+    const uint64_t tiles = (n_groups + tile - 1) / tile;
+    const unsigned grid = static_cast<unsigned>(tiles < static_cast<uint64_t>(di.sms) ? tiles : di.sms);
+    kernel<<<grid, kDecompressWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out));
+    return check_launch();
+}
+
+extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch)
+{
+    if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return 0;
+    // sized for the largest plan any supported device can ask for (k-split count <= 256)
+    const int rows_per_cta = kFusedWarps * 32;
+    const int row_tiles = (n_out + rows_per_cta - 1) / rows_per_cta;
+    const int kblocks = k / kGroup;
+    const int ksplit = kblocks < 256 ? kblocks : 256;
+    size_t partial = (static_cast<size_t>(ksplit) * pad_v(batch) * n_out * sizeof(float) + 255) & ~static_cast<size_t>(255);
+    size_t tickets = (static_cast<size_t>(row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return partial + tickets;
+}
+
+template <int kV>
+static int launch_gemv(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
+                       const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+{
+    auto kernel = ecco_gemv_kernel<kV, kFusedWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + 2 * kGroup * kV * 4;
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        int rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    const GemvPlan p = gemv_plan(n_out, kblocks, kV, di.sms);
+    float* partial = nullptr;
+    unsigned int* tickets = nullptr;
+    if (p.ksplit > 1) {
+        if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
+        if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
+        partial = static_cast<float*>(d_ws);
+        tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
+        // the workspace's previous contents are irrelevant: tickets start from zero on every call
+        cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
+        if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    }
+    dim3 grid(static_cast<unsigned>(p.row_tiles), static_cast<unsigned>(p.ksplit));
+    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
+                                                     static_cast<const __half*>(d_x), batch, d_y, partial, tickets, p.ksplit);
+    return check_launch();
+}
+
+extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x,
+                         int32_t batch, float* d_y, void* d_workspace, size_t workspace_bytes, void* stream)
+{
+    if (!d_meta || !d_blocks || !d_x || !d_y) return ECCO_ERR_INVALID_ARG;
+    if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_x) || !aligned16(d_y)) return ECCO_ERR_ALIGNMENT;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int kblocks = k / kGroup;
+    switch (pad_v(batch)) {
+        case 1: return launch_gemv<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+        case 2: return launch_gemv<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+        case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+        default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+    }
+}
+
+template <int kV>
+static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* d_kblocks, int batch, int n_kv_heads,
+                       int seq, int q_per_kv, const void* d_q, float scale, float* d_scores, cudaStream_t stream)
+{
+    auto kernel = ecco_attn_scores_kernel<kV, kFusedWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + kGroup * kV * 4;
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        int rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    const int tile = kFusedWarps * 32;
+    const int heads = batch * n_kv_heads;
+    const int max_chunks = (seq + tile - 1) / tile;
+    // about two CTAs per SM in total, at least one per head, at most one per tile of tokens
+    int chunks = (2 * di.sms + heads - 1) / heads;
+    chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
+    const unsigned grid = static_cast<unsigned>(heads) * static_cast<unsigned>(chunks);
+    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, seq, q_per_kv,
+                                                     static_cast<const __half*>(d_q), scale, d_scores, chunks);
+    return check_launch();
+}
+
+extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
+                                int32_t q_per_kv, const void* d_q, float scale, float* d_scores, void* stream)
+{
+    if (batch == 0 || n_kv_heads == 0 || seq == 0) return (batch < 0 || n_kv_heads < 0 || seq < 0) ? ECCO_ERR_INVALID_ARG : ECCO_OK;
+    if (!d_meta || !d_kblocks || !d_q || !d_scores) return ECCO_ERR_INVALID_ARG;
+    if (batch < 0 || n_kv_heads < 0 || seq < 0 || q_per_kv < 1 || q_per_kv > 8) return ECCO_ERR_INVALID_ARG;
+    if (static_cast<int64_t>(batch) * n_kv_heads > (1 << 24)) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_kblocks) || !aligned16(d_q) || !aligned16(d_scores)) return ECCO_ERR_ALIGNMENT;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (pad_v(q_per_kv)) {
+        case 1: return launch_attn<1>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
+        case 2: return launch_attn<2>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
+        case 4: return launch_attn<4>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
+        default: return launch_attn<8>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
+    }
+}

@@ -1,0 +1,188 @@
+"""CPU tests of the library's host half: ABI surface, encoder parity with the oracle (byte for
+byte, given the oracle's metadata), calibrator invariants, decode-table image."""
+import ctypes
+import re
+import os
+
+import numpy as np
+import pytest
+
+from helpers import lib_meta_from_oracle, oracle_meta_from_lib
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="session")
+def binding():
+    from paper_2505_06901_b200 import binding as b
+
+    b.lib()
+    return b
+
+
+def test_library_exports_every_declared_symbol(binding):
+    header = open(os.path.join(ROOT, "include", "ecco.h")).read()
+    declared = set(re.findall(r"\b(ecco_[a-z0-9_]+)\s*\(", header))
+    declared -= {"ecco_meta"}
+    assert declared == set(binding.EXPORTS), declared ^ set(binding.EXPORTS)
+    L = ctypes.CDLL(binding.lib_path())
+    for name in declared:
+        assert hasattr(L, name), name
+    assert ctypes.sizeof(binding.Stats) == 8 * (6 + 64 + 4 + 16)
+    assert binding.lib().ecco_error_string(-3) == b"non-finite input value"
+
+
+def test_argument_errors_without_a_gpu(binding, cfg1_small, eo):
+    L = binding.lib()
+    lm = lib_meta_from_oracle(binding, cfg1_small["meta"])
+    assert L.ecco_decompress(None, None, 0, None, None) == 0                    # empty input is a no-op
+    assert L.ecco_decompress(None, None, 5, None, None) == binding.ERR_INVALID_ARG
+    assert L.ecco_decompress(16, 32, 5, 48 + 1, None) == binding.ERR_ALIGNMENT  # checked before any CUDA call
+    assert L.ecco_gemv(16, 32, 100, 100, 64, 1, 128, None, 0, None) == binding.ERR_INVALID_ARG   # k % 128
+    assert L.ecco_gemv(16, 32, 100, 128, 64, 9, 128, None, 0, None) == binding.ERR_INVALID_ARG   # batch > 8
+    assert L.ecco_attn_scores(16, 32, 1, 1, 8, 9, 64, ctypes.c_float(1.0), 128, None) == binding.ERR_INVALID_ARG
+    assert L.ecco_gemv_workspace_bytes(4096, 4096, 1) >= 4096 * 4 * 32
+    assert L.ecco_gemv_workspace_bytes(4096, 100, 1) == 0
+    # bad metadata tables are refused
+    pat, cb, kp = cfg1_small["meta"].patterns(), cfg1_small["meta"].cb_lengths(), cfg1_small["meta"].kp_lengths()
+    bad_cb = cb.copy(); bad_cb[3, 1, 0] = 9
+    with pytest.raises(binding.EccoError) as ei:
+        binding.ecco_meta_create(64, -9, pat, bad_cb, kp)
+    assert ei.value.code == binding.ERR_BAD_META
+    bad_cb = cb.copy(); bad_cb[3, 1, 0] = 2 if cb[3, 1, 0] != 2 else 3          # breaks the Kraft equality
+    with pytest.raises(binding.EccoError):
+        binding.ecco_meta_create(64, -9, pat, bad_cb, kp)
+    bad_pat = pat.copy(); bad_pat[5, 3], bad_pat[5, 4] = pat[5, 4] + np.float16(0.5), pat[5, 3]
+    with pytest.raises(binding.EccoError):
+        binding.ecco_meta_create(64, -9, bad_pat, cb, kp)
+    x = cfg1_small["w"].copy().reshape(-1); x[77] = np.inf
+    with pytest.raises(binding.EccoError) as ei:
+        binding.ecco_encode_host(lm, x)
+    assert ei.value.code == binding.ERR_NONFINITE_INPUT
+
+
+@pytest.mark.parametrize("which", ["weights_mse", "kv_minmax", "kv_mse"])
+def test_host_encoder_matches_oracle_byte_for_byte(binding, eo, cfg1_small, kv_small, which):
+    if which == "weights_mse":
+        ometa, x, flags, want = cfg1_small["meta"], cfg1_small["w"], binding.SELECT_MSE, cfg1_small["blocks"]
+    elif which == "kv_minmax":
+        ometa, x, flags, want = kv_small["meta"], kv_small["k"], binding.SELECT_MINMAX | binding.KEEP_EXPONENT, kv_small["blocks"]
+    else:
+        ometa, x, flags = kv_small["meta"], kv_small["k"], binding.SELECT_MSE | binding.KEEP_EXPONENT
+        want, _ = eo.encode(ometa, x, eo.SELECT_MSE)
+    lm = lib_meta_from_oracle(binding, ometa)
+    got, st = binding.ecco_encode_host(lm, x, flags)
+    assert lm.tables()[1] == ometa.e
+    bad = np.nonzero((got != want).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} blocks differ, first {bad[:5]}"
+    _, ost = eo.encode(ometa, x, flags & 1)
+    for f in ("n_groups", "clipped_groups", "clipped_values", "padded_groups", "padded_values", "total_bits"):
+        assert getattr(st, f) == getattr(ost, f), f
+    assert list(st.kp_usage) == list(ost.kp_usage) and list(st.sym_count) == list(ost.sym_count)
+
+
+def test_host_encoder_refits_the_exponent_like_the_oracle(binding, eo, cfg1_small):
+    ometa = cfg1_small["meta"].copy()
+    x = (cfg1_small["w"].astype(np.float32) * 37.0).astype(np.float16)
+    eo.set_exponent(ometa, x)
+    assert ometa.e != cfg1_small["meta"].e
+    lm = lib_meta_from_oracle(binding, cfg1_small["meta"])
+    got, _ = binding.ecco_encode_host(lm, x, binding.SELECT_MSE)
+    want, _ = eo.encode(ometa, x, eo.SELECT_MSE)
+    assert lm.tables()[1] == ometa.e and np.array_equal(got, want)
+
+
+def test_host_encoder_on_adversarial_patterns_and_inputs(binding, eo):
+    """Duplicate centroids, distance plateaus, exact midpoints, zero/constant/tiny groups."""
+    rng = np.random.Generator(np.random.PCG64(42))
+    m = eo.Meta()
+    m.S, m.H, m.e = 8, 4, -6
+    base = np.array([-1, -0.5, -0.5, -0.25, -0.25, -0.25, 0, 0, 0.125, 0.25, 0.25, 0.5, 0.5, 1, 1], dtype=np.float64)
+    for k in range(8):
+        pat = np.sort(base * (0.4 + 0.1 * k)) if k % 2 == 0 else np.sort(rng.uniform(-1, 1, 15).round(2))
+        if k == 7:
+            pat = np.zeros(15)
+        for j in range(15):
+            m.pattern[k][j] = int(np.float16(pat[j]).view(np.uint16))
+        m.kp_len[k] = 3
+        for h in range(4):
+            ln = eo.huffman_2_8(rng.dirichlet(np.ones(16) * 0.5))
+            for s in range(16):
+                m.cb_len[k][h][s] = int(ln[s])
+    assert eo.meta_check(m) == 0
+    groups = []
+    grid = np.array([-1, -0.75, -0.5, -0.375, -0.25, -0.125, 0, 0.0625, 0.125, 0.1875, 0.25, 0.375, 0.5, 0.75, 1.0])
+    for t in range(300):
+        g = rng.choice(grid, 128) * rng.choice([0.5, 1.0, 2.0, 0.01])
+        g[rng.integers(128)] = rng.choice([-3.0, 3.0, 2.0])
+        groups.append(g)
+    groups.append(np.zeros(128)); groups.append(np.full(128, 0.25)); groups.append(np.full(128, 2.0 ** -24))
+    groups.append(np.concatenate([np.full(64, 1.0), np.full(64, -1.0)]))
+    x = np.array(groups, dtype=np.float16)
+    for sel in (0, 1):
+        want, _ = eo.encode(m, x, sel)
+        lm = lib_meta_from_oracle(binding, m)
+        got, _ = binding.ecco_encode_host(lm, x, sel | binding.KEEP_EXPONENT)
+        assert np.array_equal(got, want), np.nonzero((got != want).any(axis=1))[0][:5]
+
+
+def test_host_calibrator_yields_valid_and_useful_metadata(binding, eo, synth):
+    cal = synth.weight_matrix(256, 1024, 2001)
+    w = synth.weight_matrix(256, 1024, 1001)
+    lm = binding.ecco_calibrate_host(cal, S=64, H=4, seed=5, select=binding.SELECT_MSE)
+    lm2 = binding.ecco_calibrate_host(cal, S=64, H=4, seed=5, select=binding.SELECT_MSE)
+    S, e, pat, cb, kp = lm.tables()
+    t2 = lm2.tables()
+    assert S == 64 and np.array_equal(pat.view(np.uint16), t2[2].view(np.uint16)) and np.array_equal(cb, t2[3])  # deterministic
+    om = oracle_meta_from_lib(eo, lm)
+    assert eo.meta_check(om) == 0                       # Kraft equality etc., checked by the oracle's validator
+    assert np.all(np.diff(pat.astype(np.float32), axis=1) >= 0) and np.abs(pat.astype(np.float32)).max() <= 1.05
+    blocks, st = binding.ecco_encode_host(lm, w, binding.SELECT_MSE)
+    om.e = lm.tables()[1]
+    out = eo.decode(om, blocks).reshape(w.shape).astype(np.float32)
+    rel = np.sqrt(((out - w.astype(np.float32)) ** 2).mean() / (w.astype(np.float32) ** 2).mean())
+    assert rel < 0.15                                   # same class as the oracle's own calibration (~0.10)
+    assert st.clipped_values / (st.n_groups * 128) < 0.02
+    # the oracle's encoder agrees with the library's on the library's metadata too
+    want, _ = eo.encode(om, w, eo.SELECT_MSE)
+    assert np.array_equal(blocks, want)
+    # sub-sampled calibration and the KV rule run and validate
+    km = binding.ecco_calibrate_host(synth.kv_cache(1, 4, 512, 2003, 3003), S=16, seed=2, select=binding.SELECT_MINMAX,
+                                     max_groups=1024)
+    assert eo.meta_check(oracle_meta_from_lib(eo, km)) == 0 and km.tables()[0] == 16
+    with pytest.raises(binding.EccoError):
+        binding.ecco_calibrate_host(cal[:1, :128 * 8].copy(), S=64)   # fewer groups than patterns
+
+
+def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
+    """The prebuilt lookup tables, read on the CPU: walking a block with them gives the oracle's
+    symbols and end position (checks table layout and bit order without a GPU)."""
+    ometa = cfg1_small["meta"]
+    lm = lib_meta_from_oracle(binding, ometa)
+    img = binding.ecco_meta_serialize_device(lm)
+    assert img.size == binding.ecco_meta_device_bytes(lm) == 75840
+    hdr = img[:64].view(np.uint32)
+    assert hdr[0] == 0x4F434345 and hdr[2] == 64 and hdr[3] == 4 and hdr[4:5].view(np.int32)[0] == ometa.e
+    assert img[20:24].view(np.float32)[0] == 2.0 ** ometa.e
+    pat = img[64:64 + 2048].view(np.float16).reshape(64, 16)
+    assert np.array_equal(pat[:, :15].view(np.uint16), ometa.patterns().view(np.uint16)) and np.all(pat[:, 15] == 0)
+    kpl = img[64 + 2048:64 + 2048 + 8192].view(np.uint16)
+    syml = img[64 + 2048 + 8192:].reshape(256, 256)
+    assert np.all((syml >> 4) >= 2) and np.all((syml >> 4) <= 8)
+    for g in range(0, 2048, 41):
+        blk = cfg1_small["blocks"][g]
+        _, sym, info = eo.decode_block(ometa, blk)
+        bits = int.from_bytes(blk.tobytes(), "little")
+        e = int(kpl[(bits >> 10) & 0xFFF])
+        assert e & 0xFF == info.kp
+        pos = 10 + (e >> 8)
+        lut = syml[info.kp * 4 + info.hf]
+        n = 0
+        while n < 128:
+            t = int(lut[(bits >> pos) & 0xFF])
+            if pos + (t >> 4) > 512:
+                break
+            assert (t & 15) == sym[n]
+            pos += t >> 4
+            n += 1
+        assert n == info.n_fit and pos == info.end_bit
