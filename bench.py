@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the Ecco decompression hot path on B200.
+
+One step = one pass of the whole hot path over the Llama-2-7B-shaped configuration:
+  1. ecco_decompress of the 7 compressed projection matrices of one decoder layer,
+  2. ecco_gemv (fused decode + GEMV) over the same 7 matrices at batch 1,
+  3. the same at batch 8,
+  4. ecco_attn_scores over the layer's compressed K cache [8][32][4096][128], one query per sequence.
+The headline `value` is the fp16 output rate of segment 1 (decompress output GB/s); the other
+segments are reported beside it (GEMV microseconds per layer, attention-score microseconds).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun): every rank runs the same step on its own copy of the workload (the blocks of
+a tensor are independent, so the path shards with no data-path collective: weak scaling); the time
+is the maximum over ranks of the device time, the value the sum of the ranks' bytes over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+G, BLOCK = 128, 64
+METRIC, UNIT = "decompress_output_GBps", "GB/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
+    ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()                  # the exact process started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_blocks(n_groups_wanted: int):
+    """Oracle-only path: calibrate on the config-2 calibration matrix and encode the first rows of the
+    q-projection-shaped matrix with the oracle's own encoder."""
+    from oracle import ecco_oracle as eo
+    from paper_2505_06901_b200 import synth
+
+    cal = synth.weight_matrix(256, 1024, 2002)
+    meta = eo.calibrate(cal, S=64, H=4, seed=2, select=eo.SELECT_MSE)
+    rows = max(1, -(-n_groups_wanted // 32))
+    w = synth.weight_matrix(rows, 4096, 1002 * 16)
+    eo.set_exponent(meta, w)
+    blocks, _ = eo.encode(meta, w.reshape(-1)[: n_groups_wanted * G], eo.SELECT_MSE)
+    return eo, meta, blocks
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    c = cores()
+    total = args.steps + args.warmup
+    # about 60 s for the whole run at ~70k groups/s per core, at most 2^16 groups per step
+    n = int(min(1 << 16, max(2048, 70000 * c * 60 // max(1, total))))
+    n = min(n, 16384)                       # the oracle's own encoder prepares the sample (~1 s per 8k groups)
+    eo, meta, blocks = oracle_sample_blocks(n)
+    for _ in range(args.warmup):
+        eo.decode_threads(meta, blocks, c)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        eo.decode_threads(meta, blocks, c)
+    dt = time.perf_counter() - t0
+    value = n * G * 2 * args.steps / dt / 1e9
+    sample = f"{n} groups of a 4096-wide q-projection-shaped matrix (config-2 distribution), decoded {args.steps}x"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "cfg2 llama2-7b decoder layer + cfg3 K cache (bounded sample, CPU oracle)", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": c, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def cpu_baseline(layer, c: int):
+    """The oracle's decoder on a bounded sample of the benchmark's own blocks (about 15 s of CPU work)."""
+    from oracle import ecco_oracle as eo
+
+    t = layer[0]
+    S, e, pat, cb, kp = t.meta.tables()
+    om = eo.Meta()
+    om.S, om.H, om.e = S, 4, e
+    for k in range(S):
+        om.kp_len[k] = int(kp[k])
+        for j in range(15):
+            om.pattern[k][j] = int(pat.view(np.uint16)[k, j])
+        for h in range(4):
+            for s in range(16):
+                om.cb_len[k][h][s] = int(cb[k, h, s])
+    probe = t.blocks[:4096]
+    t0 = time.perf_counter()
+    eo.decode(om, probe)
+    rate = 4096 / (time.perf_counter() - t0)          # groups/s on one core
+    n = int(min(t.n_groups, max(8192, rate * 15)))
+    t0 = time.perf_counter()
+    eo.decode_threads(om, t.blocks[:n], c)
+    dt = time.perf_counter() - t0
+    return {"value": n * G * 2 / dt / 1e9, "unit": UNIT, "cores": c, "kind": "oracle",
+            "sample": f"first {n} groups of the 4096x4096 q projection, one pass on {c} threads",
+            "groups_per_s": n / dt, "single_core_groups_per_s": rate}
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+
+    from paper_2505_06901_b200 import binding as B
+    from paper_2505_06901_b200 import synth, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+
+    # ---- workload (the same seeded tensors on every rank)
+    if args.small:
+        layer = workloads.config2(names=("q", "gate"))
+        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, workloads.calibrate_kv(3, 32))
+    else:
+        layer = workloads.config2()
+        (kt,) = workloads.config3(which=("K",))
+    kb, kh, kseq, _ = kt.shape
+    stream = torch.cuda.current_stream()
+    dl = []
+    for t in layer:
+        n_out, k = t.shape
+        wsb = B.ecco_gemv_workspace_bytes(n_out, k, 8)
+        dl.append(dict(t=t, n=t.n_groups, n_out=n_out, k=k, meta=B.meta_to_device(t.meta), blocks=torch.from_numpy(t.blocks).cuda(),
+                       out=torch.empty(t.n_groups * G, dtype=torch.float16, device="cuda"),
+                       x1=torch.from_numpy(synth.activations(1, k, 11)).cuda(), x8=torch.from_numpy(synth.activations(8, k, 12)).cuda(),
+                       y1=torch.empty((1, n_out), dtype=torch.float32, device="cuda"),
+                       y8=torch.empty((8, n_out), dtype=torch.float32, device="cuda"),
+                       ws=torch.empty(wsb, dtype=torch.uint8, device="cuda"), wsb=wsb))
+    k_meta, k_blocks = B.meta_to_device(kt.meta), torch.from_numpy(kt.blocks).cuda()
+    q = torch.from_numpy(synth.queries(kb, kh, 13)).cuda()
+    scores = torch.empty((kb, kh, kseq), dtype=torch.float32, device="cuda")
+    segs = [s for s in args.only.split(",") if s] or ["decompress", "gemv1", "gemv8", "attn"]
+
+    def step():
+        if "decompress" in segs:
+            for d in dl:
+                B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
+        if "gemv1" in segs:
+            for d in dl:
+                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1"], 1, d["y1"], d["ws"], d["wsb"], stream)
+        if "gemv8" in segs:
+            for d in dl:
+                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
+        if "attn" in segs:
+            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, 1, q, 128 ** -0.5, scores, stream)
+
+    def timed_step(ev):
+        ev[0].record(stream)
+        if "decompress" in segs:
+            for d in dl:
+                B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
+        ev[1].record(stream)
+        if "gemv1" in segs:
+            for d in dl:
+                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1"], 1, d["y1"], d["ws"], d["wsb"], stream)
+        ev[2].record(stream)
+        if "gemv8" in segs:
+            for d in dl:
+                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
+        ev[3].record(stream)
+        if "attn" in segs:
+            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, 1, q, 128 ** -0.5, scores, stream)
+        ev[4].record(stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = B.ecco_kernel_launch_count()
+    barrier()
+    for ev in events:
+        timed_step(ev)
+    barrier()
+    launches = B.ecco_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    assert B.ecco_device_status() == 0, "a kernel reported a device-side timeout"
+
+    total_ms = events[0][0].elapsed_time(events[-1][4])
+    seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(4)]
+    tvec = torch.tensor([total_ms] + seg_ms, dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(tvec, op=dist.ReduceOp.MAX)       # slowest rank decides
+    total_ms, dec_ms, g1_ms, g8_ms, at_ms = [float(v) for v in tvec.cpu()]
+
+    groups = sum(d["n"] for d in dl)
+    out_bytes = groups * G * 2
+    value = world * out_bytes * args.steps / (dec_ms / 1e3) / 1e9 if dec_ms > 0 else 0.0
+
+    # ---- end to end through the C ABI with host buffers: H2D of the blocks, decompress, D2H of the fp16
+    e2e = None
+    if "decompress" in segs:
+        h_in = [torch.from_numpy(d["t"].blocks).pin_memory() for d in dl]
+        h_out = [torch.empty(d["n"] * G, dtype=torch.float16).pin_memory() for d in dl]
+
+        def e2e_step():
+            for d, hi, ho in zip(dl, h_in, h_out):
+                d["blocks"].copy_(hi, non_blocking=True)
+                B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
+                ho.copy_(d["out"], non_blocking=True)
+
+        for _ in range(3):
+            e2e_step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        esteps = max(3, min(args.steps, 10))
+        barrier()
+        e0.record(stream)
+        for _ in range(esteps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        ems = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+        if dist is not None:
+            dist.all_reduce(ems, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * out_bytes * esteps / (float(ems.cpu()[0]) / 1e3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": groups * BLOCK, "d2h_bytes_per_step": out_bytes, "steps": esteps}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = measured_peaks()
+    n_launch = len(dl)
+    avg_launch_s = dec_ms / 1e3 / (args.steps * n_launch) if dec_ms > 0 else float("nan")
+    alg_bytes_per_launch = groups * (BLOCK + G * 2) / n_launch
+    achieved = alg_bytes_per_launch / avg_launch_s / 1e9 if dec_ms > 0 else 0.0
+    traffic = None
+    tp = os.path.join(ROOT, "profiles", "decompress_dram_bytes_per_group.json")
+    if os.path.exists(tp):
+        with open(tp) as f:
+            traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": ("reduced (profiling): q+gate, K cache batch 2" if args.small else
+                                "cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
+                                "+ cfg3 K cache [8][32][4096][128]"),
+                   "step": "decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1",
+                   "l2": "inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited",
+                   "format": "S=64, H=4, group 128, 64-byte blocks"},
+        "segments_us_per_step": {"decompress_layer": dec_ms / args.steps * 1e3, "gemv_layer_batch1": g1_ms / args.steps * 1e3,
+                                 "gemv_layer_batch8": g8_ms / args.steps * 1e3, "attn_scores_cfg3": at_ms / args.steps * 1e3},
+        "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3,
+        "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
+        "roofline": {"kernel": "ecco_decompress_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
+                     "algorithmic_bytes_per_launch": alg_bytes_per_launch, "avg_launch_us": avg_launch_s * 1e6},
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(layer, cores())
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

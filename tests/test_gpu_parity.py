@@ -1,0 +1,351 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle.
+
+Decompression must match the oracle bit for bit.  The fused calls accumulate in fp32 and are held
+to |y - y_ref| <= 1e-3 * sum_i |w_i x_i| per output (y_ref = the oracle's fp64 sum over the
+decompressed fp16 values); the plain relative error is also checked where |y_ref| is not small.
+"""
+import numpy as np
+import pytest
+
+from helpers import lib_meta_from_oracle, oracle_meta_from_lib
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-3
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.fail("the gpu tests need a CUDA device")
+    from paper_2505_06901_b200 import binding
+
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def W():
+    from paper_2505_06901_b200 import workloads
+
+    return workloads
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def gpu_decompress(B, lmeta, blocks):
+    n = blocks.shape[0]
+    d_meta = B.meta_to_device(lmeta)
+    d_blocks = dev(blocks)
+    d_out = torch.empty(max(n, 1) * 128, dtype=torch.float16, device="cuda")
+    before = B.ecco_kernel_launch_count()
+    B.ecco_decompress(d_meta, d_blocks, n, d_out)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    assert B.ecco_kernel_launch_count() == before + (1 if n else 0)
+    return d_out[: n * 128].cpu().numpy().reshape(n, 128)
+
+
+def assert_bit_exact(got, want):
+    g, w = got.view(np.uint16), want.view(np.uint16)
+    bad = np.nonzero((g != w).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} of {g.shape[0]} groups differ; first group {bad[:3]}, positions {np.nonzero(g[bad[0]] != w[bad[0]])[0][:8]}"
+
+
+def gpu_gemv(B, lmeta, blocks, n_out, k, x, batch):
+    d_meta, d_blocks, d_x = B.meta_to_device(lmeta), dev(blocks), dev(x)
+    d_y = torch.full((batch, n_out), float("nan"), dtype=torch.float32, device="cuda")
+    wsb = B.ecco_gemv_workspace_bytes(n_out, k, batch)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    ws.fill_(0xCD)                                   # stale contents must not matter
+    B.ecco_gemv(d_meta, d_blocks, n_out, k, d_x, batch, d_y, ws, wsb)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    return d_y.cpu().numpy().astype(np.float64), (d_meta, d_blocks, d_x, ws, wsb)
+
+
+def check_fused(got, ref, refabs):
+    err = np.abs(got - ref)
+    assert np.all(err <= TOL * refabs + 1e-30), float((err / (refabs + 1e-30)).max())
+    big = np.abs(ref) >= 0.1 * np.sqrt((ref ** 2).mean())
+    if big.any():
+        assert (err[big] / np.abs(ref[big])).max() <= TOL * 10
+
+
+# ------------------------------------------------------------------ decompress
+@pytest.mark.parametrize("n_groups", [0, 1, 31, 32, 33, 1000, 1023, 1025, 2048])
+def test_decompress_matches_oracle_ragged_sizes(B, eo, cfg1_small, n_groups):
+    lm = lib_meta_from_oracle(B, cfg1_small["meta"])
+    blocks = cfg1_small["blocks"][:n_groups]
+    got = gpu_decompress(B, lm, blocks)
+    if n_groups:
+        assert_bit_exact(got, eo.decode(cfg1_small["meta"], blocks))
+
+
+def test_decompress_config1_full_with_library_metadata(B, eo, W):
+    t = W.config1(keep_source=True)
+    assert t.n_groups == 8192
+    om = oracle_meta_from_lib(eo, t.meta)
+    want_blocks, _ = eo.encode(om, t.source, eo.SELECT_MSE)
+    assert np.array_equal(t.blocks, want_blocks)             # CPU encode: library == oracle
+    got = gpu_decompress(B, t.meta, t.blocks)
+    assert_bit_exact(got, eo.decode(om, t.blocks))
+    src = t.source.astype(np.float32).reshape(-1, 128)
+    rel = np.sqrt(((got.astype(np.float32) - src) ** 2).mean() / (src ** 2).mean())
+    assert rel < 0.15
+
+
+def test_decompress_kv_blocks_and_s16(B, eo, kv_small, synth):
+    lm = lib_meta_from_oracle(B, kv_small["meta"])
+    assert_bit_exact(gpu_decompress(B, lm, kv_small["blocks"]), eo.decode(kv_small["meta"], kv_small["blocks"]))
+    # the paper's hardware compressor uses 16 patterns for the KV cache
+    cal = synth.kv_cache(1, 4, 512, 2003, 3003)
+    m16 = eo.calibrate(cal, S=16, H=4, seed=3, select=eo.SELECT_MINMAX)
+    blocks, _ = eo.encode(m16, kv_small["k"], eo.SELECT_MINMAX)
+    assert_bit_exact(gpu_decompress(B, lib_meta_from_oracle(B, m16), blocks), eo.decode(m16, blocks))
+
+
+def test_decompress_is_total_on_garbage_and_edge_blocks(B, eo, cfg1_small, synth):
+    meta = cfg1_small["meta"]
+    lm = lib_meta_from_oracle(B, meta)
+    rb = synth.random_blocks(4096, 99)
+    assert_bit_exact(gpu_decompress(B, lm, rb), eo.decode(meta, rb))
+    edge = np.stack([np.full(64, v, dtype=np.uint8) for v in (0x00, 0xFF, 0xAA, 0x55, 0x7F, 0x80)] * 8)
+    assert_bit_exact(gpu_decompress(B, lm, edge), eo.decode(meta, edge))
+
+
+def make_meta(eo, lens_fn, S=4, e=-5, seed=0):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    m = eo.Meta()
+    m.S, m.H, m.e = S, 4, e
+    kl = eo.huffman_limited(np.ones(S), 12)
+    for k in range(S):
+        m.kp_len[k] = int(kl[k])
+        pat = np.sort(rng.uniform(-1, 1, 15))
+        for j in range(15):
+            m.pattern[k][j] = int(np.float16(pat[j]).view(np.uint16))
+        for h in range(4):
+            ln = lens_fn(k, h, rng)
+            for s in range(16):
+                m.cb_len[k][h][s] = int(ln[s])
+    assert eo.meta_check(m) == 0
+    return m
+
+
+def skew_lens(k, h, rng):
+    """The most skewed admissible code (Kraft: 3/4 + 3/16 + 2/64 + 8/256 = 1).  Codebook 0 gives the
+    2-bit codes to the middle centroids, where the values cluster (short streams, up to 16 pads); the
+    other codebooks are random permutations (long streams, heavy clipping)."""
+    lens = np.array([2, 2, 2, 4, 4, 4, 6, 6, 8, 8, 8, 8, 8, 8, 8, 8])
+    out = np.zeros(16, dtype=np.int64)
+    if h == 0:
+        out[[7, 6, 8, 5, 9, 4, 10, 3, 11, 2, 12, 1, 13, 0, 14, 15]] = lens
+    else:
+        out[rng.permutation(16)] = lens
+    return list(out)
+
+
+def test_decompress_adversarial_codebooks(B, eo):
+    """All-4-bit codes (10 + ID_KP + 128 x 4 > 512 bits: every group clips), the most skewed admissible
+    code (2-bit symbols next to 8-bit ones: heavy clipping and up to 16 pads), long ID_KP codes,
+    extreme exponents."""
+    rng = np.random.Generator(np.random.PCG64(11))
+    flat = make_meta(eo, lambda k, h, r: [4] * 16)
+    skew = make_meta(eo, skew_lens, seed=3)
+    for meta in (flat, skew):
+        x = (rng.standard_t(3, size=(512, 128)) * 0.05).astype(np.float16)
+        blocks, st = eo.encode(meta, x, eo.SELECT_MSE)
+        got = gpu_decompress(B, lib_meta_from_oracle(B, meta), blocks)
+        assert_bit_exact(got, eo.decode(meta, blocks))
+        assert st.clipped_groups == st.n_groups if meta is flat else (st.padded_groups > 0 and st.clipped_groups > 0)
+    # symbols forced to the longest codes -> every group clips; to the shortest -> 16 pads
+    m = skew
+    x = np.zeros((64, 128), dtype=np.float16)
+    x[:, 0] = 1.0
+    blocks, st = eo.encode(m, x, eo.SELECT_MSE)
+    assert_bit_exact(gpu_decompress(B, lib_meta_from_oracle(B, m), blocks), eo.decode(m, blocks))
+    for e in (-32, 16):
+        m2 = make_meta(eo, lambda k, h, r: [4] * 16, e=e, seed=5)
+        rb = np.random.Generator(np.random.PCG64(e + 100)).integers(0, 256, size=(256, 64), dtype=np.uint8)
+        assert_bit_exact(gpu_decompress(B, lib_meta_from_oracle(B, m2), rb), eo.decode(m2, rb))
+    # S = 64 with a deliberately unbalanced ID_KP code (lengths up to 12 bits)
+    m3 = make_meta(eo, lambda k, h, r: [4] * 16, S=64, seed=7)
+    kl = eo.huffman_limited(1.7 ** np.arange(64), 12)
+    assert kl.max() == 12
+    for k in range(64):
+        m3.kp_len[k] = int(kl[k])
+    assert eo.meta_check(m3) == 0
+    rb = np.random.Generator(np.random.PCG64(8)).integers(0, 256, size=(2048, 64), dtype=np.uint8)
+    assert_bit_exact(gpu_decompress(B, lib_meta_from_oracle(B, m3), rb), eo.decode(m3, rb))
+
+
+def test_decompress_rejects_bad_arguments_on_device(B, cfg1_small):
+    lm = lib_meta_from_oracle(B, cfg1_small["meta"])
+    d_meta, d_blocks = B.meta_to_device(lm), dev(cfg1_small["blocks"])
+    d_out = torch.empty(2048 * 128 + 8, dtype=torch.float16, device="cuda")
+    L = B.lib()
+    assert L.ecco_decompress(d_meta.data_ptr(), d_blocks.data_ptr(), 10, d_out.data_ptr() + 2, None) == B.ERR_ALIGNMENT
+    assert L.ecco_decompress(d_meta.data_ptr(), d_blocks.data_ptr() + 8, 10, d_out.data_ptr(), None) == B.ERR_ALIGNMENT
+    assert L.ecco_decompress(None, d_blocks.data_ptr(), 10, d_out.data_ptr(), None) == B.ERR_INVALID_ARG
+    # a side stream works like the current one
+    s = torch.cuda.Stream()
+    B.ecco_decompress(d_meta, d_blocks, 2048, d_out, stream=s)
+    s.synchronize()
+    assert B.ecco_device_status() == 0
+
+
+# ------------------------------------------------------------------ fused GEMV
+@pytest.mark.parametrize("n_out,k,batch", [(256, 1024, 1), (256, 1024, 3), (256, 1024, 8), (100, 1024, 2), (513, 512, 5),
+                                           (2048, 128, 1), (64, 4096, 4), (1, 128, 1)])
+def test_gemv_matches_oracle(B, eo, cfg1_small, synth, n_out, k, batch):
+    meta = cfg1_small["meta"]
+    n_groups = n_out * (k // 128)
+    reps = -(-n_groups // 2048)
+    blocks = np.tile(cfg1_small["blocks"], (reps, 1))[:n_groups]
+    x = synth.activations(batch, k, 50 + n_out + batch)
+    got, keep = gpu_gemv(B, lib_meta_from_oracle(B, meta), blocks, n_out, k, x, batch)
+    ref, refabs = eo.gemv(meta, blocks, n_out, k, x, batch)
+    check_fused(got, ref, refabs)
+    # a second call on the same (now dirty) workspace gives the same bits: fixed summation order
+    d_meta, d_blocks, d_x, ws, wsb = keep
+    d_y2 = torch.empty((batch, n_out), dtype=torch.float32, device="cuda")
+    B.ecco_gemv(d_meta, d_blocks, n_out, k, d_x, batch, d_y2, ws, wsb)
+    torch.cuda.synchronize()
+    assert np.array_equal(d_y2.cpu().numpy().astype(np.float64), got)
+
+
+def test_gemv_handles_pads_clips_and_garbage(B, eo, cfg1_small, synth):
+    meta = cfg1_small["meta"]
+    rb = synth.random_blocks(512 * 4, 123)                 # garbage streams: duplicate pad locations etc.
+    x = synth.activations(8, 512, 9)
+    got, _ = gpu_gemv(B, lib_meta_from_oracle(B, meta), rb, 512, 512, x, 8)
+    ref, refabs = eo.gemv(meta, rb, 512, 512, x, 8)
+    check_fused(got, ref, refabs)
+    skew = make_meta(eo, skew_lens, seed=3)   # many pads, many clips
+    w = (np.random.Generator(np.random.PCG64(1)).standard_t(3, size=(256, 256)) * 0.05).astype(np.float16)
+    blocks, st = eo.encode(skew, w, eo.SELECT_MSE)
+    assert st.padded_values > st.n_groups and st.clipped_groups > 0
+    x = synth.activations(2, 256, 10)
+    got, _ = gpu_gemv(B, lib_meta_from_oracle(B, skew), blocks, 256, 256, x, 2)
+    ref, refabs = eo.gemv(skew, blocks, 256, 256, x, 2)
+    check_fused(got, ref, refabs)
+
+
+def test_gemv_workspace_errors(B, cfg1_small, synth):
+    lm = lib_meta_from_oracle(B, cfg1_small["meta"])
+    d_meta, d_blocks = B.meta_to_device(lm), dev(cfg1_small["blocks"])
+    d_x, d_y = dev(synth.activations(1, 1024, 1)), torch.empty((1, 256), dtype=torch.float32, device="cuda")
+    with pytest.raises(B.EccoError) as ei:
+        B.ecco_gemv(d_meta, d_blocks, 256, 1024, d_x, 1, d_y, None, 0)
+    assert ei.value.code == B.ERR_WORKSPACE
+    small = torch.empty(64, dtype=torch.uint8, device="cuda")
+    with pytest.raises(B.EccoError) as ei:
+        B.ecco_gemv(d_meta, d_blocks, 256, 1024, d_x, 1, d_y, small, 64)
+    assert ei.value.code == B.ERR_WORKSPACE
+
+
+# ------------------------------------------------------------------ fused attention scores
+@pytest.mark.parametrize("batch,heads,seq,qpk", [(2, 4, 256, 1), (2, 4, 256, 2), (2, 4, 256, 8), (1, 3, 77, 4), (1, 1, 1, 1),
+                                                 (2, 2, 513, 3)])
+def test_attn_scores_match_oracle(B, eo, kv_small, synth, batch, heads, seq, qpk):
+    meta = kv_small["meta"]
+    n = batch * heads * seq
+    blocks = np.tile(kv_small["blocks"], (-(-n // 2048), 1))[:n]
+    q = synth.queries(batch, heads * qpk, 60 + seq)
+    scale = 128 ** -0.5
+    d_meta, d_blocks, d_q = B.meta_to_device(lib_meta_from_oracle(B, meta)), dev(blocks), dev(q)
+    d_s = torch.full((batch, heads * qpk, seq), float("nan"), dtype=torch.float32, device="cuda")
+    B.ecco_attn_scores(d_meta, d_blocks, batch, heads, seq, qpk, d_q, scale, d_s)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    ref, refabs = eo.attn_scores(meta, blocks, batch, heads, seq, qpk, q, scale)
+    check_fused(d_s.cpu().numpy().astype(np.float64), ref, refabs)
+
+
+# ------------------------------------------------------------------ full-size configurations
+def sample_groups(n, rng, k=6144):
+    idx = np.unique(np.concatenate([np.arange(min(n, 1024)), np.arange(max(0, n - 1024), n), rng.integers(0, n, k)]))
+    return idx
+
+
+def check_full_decompress(B, eo, t, d_out=None):
+    d_meta, d_blocks = B.meta_to_device(t.meta), dev(t.blocks)
+    d_out = torch.empty(t.n_groups * 128, dtype=torch.float16, device="cuda")
+    B.ecco_decompress(d_meta, d_blocks, t.n_groups, d_out)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    om = oracle_meta_from_lib(eo, t.meta)
+    idx = sample_groups(t.n_groups, np.random.Generator(np.random.PCG64(t.n_groups)))
+    got = d_out.view(-1, 128)[torch.from_numpy(idx).cuda()].cpu().numpy()
+    assert_bit_exact(got, eo.decode_threads(om, t.blocks[idx], 8))
+    assert bool(torch.isfinite(d_out).all())
+    return om, d_meta, d_blocks
+
+
+def check_full_gemv(B, eo, synth, t, om, d_meta, d_blocks, batch):
+    n_out, k = t.shape
+    x = synth.activations(batch, k, 70 + batch)
+    d_x = dev(x)
+    d_y = torch.empty((batch, n_out), dtype=torch.float32, device="cuda")
+    wsb = B.ecco_gemv_workspace_bytes(n_out, k, batch)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    B.ecco_gemv(d_meta, d_blocks, n_out, k, d_x, batch, d_y, ws, wsb)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    y = d_y.cpu().numpy().astype(np.float64)
+    rows = np.unique(np.concatenate([[0, n_out - 1], np.random.Generator(np.random.PCG64(n_out + batch)).integers(0, n_out, 48)]))
+    kb = k // 128
+    sub = np.concatenate([t.blocks[r * kb:(r + 1) * kb] for r in rows])
+    ref, refabs = eo.gemv(om, sub, len(rows), k, x, batch)
+    check_fused(y[:, rows], ref, refabs)
+
+
+def test_config2_llama7b_layer_full_size(B, eo, W, synth):
+    for t in W.config2(names=("q", "gate", "down")):
+        om, d_meta, d_blocks = check_full_decompress(B, eo, t)
+        for batch in (1, 8):
+            check_full_gemv(B, eo, synth, t, om, d_meta, d_blocks, batch)
+
+
+def check_full_attn(B, eo, synth, t, qpk):
+    batch, heads, seq, _ = t.shape
+    om = oracle_meta_from_lib(eo, t.meta)
+    q = synth.queries(batch, heads * qpk, 80 + qpk)
+    d_meta, d_blocks, d_q = B.meta_to_device(t.meta), dev(t.blocks), dev(q)
+    d_s = torch.empty((batch, heads * qpk, seq), dtype=torch.float32, device="cuda")
+    B.ecco_attn_scores(d_meta, d_blocks, batch, heads, seq, qpk, d_q, 128 ** -0.5, d_s)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    s = d_s.cpu().numpy().astype(np.float64)
+    rng = np.random.Generator(np.random.PCG64(seq + qpk))
+    for _ in range(6):
+        b, h = int(rng.integers(batch)), int(rng.integers(heads))
+        t0 = int(rng.integers(0, seq - 256 + 1))
+        g0 = (b * heads + h) * seq + t0
+        ref, refabs = eo.attn_scores(om, t.blocks[g0:g0 + 256], 1, 1, 256, qpk, q[b, h * qpk:(h + 1) * qpk], 128 ** -0.5)
+        check_fused(s[b, h * qpk:(h + 1) * qpk, t0:t0 + 256], ref[0], refabs[0])
+    assert np.isfinite(s).all()
+
+
+def test_config3_kv_cache_full_size(B, eo, W, synth):
+    (t,) = W.config3(which=("K",))
+    assert t.n_groups == 8 * 32 * 4096
+    check_full_decompress(B, eo, t)
+    check_full_attn(B, eo, synth, t, 1)
+
+
+def test_config4_llama70b_mlp_full_size(B, eo, W, synth):
+    for t in W.config4(names=("gate", "down")):
+        assert t.n_groups == 1835008
+        om, d_meta, d_blocks = check_full_decompress(B, eo, t)
+        check_full_gemv(B, eo, synth, t, om, d_meta, d_blocks, 1)
+
+
+def test_config5_long_context_gqa_full_size(B, eo, W, synth):
+    (t,) = W.config5(which=("K",))
+    assert t.n_groups == 16 * 8 * 32768
+    check_full_decompress(B, eo, t)
+    check_full_attn(B, eo, synth, t, 8)
