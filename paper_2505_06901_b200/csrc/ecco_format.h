@@ -42,5 +42,16 @@ constexpr uint32_t kDevBytes = kOffSymLut + kSymLutBytes;             // 75840
 constexpr uint32_t kTableBytes = kDevBytes - kOffPattern;             // 75776, a multiple of 16
 // Both lookup tables are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.
+//
+// Symbol tables are stored with a per-codebook index rotation: the entry for window value i of
+// codebook cb sits at index i ^ lut_rotation(cb).  The rotation touches index bits 2..6, which
+// select the shared-memory bank of a byte entry, so lanes that decode with different codebooks
+// spread over different banks even when their windows agree.
+#ifdef __CUDACC__
+#define ECCO_HD __host__ __device__
+#else
+#define ECCO_HD
+#endif
+ECCO_HD constexpr uint32_t lut_rotation(uint32_t cb) { return ((cb * 11u + (cb >> 3)) & 31u) << 2; }
 
 }  // namespace ecco

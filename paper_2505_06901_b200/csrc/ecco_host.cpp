@@ -786,11 +786,12 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
     uint8_t* sl = base + kOffSymLut;
     for (int k = 0; k < tmp.S; ++k)
         for (int c = 0; c < kCodebooks; ++c) {
-            uint8_t* t = sl + (static_cast<size_t>(k) * kCodebooks + c) * 256;
+            const uint32_t cb = static_cast<uint32_t>(k) * kCodebooks + c, rot = lut_rotation(cb);
+            uint8_t* t = sl + static_cast<size_t>(cb) * 256;
             for (int s = 0; s < kSymbols; ++s) {
                 int L = tmp.cb_len[k][c][s];
                 for (uint32_t hi = 0; hi < (1u << (kMaxLen - L)); ++hi)
-                    t[tmp.cb_rev[k][c][s] | (hi << L)] = static_cast<uint8_t>((L << 4) | s);
+                    t[(tmp.cb_rev[k][c][s] | (hi << L)) ^ rot] = static_cast<uint8_t>((L << 4) | s);
             }
         }
     // unused pattern rows (S < 64) decode with 4-bit codes so that every table entry is valid

@@ -90,11 +90,16 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
     return v;
 }
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
-__device__ __forceinline__ uint4 ldg_nc_v4(const void* p)
+// one 64-byte block = two 32-byte loads per lane: every load instruction asks for whole sectors
+struct Block { uint32_t w[16]; };
+__device__ __forceinline__ void ldg_block(Block& b, const uint8_t* p)
 {
-    uint4 v;
-    asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
-    return v;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(b.w[0]), "=r"(b.w[1]), "=r"(b.w[2]), "=r"(b.w[3]), "=r"(b.w[4]), "=r"(b.w[5]), "=r"(b.w[6]), "=r"(b.w[7])
+                 : "l"(p));
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(b.w[8]), "=r"(b.w[9]), "=r"(b.w[10]), "=r"(b.w[11]), "=r"(b.w[12]), "=r"(b.w[13]), "=r"(b.w[14]), "=r"(b.w[15])
+                 : "l"(p + 32));
 }
 __device__ __forceinline__ void stg_v8(void* p, const uint32_t (&r)[8])
 {
@@ -145,16 +150,15 @@ struct WarpSmem {
 
 struct GroupHeader {
     uint32_t pos;       // first bit of the coded indices
-    uint32_t lut;       // shared address of the symbol table of (ID_KP, ID_HF)
+    uint32_t lut;       // shared address of the symbol table of (ID_KP, ID_HF), OR-ed with its index rotation
 };
 
 // Pattern retriever (Sec. 4.2): scale byte, ID_HF, Huffman-coded ID_KP; writes the lane's 16
 // dequantised values (fp16 bits, or fp32 bits when kFloatTab) and the transposed bit stream.
 template <bool kFloatTab>
-__device__ __forceinline__ GroupHeader open_group(const uint4 (&blk)[4], uint32_t smem_base, const WarpSmem& ws, float T)
+__device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T)
 {
-    const uint32_t w[16] = {blk[0].x, blk[0].y, blk[0].z, blk[0].w, blk[1].x, blk[1].y, blk[1].z, blk[1].w,
-                            blk[2].x, blk[2].y, blk[2].z, blk[2].w, blk[3].x, blk[3].y, blk[3].z, blk[3].w};
+    const uint32_t (&w)[16] = blk.w;
 #pragma unroll
     for (int i = 0; i < 16; ++i) sts_u32(ws.bits + i * 128, w[i]);
     const uint32_t qs = w[0] & 0xffu, hf = (w[0] >> 8) & 3u;
@@ -164,7 +168,8 @@ __device__ __forceinline__ GroupHeader open_group(const uint4 (&blk)[4], uint32_
     const uint32_t kp = kpe & 0xffu;
     GroupHeader h;
     h.pos = kHeaderBits + (kpe >> 8);
-    h.lut = smem_base + kSmemSymLut + (kp * kCodebooks + hf) * 256;
+    const uint32_t cb = kp * kCodebooks + hf;
+    h.lut = (smem_base + kSmemSymLut + cb * 256) | lut_rotation(cb);   // table rows are 256-byte aligned
     const float top = fp8_to_float(qs) * T;           // FP8 -> FP16 range by the power-of-two factor
     const float s = fabsf(top);
     uint4 p0, p1;
@@ -184,6 +189,8 @@ __device__ __forceinline__ GroupHeader open_group(const uint4 (&blk)[4], uint32_
 // Decodes the 128 indices of the lane's group (Sec. 4.2, Huffman decode) and hands each value to
 // sink(n, value_bits, symbol).  A codeword that would cross bit 512 ends the group: that and all
 // later positions are delivered as zero (clipped).  Returns the end bit if all 128 fitted, else 0.
+// Must be called by all 32 lanes of the warp.  Four symbols are decoded per window refill; the
+// per-symbol clip test runs only in steps where some lane of the warp reaches bit 512.
 template <class Sink>
 __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const WarpSmem& ws, Sink&& sink)
 {
@@ -194,15 +201,24 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         const uint32_t wi = min(pos >> 5, 16u);
         const uint32_t lo = lds_u32(ws.bits + wi * 128), hi = lds_u32(ws.bits + wi * 128 + 128);
         const uint32_t win = __funnelshift_r(lo, hi, pos);           // 32 stream bits from pos
-        const uint32_t limit = kBlockBits - min(pos, static_cast<uint32_t>(kBlockBits));
-        uint32_t acc = 0;
+        uint32_t e[4], end[4], acc = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            const uint32_t e = lds_u8(h.lut + ((win >> acc) & 0xffu));
-            acc += e >> 4;
-            alive = alive && (acc <= limit);
-            const uint32_t v = lds_u32(ws.tab + (e & 15u) * 128);
-            sink(step * 4 + j, alive ? v : 0u, e & 15u);
+            e[j] = lds_u8(h.lut ^ ((win >> acc) & 0xffu));           // rotated index, see lut_rotation()
+            acc += e[j] >> 4;
+            end[j] = acc;
+        }
+        if (__any_sync(0xffffffffu, pos + acc > static_cast<uint32_t>(kBlockBits))) {
+            const uint32_t limit = kBlockBits - min(pos, static_cast<uint32_t>(kBlockBits));
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                alive = alive && (end[j] <= limit);
+                const uint32_t v = lds_u32(ws.tab + (e[j] & 15u) * 128);
+                sink(step * 4 + j, alive ? v : 0u, e[j] & 15u);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) sink(step * 4 + j, lds_u32(ws.tab + (e[j] & 15u) * 128), e[j] & 15u);
         }
         pos += acc;
     }
@@ -222,6 +238,8 @@ __device__ __forceinline__ uint32_t read_pad(const WarpSmem& ws, int j)
 // ---------------------------------------------------------------------------------------------
 // K1: ecco_decompress
 // ---------------------------------------------------------------------------------------------
+// Work is dealt out in warp tiles of 32 consecutive groups, tile i to warp (i mod total warps):
+// every SM then gets the same number of tiles to within one, whatever the tensor size.
 template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
@@ -238,31 +256,30 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
     sts_u32(ws.bits + 16 * 128, 0u);
     sts_u32(ws.bits + 17 * 128, 0u);
 
-    const uint64_t tile = static_cast<uint64_t>(kWarps) * 32u;
-    uint64_t g = blockIdx.x * tile + threadIdx.x;
-    uint4 blk[4];
-    if (g < n_groups) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(d_blocks + g * kBlockBytes + i * 16);
-    }
+    const uint64_t n_tiles = (n_groups + 31) / 32;
+    const uint64_t tile_stride = static_cast<uint64_t>(gridDim.x) * kWarps;
+    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;   // warps of one CTA take tiles far apart
+    Block blk;
+    // lanes past the end of the tensor decode the last group again and store nothing
+    if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
     if (!stage_tables(smem, d_meta, &bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
-    for (; g < n_groups; g += gridDim.x * tile) {
+    for (; tile < n_tiles; tile += tile_stride) {
+        const uint64_t g = tile * 32 + lane;
+        const bool store = g < n_groups;
         const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
-        const uint64_t gn = g + gridDim.x * tile;
-        if (gn < n_groups) {                               // next block in flight while this one decodes
-#pragma unroll
-            for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(d_blocks + gn * kBlockBytes + i * 16);
-        }
-        uint16_t* out = d_out + g * kGroup;
+        const uint64_t tn = tile + tile_stride;
+        if (tn < n_tiles)                                  // next block in flight while this one decodes
+            ldg_block(blk, d_blocks + min(tn * 32 + lane, n_groups - 1) * kBlockBytes);
+        uint16_t* out = d_out + min(g, n_groups - 1) * kGroup;
         uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t) {
             const int slot = (n & 15) >> 1;
             if (n & 1) r[slot] |= v << 16; else r[slot] = v;
-            if ((n & 15) == 15) stg_v8(out + (n - 15), r);
+            if ((n & 15) == 15 && store) stg_v8(out + (n - 15), r);
         });
-        if (end) {
+        if (end && store) {
             const int n_pad = min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits));
             for (int j = 0; j < n_pad; ++j) {
                 const uint32_t f = read_pad(ws, j);
@@ -313,7 +330,7 @@ struct Accum {
 
 // decode one group and accumulate its kV dot products against xs (shared address of xs[0][0])
 template <int kV>
-__device__ __forceinline__ void fused_group(const uint4 (&blk)[4], uint32_t smem_base, const WarpSmem& ws, float T,
+__device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T,
                                             uint32_t xs, Accum<kV>& acc)
 {
     const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
@@ -376,12 +393,10 @@ ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__
     const int kb_hi = static_cast<int>(static_cast<int64_t>(kblocks) * (split + 1) / ksplit);
     const int k = kblocks * kGroup;
 
-    uint4 blk[4];
-    const uint8_t* row_blocks = d_blocks + static_cast<uint64_t>(row_ok ? row : 0) * kblocks * kBlockBytes;
-    if (row_ok && kb_lo < kb_hi) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(row_blocks + static_cast<uint64_t>(kb_lo) * kBlockBytes + i * 16);
-    }
+    // rows past the end of the matrix decode the last row again and store nothing
+    Block blk;
+    const uint8_t* row_blocks = d_blocks + static_cast<uint64_t>(row_ok ? row : n_out - 1) * kblocks * kBlockBytes;
+    if (kb_lo < kb_hi) ldg_block(blk, row_blocks + static_cast<uint64_t>(kb_lo) * kBlockBytes);
     if (!stage_tables(smem, d_meta, &bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
@@ -395,12 +410,9 @@ ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__
             xs[i] = (b < batch) ? __half2float(d_x[static_cast<size_t>(b) * k + kb * kGroup + e]) : 0.0f;
         }
         __syncthreads();                                   // slice visible; the other slice is free again
-        if (row_ok) {
-            uint4 cur[4] = {blk[0], blk[1], blk[2], blk[3]};
-            if (kb + 1 < kb_hi) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(row_blocks + static_cast<uint64_t>(kb + 1) * kBlockBytes + i * 16);
-            }
+        {
+            const Block cur = blk;
+            if (kb + 1 < kb_hi) ldg_block(blk, row_blocks + static_cast<uint64_t>(kb + 1) * kBlockBytes);
             fused_group<kV>(cur, smem_base, ws, T, xs_base + ((kb - kb_lo) & 1) * kXsBytes, acc);
         }
     }
@@ -456,11 +468,11 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const int tile = kWarps * 32;
     int t = chunk * tile + static_cast<int>(threadIdx.x);
     const uint8_t* head_blocks = d_kblocks + static_cast<uint64_t>(bh) * seq * kBlockBytes;
-    uint4 blk[4];
-    if (t < seq) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(head_blocks + static_cast<uint64_t>(t) * kBlockBytes + i * 16);
-    }
+    // the loop below runs whole warps: lanes past the end of the sequence decode the last token
+    // again and store nothing
+    Block blk;
+    const int t_warp = t - static_cast<int>(lane);
+    if (t_warp < seq) ldg_block(blk, head_blocks + static_cast<uint64_t>(min(t, seq - 1)) * kBlockBytes);
     // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
     for (int i = threadIdx.x; i < kGroup * kV; i += tile) {
         const int r = i % kV, d = i / kV;
@@ -469,19 +481,18 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     if (!stage_tables(smem, d_meta, &bar)) return;        // also orders the xs writes (barrier inside)
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
-    for (; t < seq; t += chunks_per_head * tile) {
-        uint4 cur[4] = {blk[0], blk[1], blk[2], blk[3]};
+    for (; t - static_cast<int>(lane) < seq; t += chunks_per_head * tile) {
+        const Block cur = blk;
         const int tn = t + chunks_per_head * tile;
-        if (tn < seq) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) blk[i] = ldg_nc_v4(head_blocks + static_cast<uint64_t>(tn) * kBlockBytes + i * 16);
-        }
+        if (tn - static_cast<int>(lane) < seq) ldg_block(blk, head_blocks + static_cast<uint64_t>(min(tn, seq - 1)) * kBlockBytes);
         Accum<kV> acc;
         acc.clear();
         fused_group<kV>(cur, smem_base, ws, T, xs_addr, acc);
+        if (t < seq) {
 #pragma unroll
-        for (int r = 0; r < kV; ++r)
-            if (r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = acc.a[r];
+            for (int r = 0; r < kV; ++r)
+                if (r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = acc.a[r];
+        }
     }
 }
 
@@ -586,9 +597,8 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
         if (rc) return rc;
         configured[di.device] = true;
     }
-    const uint64_t tile = kDecompressWarps * 32;
-    const uint64_t tiles = (n_groups + tile - 1) / tile;
-    const unsigned grid = static_cast<unsigned>(tiles < static_cast<uint64_t>(di.sms) ? tiles : di.sms);
+    const uint64_t cta_tiles = (n_groups + kDecompressWarps * 32 - 1) / (kDecompressWarps * 32);   // one tile per warp
+    const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
     kernel<<<grid, kDecompressWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out));
     return check_launch();

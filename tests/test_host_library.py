@@ -176,10 +176,12 @@ def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
         e = int(kpl[(bits >> 10) & 0xFFF])
         assert e & 0xFF == info.kp
         pos = 10 + (e >> 8)
-        lut = syml[info.kp * 4 + info.hf]
+        cb = info.kp * 4 + info.hf
+        lut = syml[cb]
+        rot = ((cb * 11 + (cb >> 3)) & 31) << 2          # per-codebook index rotation of the image
         n = 0
         while n < 128:
-            t = int(lut[(bits >> pos) & 0xFF])
+            t = int(lut[((bits >> pos) & 0xFF) ^ rot])
             if pos + (t >> 4) > 512:
                 break
             assert (t & 15) == sym[n]
