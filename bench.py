@@ -192,11 +192,9 @@ def run_ours(args):
     import torch
 
     from paper_2505_06901_b200 import binding as B
-    from paper_2505_06901_b200 import synth, workloads
+    from paper_2505_06901_b200 import distutil, synth, workloads
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = distutil.rank_info()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
@@ -284,10 +282,7 @@ def run_ours(args):
 
     total_ms = events[0][0].elapsed_time(events[-1][4])
     seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(4)]
-    tvec = torch.tensor([total_ms] + seg_ms, dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(tvec, op=dist.ReduceOp.MAX)       # slowest rank decides
-    total_ms, dec_ms, g1_ms, g8_ms, at_ms = [float(v) for v in tvec.cpu()]
+    total_ms, dec_ms, g1_ms, g8_ms, at_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
 
     groups = sum(d["n"] for d in dl)
     out_bytes = groups * G * 2
@@ -315,10 +310,8 @@ def run_ours(args):
             e2e_step()
         e1.record(stream)
         barrier()
-        ems = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-        if dist is not None:
-            dist.all_reduce(ems, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * out_bytes * esteps / (float(ems.cpu()[0]) / 1e3) / 1e9, "unit": UNIT,
+        (ems,) = distutil.max_over_ranks([e0.elapsed_time(e1)], dist, "cuda")
+        e2e = {"value": world * out_bytes * esteps / (ems / 1e3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": groups * BLOCK, "d2h_bytes_per_step": out_bytes, "steps": esteps}
 
     if rank != 0:

@@ -1,0 +1,49 @@
+"""The N > 1 bookkeeping of bench.py on two gloo ranks (CPU): slowest rank decides, bytes add up."""
+import os
+import socket
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world), LOCAL_RANK=str(rank))
+    from paper_2505_06901_b200 import distutil
+
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        assert distutil.rank_info() == (rank, world, rank)
+        times = [1.0 + rank, 5.0 - rank, 2.0]
+        mx = distutil.max_over_ranks(times, dist)
+        rate = distutil.aggregate_throughput(1e9, 0.5 * (rank + 1), world, dist)
+        out.put((rank, mx, rate))
+        dist.barrier()
+    finally:
+        dist.destroy_process_group()
+
+
+def test_max_over_ranks_and_weak_scaling_rate_with_two_gloo_ranks():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker, args=(r, 2, port, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    for rank, mx, rate in results:
+        assert mx == [2.0, 5.0, 2.0]
+        assert rate == pytest.approx(2 * 1e9 / 1.0)      # 2 ranks x 1 GB over the slower rank's 1.0 s
+
+
+def test_single_process_is_identity():
+    from paper_2505_06901_b200 import distutil
+
+    assert distutil.max_over_ranks([3.0, 1.0]) == [3.0, 1.0]
+    assert distutil.aggregate_throughput(10.0, 2.0, 1) == 5.0
