@@ -131,6 +131,26 @@ size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch);
 int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x_fp16,
               int32_t batch, float* d_y, void* d_workspace, size_t workspace_bytes, void* stream);
 
+/* Allocation-free variant of ecco_gemv.  The paper has no counterpart: this entry point exists for
+ * callers that are not allowed to obtain device memory at the time they need the product -- a
+ * layer plugged into an inference engine whose memory plan was fixed when the engine was built, a
+ * serving loop that must not call cudaMalloc because it synchronises the whole device and stalls
+ * every other stream, or a process whose memory budget was handed out in full at start-up.  Same
+ * arguments and result as ecco_gemv, but the scratch for the split-k partial sums is a fixed array
+ * of ECCO_STATIC_WORKSPACE_BYTES inside the library's device image (every GPU that loads the
+ * library carries it until the process exits) instead of a caller buffer.  The call allocates
+ * nothing.  A shape whose plan needs more scratch than that is refused with ECCO_ERR_WORKSPACE
+ * before anything is launched (for scale: batch 8 on an 11008 x 4096 matrix needs about 2.5 MB).
+ * The first call on each device looks up the array's device address (with that device current);
+ * make that first call outside any stream capture.  All calls on a device share the one array:
+ * it still holds the previous call's values when the next call starts (each call clears the part
+ * that must start from zero), and two calls whose kernels overlap on the GPU -- different streams,
+ * no dependency between them -- race on it and give undefined results.  Serialise them, or use
+ * ecco_gemv with separate workspaces. */
+#define ECCO_STATIC_WORKSPACE_BYTES (4u << 20)
+int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x_fp16,
+                        int32_t batch, float* d_y, void* stream);
+
 /* Fused attention scores over a compressed K cache (Eq. 3: Q K^T / sqrt(d_k), without the
  * softmax): scores[b][hq][t] = scale * sum_d q[b][hq][d] * K~[b][hq / q_per_kv][t][d].  One group
  * is the 128-wide head vector of one token; blocks are ordered [batch][n_kv_heads][seq]; q is

@@ -33,7 +33,7 @@ ERR_DEVICE_TIMEOUT = -8
 EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
-    "ecco_gemv", "ecco_attn_scores", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
+    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
 
@@ -87,6 +87,7 @@ def lib():
         L.ecco_gemv_workspace_bytes.argtypes = [i32, i32, i32]
         L.ecco_gemv_workspace_bytes.restype = sz
         L.ecco_gemv.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, vp]
+        L.ecco_gemv_static_ws.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
         L.ecco_attn_scores.argtypes = [vp, vp, i32, i32, i32, i32, vp, C.c_float, vp, vp]
         L.ecco_error_string.argtypes = [C.c_int]
         L.ecco_error_string.restype = C.c_char_p
@@ -232,6 +233,19 @@ def ecco_gemv(d_meta, d_blocks, n_out: int, k: int, d_x_fp16, batch: int, d_y, d
     _check(lib().ecco_gemv(_ptr(d_meta), _ptr(d_blocks), n_out, k, _ptr(d_x_fp16), batch, _ptr(d_y),
                            _ptr(d_workspace) if d_workspace is not None else None, workspace_bytes, _stream(stream)),
            "ecco_gemv")
+
+
+STATIC_WORKSPACE_BYTES = 4 << 20
+
+
+def ecco_gemv_static_ws(d_meta, d_blocks, n_out: int, k: int, d_x_fp16, batch: int, d_y, stream=None) -> None:
+    """ecco_gemv without a caller workspace and without any allocation: the scratch is a fixed
+    STATIC_WORKSPACE_BYTES array inside the library, shared by all calls on the device (so calls that
+    overlap on the GPU race).  For callers that may not allocate device memory when they run, such
+    as engine plug-ins with a fixed memory plan.  Make the first call on a device outside stream
+    capture.  Raises EccoError(ERR_WORKSPACE) for shapes that need more scratch than the array."""
+    _check(lib().ecco_gemv_static_ws(_ptr(d_meta), _ptr(d_blocks), n_out, k, _ptr(d_x_fp16), batch, _ptr(d_y),
+                                     _stream(stream)), "ecco_gemv_static_ws")
 
 
 def ecco_attn_scores(d_meta, d_kblocks, batch: int, n_kv_heads: int, seq: int, q_per_kv: int, d_q_fp16, scale: float,

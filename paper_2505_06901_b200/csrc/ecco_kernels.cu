@@ -21,6 +21,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstdio>
+#include <mutex>
 
 #include "../../include/ecco.h"
 #include "ecco_format.h"
@@ -663,6 +664,50 @@ extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_
         case 2: return launch_gemv<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
         case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
         default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// ecco_gemv_static_ws: ecco_gemv for callers that cannot allocate.  The split-k scratch is this
+// fixed array in the library's device image.  In host code the name below is only a handle for
+// the runtime, not a device address: the address comes from cudaGetSymbolAddress, once per
+// device, and that pointer is what the kernel receives.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_workspace[ECCO_STATIC_WORKSPACE_BYTES];
+
+extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x,
+                                   int32_t batch, float* d_y, void* stream)
+{
+    if (!d_meta || !d_blocks || !d_x || !d_y) return ECCO_ERR_INVALID_ARG;
+    if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_x) || !aligned16(d_y)) return ECCO_ERR_ALIGNMENT;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    const int kblocks = k / kGroup, vpad = pad_v(batch);
+    // refuse, before any launch, a shape whose plan does not fit the fixed array
+    const GemvPlan p = gemv_plan(n_out, kblocks, vpad, di.sms);
+    if (p.ksplit > 1 && p.partial_bytes + p.ticket_bytes > ECCO_STATIC_WORKSPACE_BYTES) return ECCO_ERR_WORKSPACE;
+    // one-time set-up per device (the current device is di.device): resolve the array's address
+    static std::mutex mu;
+    static void* address[64] = {};
+    void* ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mu);
+        if (!address[di.device]) {
+            void* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_workspace);
+            if (e != cudaSuccess || !ptr) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+            address[di.device] = ptr;
+        }
+        ws = address[di.device];
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (vpad) {
+        case 1: return launch_gemv<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        case 2: return launch_gemv<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
     }
 }
 
