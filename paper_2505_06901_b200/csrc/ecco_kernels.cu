@@ -15,6 +15,7 @@
 //            tab[16][32]  u32   per-lane dequantised centroids (entry 15 = the abs-max)
 //            syms[16][32] u32   (fused kernels) decoded indices, 8 nibbles per word, for the
 //                               outlier fix-up
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
@@ -108,6 +109,22 @@ __device__ __forceinline__ void stg_v8(void* p, const uint32_t (&r)[8])
                  "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
                  : "memory");
 }
+
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// 2-D tiled bulk store shared -> global through a tensor map (TMA); rows outside the tensor are dropped
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x),
+                 "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // OCP E4M3 byte -> fp32, arithmetically (the all-ones exponent/mantissa code reads as 480)
 __device__ __forceinline__ float fp8_to_float(uint32_t b)
@@ -289,6 +306,89 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
             }
         }
     }
+}
+
+// K1, bulk-store variant.  Per-lane 32-byte stores land in 32 different 128-byte lines and cost the
+// load/store pipe one pass per sector.  Here every 16 decoded values per lane go to a 1 KB
+// staging tile in shared memory ([32 groups][32 bytes], 16-byte halves swizzled the way the
+// tensor map's 32-byte swizzle expects, so the 128-bit shared stores are conflict-free) and one
+// lane hands the tile to the TMA engine, which writes the 32 rows of the [n_groups][128] fp16
+// tensor and drops rows past its end.  Outliers: those in the last tile (positions >= 112) are
+// patched in shared memory before that tile leaves; the others are 2-byte global stores issued
+// after the group's earlier tiles have been written (bulk wait + warp barrier), so they land last.
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
+                           uint16_t* __restrict__ d_out, const __grid_constant__ CUtensorMap out_map)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t smem_base = smem_u32(smem);
+    constexpr uint32_t kStageBase = (kSmemWarpBase + kWarps * (kBitsBytes + kTabBytes) + 1023u) & ~1023u;
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * (kBitsBytes + kTabBytes) + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = 0;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kStageBase + warp * 1024;                 // this warp's staging tile
+    const uint32_t swz = ((lane >> 2) & 1u) << 4;                               // 32-byte swizzle: bit 4 ^= bit 7
+    const uint32_t my_row = stage + lane * 32;
+
+    const uint64_t n_tiles = (n_groups + 31) / 32;
+    const uint64_t tile_stride = static_cast<uint64_t>(gridDim.x) * kWarps;
+    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
+    Block blk;
+    if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    for (; tile < n_tiles; tile += tile_stride) {
+        const uint64_t g = tile * 32 + lane;
+        const bool store = g < n_groups;
+        const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
+        const uint64_t tn = tile + tile_stride;
+        if (tn < n_tiles) ldg_block(blk, d_blocks + min(tn * 32 + lane, n_groups - 1) * kBlockBytes);
+        const int row0 = static_cast<int>(tile * 32);
+        uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        auto stage_rows = [&]() {
+            if (lane == 0) bulk_wait_read0();              // the engine has read the previous tile
+            __syncwarp();
+            sts_v4(my_row + swz, r[0], r[1], r[2], r[3]);
+            sts_v4(my_row + (swz ^ 16u), r[4], r[5], r[6], r[7]);
+        };
+        auto send_tile = [&](int chunk) {
+            fence_async_smem();                            // generic-proxy writes -> visible to the engine
+            __syncwarp();
+            if (lane == 0) { tma_store_2d(&out_map, stage, chunk * 16, row0); bulk_commit(); }
+        };
+        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t) {
+            const int slot = (n & 15) >> 1;
+            if (n & 1) r[slot] |= v << 16; else r[slot] = v;
+            if ((n & 15) == 15 && n != 127) { stage_rows(); send_tile(n >> 4); }
+        });
+        stage_rows();                                      // values 112..127
+        const int n_pad = end ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
+        if (__any_sync(0xffffffffu, n_pad > 0)) {
+            if (lane == 0) bulk_wait_all();                // tiles 0..6 of this group are in memory
+            __syncwarp();
+            uint16_t* out = d_out + min(g, n_groups - 1) * kGroup;
+            for (int j = 0; j < n_pad; ++j) {              // ascending: a later pad overrides an earlier one
+                const uint32_t f = read_pad(ws, j);
+                const uint32_t loc = f & 127u;
+                const uint16_t val = static_cast<uint16_t>(f2h_bits(fp8_to_float(f >> 7) * T));
+                if (loc >= 112u) {
+                    const uint32_t byte = (loc - 112u) * 2;
+                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)), "h"(val) : "memory");
+                } else if (store) {
+                    out[loc] = val;
+                }
+            }
+        }
+        send_tile(7);
+    }
+    if (lane == 0) bulk_wait_all();                        // shared memory must outlive the engine's reads
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -581,6 +681,39 @@ extern "C" int ecco_device_status(void)
     return st;
 }
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point query (no link against libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn encode_tiled_fn()
+{
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// tensor map of the output seen as [n_groups][128] fp16, box = 32 rows x 16 values, 32-byte swizzle
+static bool make_out_map(CUtensorMap* map, void* d_out, uint64_t n_groups)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {kGroup, n_groups};
+    const cuuint64_t strides[1] = {kGroup * 2};
+    const cuuint32_t box[2] = {16, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, d_out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kDecompressTmaWarps = 28;
+
 extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out, void* stream)
 {
     if (n_groups == 0) return ECCO_OK;
@@ -590,9 +723,28 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;
+    static thread_local bool configured[64] = {};
+    static thread_local bool configured_tma[64] = {};
+    // bulk-store variant for everything but tiny tensors (its box is 32 rows tall)
+    CUtensorMap map;
+    if (n_groups >= 32 && make_out_map(&map, d_out, n_groups)) {
+        auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps>;
+        constexpr size_t smem =
+            ((kSmemWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
+            static_cast<size_t>(kDecompressTmaWarps) * 1024;
+        if (!configured_tma[di.device]) {
+            rc = set_smem(kernel, smem);
+            if (rc) return rc;
+            configured_tma[di.device] = true;
+        }
+        const uint64_t cta_tiles = (n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
+        const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
+        kernel<<<grid, kDecompressTmaWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+            static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), map);
+        return check_launch();
+    }
     auto kernel = ecco_decompress_kernel<kDecompressWarps>;
     const size_t smem = kSmemWarpBase + static_cast<size_t>(kDecompressWarps) * (kBitsBytes + kTabBytes);
-    static thread_local bool configured[64] = {};
     if (!configured[di.device]) {
         rc = set_smem(kernel, smem);
         if (rc) return rc;
