@@ -42,6 +42,9 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5"],
+                    help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg5: long-context GQA K cache "
+                         "[16][8][32768][128] (decompress + attention scores with 8 query heads per KV head)")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -181,7 +184,7 @@ def cpu_baseline(layer, c: int):
     eo.decode_threads(om, t.blocks[:n], c)
     dt = time.perf_counter() - t0
     return {"value": n * G * 2 / dt / 1e9, "unit": UNIT, "cores": c, "kind": "oracle",
-            "sample": f"first {n} groups of the 4096x4096 q projection, one pass on {c} threads",
+            "sample": f"first {n} groups of tensor '{t.name}' {tuple(t.shape)}, one pass on {c} threads",
             "groups_per_s": n / dt, "single_core_groups_per_s": rate}
 
 
@@ -206,7 +209,11 @@ def run_ours(args):
     B.lib()
 
     # ---- workload (the same seeded tensors on every rank)
-    if args.small:
+    q_per_kv = 1
+    if args.workload == "cfg5":
+        (kt,) = workloads.config5(which=("K",))
+        layer, q_per_kv = [], 8
+    elif args.small:
         layer = workloads.config2(names=("q", "gate"))
         kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, workloads.calibrate_kv(3, 32))
     else:
@@ -225,9 +232,13 @@ def run_ours(args):
                        y8=torch.empty((8, n_out), dtype=torch.float32, device="cuda"),
                        ws=torch.empty(wsb, dtype=torch.uint8, device="cuda"), wsb=wsb))
     k_meta, k_blocks = B.meta_to_device(kt.meta), torch.from_numpy(kt.blocks).cuda()
-    q = torch.from_numpy(synth.queries(kb, kh, 13)).cuda()
-    scores = torch.empty((kb, kh, kseq), dtype=torch.float32, device="cuda")
-    segs = [s for s in args.only.split(",") if s] or ["decompress", "gemv1", "gemv8", "attn"]
+    q = torch.from_numpy(synth.queries(kb, kh * q_per_kv, 13)).cuda()
+    scores = torch.empty((kb, kh * q_per_kv, kseq), dtype=torch.float32, device="cuda")
+    if args.workload == "cfg5":          # the cache itself is the tensor to decompress; no weight matrices, no GEMV
+        dl.append(dict(t=kt, n=kt.n_groups, meta=k_meta, blocks=k_blocks,
+                       out=torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")))
+    segs = [s for s in args.only.split(",") if s] or (["decompress", "attn"] if args.workload == "cfg5" else
+                                                         ["decompress", "gemv1", "gemv8", "attn"])
 
     def step():
         if "decompress" in segs:
@@ -240,7 +251,7 @@ def run_ours(args):
             for d in dl:
                 B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
         if "attn" in segs:
-            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, 1, q, 128 ** -0.5, scores, stream)
+            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, q_per_kv, q, 128 ** -0.5, scores, stream)
 
     def timed_step(ev):
         ev[0].record(stream)
@@ -257,7 +268,7 @@ def run_ours(args):
                 B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
         ev[3].record(stream)
         if "attn" in segs:
-            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, 1, q, 128 ** -0.5, scores, stream)
+            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, q_per_kv, q, 128 ** -0.5, scores, stream)
         ev[4].record(stream)
 
     def barrier():
@@ -333,11 +344,14 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": ("reduced (profiling): q+gate, K cache batch 2" if args.small else
+        "config": {"workload": ("cfg5 long-context GQA K cache [16][8][32768][128] (4,194,304 groups)" if args.workload == "cfg5" else
+                                "reduced (profiling): q+gate, K cache batch 2" if args.small else
                                 "cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
                                 "+ cfg3 K cache [8][32][4096][128]"),
-                   "step": "decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1",
-                   "l2": "inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited",
+                   "step": ("decompress x1, attn_scores x1 (8 query heads per KV head)" if args.workload == "cfg5" else
+                            "decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1"),
+                   "l2": ("inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB" if args.workload == "cfg5" else
+                          "inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
                    "format": "S=64, H=4, group 128, 64-byte blocks"},
         "segments_us_per_step": {"decompress_layer": dec_ms / args.steps * 1e3, "gemv_layer_batch1": g1_ms / args.steps * 1e3,
                                  "gemv_layer_batch8": g8_ms / args.steps * 1e3, "attn_scores_cfg3": at_ms / args.steps * 1e3},
@@ -348,7 +362,7 @@ def run_ours(args):
                      "algorithmic_bytes_per_launch": alg_bytes_per_launch, "avg_launch_us": avg_launch_s * 1e6},
     }
     if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline(layer, cores())
+        line["cpu_baseline"] = cpu_baseline([d["t"] for d in dl], cores())
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

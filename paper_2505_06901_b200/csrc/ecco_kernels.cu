@@ -394,37 +394,54 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
 // ---------------------------------------------------------------------------------------------
 // K2/K3: fused consumers.  kV = number of dot products per group (batch rows of x, or query
 // heads per KV head).  The vector slice xs[128][kV] fp32 lives in shared memory; every lane reads
-// the same element at the same time (broadcast).
+// the same element at the same time (one broadcast wavefront), 16 bytes per load, so a slice
+// element costs 1/4 (kV = 1) to 2 (kV = 8) loads per symbol.
 // ---------------------------------------------------------------------------------------------
 template <int kV>
 struct Accum {
     float a[kV];
+    float4 cache;                       // the current 16 bytes of the slice (kV <= 2)
     __device__ __forceinline__ void clear()
     {
 #pragma unroll
         for (int v = 0; v < kV; ++v) a[v] = 0.0f;
     }
-    __device__ __forceinline__ void fma(float w, uint32_t xs_addr)
+    static __device__ __forceinline__ float4 lds_f4(uint32_t addr)
+    {
+        float4 x;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr));
+        return x;
+    }
+    // value w of position n (n is a compile-time constant after unrolling); xs = shared address of xs[0][0]
+    __device__ __forceinline__ void fma(int n, float w, uint32_t xs)
     {
         if constexpr (kV == 1) {
-            float x;
-            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(xs_addr));
+            if ((n & 3) == 0) cache = lds_f4(xs + n * 4);
+            const float x = (n & 3) == 0 ? cache.x : (n & 3) == 1 ? cache.y : (n & 3) == 2 ? cache.z : cache.w;
             a[0] = fmaf(w, x, a[0]);
         } else if constexpr (kV == 2) {
-            float x0, x1;
-            asm volatile("ld.shared.v2.f32 {%0,%1}, [%2];" : "=f"(x0), "=f"(x1) : "r"(xs_addr));
-            a[0] = fmaf(w, x0, a[0]);
-            a[1] = fmaf(w, x1, a[1]);
+            if ((n & 1) == 0) cache = lds_f4(xs + n * 8);
+            a[0] = fmaf(w, (n & 1) ? cache.z : cache.x, a[0]);
+            a[1] = fmaf(w, (n & 1) ? cache.w : cache.y, a[1]);
         } else {
 #pragma unroll
             for (int q = 0; q < kV / 4; ++q) {
-                float x0, x1, x2, x3;
-                asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(xs_addr + q * 16));
-                a[q * 4 + 0] = fmaf(w, x0, a[q * 4 + 0]);
-                a[q * 4 + 1] = fmaf(w, x1, a[q * 4 + 1]);
-                a[q * 4 + 2] = fmaf(w, x2, a[q * 4 + 2]);
-                a[q * 4 + 3] = fmaf(w, x3, a[q * 4 + 3]);
+                const float4 x = lds_f4(xs + n * (kV * 4) + q * 16);
+                a[q * 4 + 0] = fmaf(w, x.x, a[q * 4 + 0]);
+                a[q * 4 + 1] = fmaf(w, x.y, a[q * 4 + 1]);
+                a[q * 4 + 2] = fmaf(w, x.z, a[q * 4 + 2]);
+                a[q * 4 + 3] = fmaf(w, x.w, a[q * 4 + 3]);
             }
+        }
+    }
+    // out-of-order correction at a run-time position (outlier fix-up)
+    __device__ __forceinline__ void fma_at(uint32_t loc, float w, uint32_t xs)
+    {
+#pragma unroll
+        for (int v = 0; v < kV; ++v) {
+            float x;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(xs + (loc * kV + v) * 4));
+            a[v] = fmaf(w, x, a[v]);
         }
     }
 };
@@ -437,7 +454,7 @@ __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base
     const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
     uint32_t packed = 0;
     const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym) {
-        acc.fma(__uint_as_float(v), xs + n * (kV * 4));
+        acc.fma(n, __uint_as_float(v), xs);
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
     });
@@ -456,136 +473,284 @@ __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base
             const uint32_t sym = (word >> ((loc & 7u) * 4)) & 15u;
             const float mapped = __uint_as_float(lds_u32(ws.tab + sym * 128));
             const float outlier = __half2float(__float2half_rn(fp8_to_float(f >> 7) * T));
-            acc.fma(outlier - mapped, xs + loc * (kV * 4));
+            acc.fma_at(loc, outlier - mapped, xs);
         }
     }
 }
 
-// K2: y[b][n] = sum_k W~[n][k] x[b][k].  A CTA owns kWarps*32 rows and a contiguous range of
-// k-blocks; a thread owns one row and walks the range.  Partial sums go to the workspace
-// [ksplit][kV][n_out]; the last CTA of a row tile (ticket counter) adds them in a fixed order,
-// so the result does not depend on scheduling.
-template <int kV, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
-ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                 const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
-                 unsigned int* __restrict__ d_tickets, int ksplit)
+// Contiguous split of U work units over G CTAs: CTA c owns [unit_begin(c), unit_begin(c + 1)).
+__host__ __device__ __forceinline__ int64_t unit_begin(int64_t U, int G, int c) { return U * c / G; }
+__host__ __device__ __forceinline__ int unit_owner(int64_t U, int G, int64_t u)
 {
-    extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    __shared__ unsigned int ticket;
+    int c = static_cast<int>(u * G / U);
+    while (c + 1 < G && unit_begin(U, G, c + 1) <= u) ++c;
+    while (c > 0 && unit_begin(U, G, c) > u) --c;
+    return c;
+}
+
+template <int kWarps>
+__device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
+{
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t smem_base = smem_u32(smem);
     constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
-    constexpr uint32_t kXsBytes = kGroup * kV * 4;
     WarpSmem ws;
     ws.bits = smem_base + kSmemWarpBase + warp * kWarpBytes + lane * 4;
     ws.tab = ws.bits + kBitsBytes;
     ws.syms = ws.tab + kTabBytes;
     sts_u32(ws.bits + 16 * 128, 0u);
     sts_u32(ws.bits + 17 * 128, 0u);
+    return ws;
+}
+
+// K2: y[b][n] = sum_k W~[n][k] x[b][k].  A work unit is (row tile of kWarps*32 rows, one k-block);
+// units are numbered row tile major and dealt to the persistent CTAs in contiguous runs, so a
+// thread (= one row) keeps its partial sums in registers across the k-blocks of its run.  When a
+// row tile is shared by several CTAs each writes its partial sums to its own workspace slot and
+// the last to arrive (ticket counter) adds the slots in CTA order: the result does not depend on
+// scheduling.  Workspace: partial[slot][kV][rows per tile] floats, then one ticket per row tile.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                 const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+                 unsigned int* __restrict__ d_tickets)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    __shared__ unsigned int ticket;
+    constexpr int kRows = kWarps * 32;
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    constexpr uint32_t kXsBytes = kGroup * kV * 4;
+    const uint32_t smem_base = smem_u32(smem);
+    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
     float* xs_ptr = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);   // two slices
     const uint32_t xs_base = smem_u32(xs_ptr);
 
-    const int row_tile = blockIdx.x, split = blockIdx.y;
-    const int row = row_tile * (kWarps * 32) + static_cast<int>(threadIdx.x);
-    const bool row_ok = row < n_out;
-    const int kb_lo = static_cast<int>(static_cast<int64_t>(kblocks) * split / ksplit);
-    const int kb_hi = static_cast<int>(static_cast<int64_t>(kblocks) * (split + 1) / ksplit);
+    const int G = gridDim.x, c = blockIdx.x;
+    const int row_tiles = (n_out + kRows - 1) / kRows;
+    const int64_t U = static_cast<int64_t>(row_tiles) * kblocks;
+    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
     const int k = kblocks * kGroup;
+    const int tid = static_cast<int>(threadIdx.x);
 
     // rows past the end of the matrix decode the last row again and store nothing
+    auto block_ptr = [&](int64_t u) {
+        const int rt = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
+        const int row = min(rt * kRows + tid, n_out - 1);
+        return d_blocks + (static_cast<uint64_t>(row) * kblocks + kb) * kBlockBytes;
+    };
     Block blk;
-    const uint8_t* row_blocks = d_blocks + static_cast<uint64_t>(row_ok ? row : n_out - 1) * kblocks * kBlockBytes;
-    if (kb_lo < kb_hi) ldg_block(blk, row_blocks + static_cast<uint64_t>(kb_lo) * kBlockBytes);
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!stage_tables(smem, d_meta, &bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     Accum<kV> acc;
     acc.clear();
-    for (int kb = kb_lo; kb < kb_hi; ++kb) {
+    auto flush = [&](int rt) {
+        const int row = rt * kRows + tid;
+        const bool row_ok = row < n_out;
+        const int c_lo = unit_owner(U, G, static_cast<int64_t>(rt) * kblocks);
+        const int c_hi = unit_owner(U, G, static_cast<int64_t>(rt + 1) * kblocks - 1);
+        if (c_lo == c_hi) {                                // this CTA owns the whole row tile
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b)
+                    if (b < batch) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
+            }
+            return;
+        }
+        // staircase of (CTA, row tile) pairs: slot = c + rt is unique
+        float* mine = d_partial + static_cast<size_t>(c + rt) * kV * kRows;
+#pragma unroll
+        for (int b = 0; b < kV; ++b) mine[b * kRows + tid] = acc.a[b];
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) ticket = atomicAdd(&d_tickets[rt], 1u);
+        __syncthreads();
+        if (ticket == static_cast<unsigned int>(c_hi - c_lo)) {   // last of the CTAs that share this row tile
+            __threadfence();
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b) {
+                    if (b >= batch) continue;
+                    float sum = 0.0f;
+                    for (int cc = c_lo; cc <= c_hi; ++cc)
+                        sum += __ldcg(d_partial + (static_cast<size_t>(cc + rt) * kV + b) * kRows + tid);
+                    d_y[static_cast<size_t>(b) * n_out + row] = sum;
+                }
+            }
+            if (tid == 0) d_tickets[rt] = 0;               // ready for the next call on this workspace
+        }
+        __syncthreads();                                   // `ticket` may be rewritten by the next flush
+    };
+
+    int cur_rt = static_cast<int>(u0 / kblocks);
+    for (int64_t u = u0; u < u1; ++u) {
+        const int rt = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
+        if (rt != cur_rt) { flush(cur_rt); acc.clear(); cur_rt = rt; }
         // stage x[b][kb*128 .. +128) as fp32 xs[i][b] (rows beyond `batch` are zero)
-        float* xs = xs_ptr + ((kb - kb_lo) & 1) * (kGroup * kV);
-        for (int i = threadIdx.x; i < kGroup * kV; i += kWarps * 32) {
+        const int buf = static_cast<int>((u - u0) & 1);
+        float* xs = xs_ptr + buf * (kGroup * kV);
+        for (int i = tid; i < kGroup * kV; i += kRows) {
             const int b = i % kV, e = i / kV;
             xs[i] = (b < batch) ? __half2float(d_x[static_cast<size_t>(b) * k + kb * kGroup + e]) : 0.0f;
         }
         __syncthreads();                                   // slice visible; the other slice is free again
-        {
-            const Block cur = blk;
-            if (kb + 1 < kb_hi) ldg_block(blk, row_blocks + static_cast<uint64_t>(kb + 1) * kBlockBytes);
-            fused_group<kV>(cur, smem_base, ws, T, xs_base + ((kb - kb_lo) & 1) * kXsBytes, acc);
-        }
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        fused_group<kV>(cur, smem_base, ws, T, xs_base + buf * kXsBytes, acc);
     }
-    if (ksplit == 1) {
-        if (row_ok) {
-#pragma unroll
-            for (int b = 0; b < kV; ++b)
-                if (b < batch) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
-        }
-        return;
-    }
-    if (row_ok)
-#pragma unroll
-        for (int b = 0; b < kV; ++b)
-            if (b < batch) d_partial[(static_cast<size_t>(split) * kV + b) * n_out + row] = acc.a[b];
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) ticket = atomicAdd(&d_tickets[row_tile], 1u);
-    __syncthreads();
-    if (ticket != static_cast<unsigned int>(ksplit - 1)) return;
-    __threadfence();
-    if (row_ok)
-        for (int b = 0; b < batch; ++b) {
-            float s = 0.0f;
-            for (int sp = 0; sp < ksplit; ++sp) s += __ldcg(&d_partial[(static_cast<size_t>(sp) * kV + b) * n_out + row]);
-            d_y[static_cast<size_t>(b) * n_out + row] = s;
-        }
-    if (threadIdx.x == 0) d_tickets[row_tile] = 0;         // ready for the next call on this workspace
+    if (u0 < u1) flush(cur_rt);
 }
 
-// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / kV][t].  A CTA owns one (batch, kv head)
-// pair and a run of kWarps*32 tokens per iteration; a thread owns one token.
+// K2 for one or two rows of x: the slice is small enough (512 B or 1 KB) for every warp to keep
+// its own, so warps never meet at a barrier.  A work unit is (32 consecutive rows, one k-block),
+// numbered row-tile major; every warp of the grid owns a contiguous run of units, keeps its rows'
+// partial sums in registers along k, and shares a row tile with the neighbouring warps through
+// the same slot-and-ticket scheme as above (slot = global warp id + row tile, 32 floats per row
+// of x).  Workspace: partial[slot][kV][32] floats, then one ticket per 32-row tile.
 template <int kV, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
-ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int seq, int q_per_kv,
-                        const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores, int chunks_per_head)
+ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                      const __half* __restrict__ d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
+                      unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ uint64_t bar;
-    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const uint32_t smem_base = smem_u32(smem);
     constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
-    WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * kWarpBytes + lane * 4;
-    ws.tab = ws.bits + kBitsBytes;
-    ws.syms = ws.tab + kTabBytes;
-    sts_u32(ws.bits + 16 * 128, 0u);
-    sts_u32(ws.bits + 17 * 128, 0u);
+    constexpr uint32_t kXsBytes = kGroup * kV * 4;
+    const uint32_t smem_base = smem_u32(smem);
+    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    const uint32_t xs = smem_base + kSmemWarpBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
+
+    const int wg = static_cast<int>(blockIdx.x) * kWarps + warp;
+    const int tiles = (n_out + 31) / 32;
+    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    // never more working warps than units: every warp in [0, W) owns at least one unit, the rest idle
+    const int W = static_cast<int>(min(static_cast<int64_t>(gridDim.x) * kWarps, U));
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    const int k = kblocks * kGroup;
+    auto block_ptr = [&](int64_t u) {
+        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
+        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
+    };
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    Accum<kV> acc;
+    acc.clear();
+    auto flush = [&](int tile) {
+        const int row = tile * 32 + lane;
+        const bool row_ok = row < n_out;
+        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
+        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
+        if (w_lo == w_hi) {
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
+            }
+            return;
+        }
+        float* mine = d_partial + static_cast<size_t>(wg + tile) * kV * 32;
+#pragma unroll
+        for (int b = 0; b < kV; ++b) mine[b * 32 + lane] = acc.a[b];
+        __threadfence();
+        __syncwarp();
+        unsigned int t = 0;
+        if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t == static_cast<unsigned int>(w_hi - w_lo)) {  // last of the warps that share this tile
+            __threadfence();
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b) {
+                    float sum = 0.0f;
+                    for (int ww = w_lo; ww <= w_hi; ++ww)
+                        sum += __ldcg(d_partial + (static_cast<size_t>(ww + tile) * kV + b) * 32 + lane);
+                    d_y[static_cast<size_t>(b) * n_out + row] = sum;
+                }
+            }
+            if (lane == 0) d_tickets[tile] = 0;
+        }
+    };
+
+    int cur_tile = static_cast<int>(u0 / kblocks);
+    for (int64_t u = u0; u < u1; ++u) {
+        const int tile = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
+        if (tile != cur_tile) { flush(cur_tile); acc.clear(); cur_tile = tile; }
+        // this warp's slice: lane l converts x[b][kb*128 + 4l .. 4l+3] to fp32, layout xs[i][b]
+        __syncwarp();
+        {
+            float v[kV][4];
+#pragma unroll
+            for (int b = 0; b < kV; ++b) {
+                const uint2 raw = *reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4);
+                const __half2 h0 = *reinterpret_cast<const __half2*>(&raw.x), h1 = *reinterpret_cast<const __half2*>(&raw.y);
+                v[b][0] = __low2float(h0); v[b][1] = __high2float(h0); v[b][2] = __low2float(h1); v[b][3] = __high2float(h1);
+            }
+            if constexpr (kV == 1) {
+                sts_v4(xs + lane * 16, __float_as_uint(v[0][0]), __float_as_uint(v[0][1]), __float_as_uint(v[0][2]), __float_as_uint(v[0][3]));
+            } else {
+                sts_v4(xs + lane * 32, __float_as_uint(v[0][0]), __float_as_uint(v[1][0]), __float_as_uint(v[0][1]), __float_as_uint(v[1][1]));
+                sts_v4(xs + lane * 32 + 16, __float_as_uint(v[0][2]), __float_as_uint(v[1][2]), __float_as_uint(v[0][3]), __float_as_uint(v[1][3]));
+            }
+        }
+        __syncwarp();
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        fused_group<kV>(cur, smem_base, ws, T, xs, acc);
+    }
+    if (u0 < u1) flush(cur_tile);
+}
+
+// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t].  A work unit is (one (batch, kv
+// head) pair, a chunk of kWarps*32 tokens); units are dealt to persistent CTAs in contiguous runs,
+// the query slice is restaged when the head changes, a thread owns one token.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
+                        int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    constexpr int kTokens = kWarps * 32;
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    const uint32_t smem_base = smem_u32(smem);
+    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
     float* xs = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);
     const uint32_t xs_addr = smem_u32(xs);
 
-    const int bh = blockIdx.x / chunks_per_head, chunk = blockIdx.x % chunks_per_head;   // bh = b * n_kv_heads + h
-    const int tile = kWarps * 32;
-    int t = chunk * tile + static_cast<int>(threadIdx.x);
-    const uint8_t* head_blocks = d_kblocks + static_cast<uint64_t>(bh) * seq * kBlockBytes;
-    // the loop below runs whole warps: lanes past the end of the sequence decode the last token
-    // again and store nothing
+    const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
+    const int chunks = (seq + kTokens - 1) / kTokens;
+    const int64_t U = static_cast<int64_t>(heads) * chunks;
+    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
+    // lanes past the end of the sequence decode its last token again and store nothing
+    auto block_ptr = [&](int64_t u) {
+        const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    };
     Block blk;
-    const int t_warp = t - static_cast<int>(lane);
-    if (t_warp < seq) ldg_block(blk, head_blocks + static_cast<uint64_t>(min(t, seq - 1)) * kBlockBytes);
-    // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
-    for (int i = threadIdx.x; i < kGroup * kV; i += tile) {
-        const int r = i % kV, d = i / kV;
-        xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
-    }
-    if (!stage_tables(smem, d_meta, &bar)) return;        // also orders the xs writes (barrier inside)
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!stage_tables(smem, d_meta, &bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
-    for (; t - static_cast<int>(lane) < seq; t += chunks_per_head * tile) {
+    int cur_bh = -1;
+    for (int64_t u = u0; u < u1; ++u) {
+        const int bh = static_cast<int>(u / chunks), t = static_cast<int>(u % chunks) * kTokens + tid;
+        if (bh != cur_bh) {
+            __syncthreads();                               // everyone is done with the previous head's slice
+            // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
+            for (int i = tid; i < kGroup * kV; i += kTokens) {
+                const int r = i % kV, d = i / kV;
+                xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
+            }
+            __syncthreads();
+            cur_bh = bh;
+        }
         const Block cur = blk;
-        const int tn = t + chunks_per_head * tile;
-        if (tn - static_cast<int>(lane) < seq) ldg_block(blk, head_blocks + static_cast<uint64_t>(min(tn, seq - 1)) * kBlockBytes);
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         Accum<kV> acc;
         acc.clear();
         fused_group<kV>(cur, smem_base, ws, T, xs_addr, acc);
@@ -642,19 +807,38 @@ int check_launch()
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 constexpr int kDecompressWarps = 32;
-constexpr int kFusedWarps = 16;
+// warps per CTA of the fused kernels: as many as shared memory allows; 20 for eight dot products
+// per group, whose accumulators need the larger register budget (96 instead of 80 per thread)
+constexpr int fused_warps(int kV) { return kV >= 8 ? 20 : 22; }
+// per-warp GEMV: every warp also carries its own slice of x, which leaves room for 22 / 20 warps
+constexpr int gemv_warp_warps(int kV) { return kV >= 2 ? 20 : 22; }
 
-struct GemvPlan { int row_tiles, ksplit; size_t partial_bytes, ticket_bytes; };
+// GEMV launch plan: one persistent CTA per SM (fewer if there are fewer work units), workspace of
+// (CTAs + row tiles) partial slots and one ticket per row tile.
+struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
 
-GemvPlan gemv_plan(int n_out, int kblocks, int vpad, int sms)
+GemvPlan gemv_plan(int n_out, int kblocks, int vpad, int ctas_max)
 {
     GemvPlan p;
-    const int rows_per_cta = kFusedWarps * 32;
-    p.row_tiles = (n_out + rows_per_cta - 1) / rows_per_cta;
-    // enough k-splits to give every SM a CTA, at most one per k-block
-    int want = (sms + p.row_tiles - 1) / p.row_tiles;
-    p.ksplit = want < 1 ? 1 : (want > kblocks ? kblocks : want);
-    p.partial_bytes = p.ksplit > 1 ? static_cast<size_t>(p.ksplit) * vpad * n_out * sizeof(float) : 0;
+    const int kFusedRows = fused_warps(vpad) * 32;
+    p.row_tiles = (n_out + kFusedRows - 1) / kFusedRows;
+    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
+    p.grid = static_cast<int>(units < ctas_max ? units : ctas_max);
+    p.partial_bytes = static_cast<size_t>(p.grid + p.row_tiles) * vpad * kFusedRows * sizeof(float);
+    p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return p;
+}
+
+// plan of the per-warp GEMV (one or two rows of x)
+GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
+{
+    GemvPlan p;
+    p.row_tiles = (n_out + 31) / 32;
+    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
+    const int64_t ctas = (units + gemv_warp_warps(vpad) - 1) / gemv_warp_warps(vpad);
+    p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
+    p.partial_bytes = static_cast<size_t>(p.grid * gemv_warp_warps(vpad) + p.row_tiles) * vpad * 32 * sizeof(float);
     p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
     p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
     return p;
@@ -760,20 +944,17 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
 extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch)
 {
     if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return 0;
-    // sized for the largest plan any supported device can ask for (k-split count <= 256)
-    const int rows_per_cta = kFusedWarps * 32;
-    const int row_tiles = (n_out + rows_per_cta - 1) / rows_per_cta;
-    const int kblocks = k / kGroup;
-    const int ksplit = kblocks < 256 ? kblocks : 256;
-    size_t partial = (static_cast<size_t>(ksplit) * pad_v(batch) * n_out * sizeof(float) + 255) & ~static_cast<size_t>(255);
-    size_t tickets = (static_cast<size_t>(row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
-    return partial + tickets;
+    // sized for the largest plan any supported device can ask for (at most 256 persistent CTAs)
+    const GemvPlan p = pad_v(batch) <= 2 ? gemv_warp_plan(n_out, k / kGroup, pad_v(batch), 256)
+                                         : gemv_plan(n_out, k / kGroup, pad_v(batch), 256);
+    return p.partial_bytes + p.ticket_bytes;
 }
 
 template <int kV>
 static int launch_gemv(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
                        const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
+    constexpr int kFusedWarps = fused_warps(kV);
     auto kernel = ecco_gemv_kernel<kV, kFusedWarps>;
     const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + 2 * kGroup * kV * 4;
     static thread_local bool configured[64] = {};
@@ -782,21 +963,42 @@ static int launch_gemv(const DeviceInfo& di, const void* d_meta, const uint8_t* 
         if (rc) return rc;
         configured[di.device] = true;
     }
-    const GemvPlan p = gemv_plan(n_out, kblocks, kV, di.sms);
-    float* partial = nullptr;
-    unsigned int* tickets = nullptr;
-    if (p.ksplit > 1) {
-        if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
-        if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
-        partial = static_cast<float*>(d_ws);
-        tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-        // the workspace's previous contents are irrelevant: tickets start from zero on every call
-        cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
-        if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    const GemvPlan p = gemv_plan(n_out, kblocks, kV, di.sms < 256 ? di.sms : 256);
+    if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
+    if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
+    float* partial = static_cast<float*>(d_ws);
+    unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
+    // the workspace's previous contents are irrelevant: tickets start from zero on every call
+    cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    kernel<<<p.grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
+                                                       static_cast<const __half*>(d_x), batch, d_y, partial, tickets);
+    return check_launch();
+}
+
+// one or two rows of x (batch == kV): the per-warp kernel
+template <int kV>
+static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
+                            const void* d_x, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+{
+    constexpr int kFusedWarps = gemv_warp_warps(kV);
+    auto kernel = ecco_gemv_warp_kernel<kV, kFusedWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes + kGroup * kV * 4);
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        int rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
     }
-    dim3 grid(static_cast<unsigned>(p.row_tiles), static_cast<unsigned>(p.ksplit));
-    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
-                                                     static_cast<const __half*>(d_x), batch, d_y, partial, tickets, p.ksplit);
+    const GemvPlan p = gemv_warp_plan(n_out, kblocks, kV, di.sms < 256 ? di.sms : 256);
+    if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
+    if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
+    float* partial = static_cast<float*>(d_ws);
+    unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
+    cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    kernel<<<p.grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
+                                                       static_cast<const __half*>(d_x), d_y, partial, tickets);
     return check_launch();
 }
 
@@ -812,8 +1014,8 @@ extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int kblocks = k / kGroup;
     switch (pad_v(batch)) {
-        case 1: return launch_gemv<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
-        case 2: return launch_gemv<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+        case 1: return launch_gemv_warp<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
+        case 2: return launch_gemv_warp<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
         case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
         default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
     }
@@ -838,8 +1040,9 @@ extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, 
     if (rc) return rc;
     const int kblocks = k / kGroup, vpad = pad_v(batch);
     // refuse, before any launch, a shape whose plan does not fit the fixed array
-    const GemvPlan p = gemv_plan(n_out, kblocks, vpad, di.sms);
-    if (p.ksplit > 1 && p.partial_bytes + p.ticket_bytes > ECCO_STATIC_WORKSPACE_BYTES) return ECCO_ERR_WORKSPACE;
+    const int ctas = di.sms < 256 ? di.sms : 256;
+    const GemvPlan p = vpad <= 2 ? gemv_warp_plan(n_out, kblocks, vpad, ctas) : gemv_plan(n_out, kblocks, vpad, ctas);
+    if (p.partial_bytes + p.ticket_bytes > ECCO_STATIC_WORKSPACE_BYTES) return ECCO_ERR_WORKSPACE;
     // one-time set-up per device (the current device is di.device): resolve the array's address
     static std::mutex mu;
     static void* address[64] = {};
@@ -856,8 +1059,8 @@ extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, 
     }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (vpad) {
-        case 1: return launch_gemv<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
-        case 2: return launch_gemv<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        case 1: return launch_gemv_warp<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        case 2: return launch_gemv_warp<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
         case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
         default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
     }
@@ -867,6 +1070,7 @@ template <int kV>
 static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* d_kblocks, int batch, int n_kv_heads,
                        int seq, int q_per_kv, const void* d_q, float scale, float* d_scores, cudaStream_t stream)
 {
+    constexpr int kFusedWarps = fused_warps(kV), kFusedRows = kFusedWarps * 32;
     auto kernel = ecco_attn_scores_kernel<kV, kFusedWarps>;
     const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + kGroup * kV * 4;
     static thread_local bool configured[64] = {};
@@ -875,15 +1079,11 @@ static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* 
         if (rc) return rc;
         configured[di.device] = true;
     }
-    const int tile = kFusedWarps * 32;
     const int heads = batch * n_kv_heads;
-    const int max_chunks = (seq + tile - 1) / tile;
-    // about two CTAs per SM in total, at least one per head, at most one per tile of tokens
-    int chunks = (2 * di.sms + heads - 1) / heads;
-    chunks = chunks < 1 ? 1 : (chunks > max_chunks ? max_chunks : chunks);
-    const unsigned grid = static_cast<unsigned>(heads) * static_cast<unsigned>(chunks);
-    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, seq, q_per_kv,
-                                                     static_cast<const __half*>(d_q), scale, d_scores, chunks);
+    const int64_t units = static_cast<int64_t>(heads) * ((seq + kFusedRows - 1) / kFusedRows);
+    const unsigned grid = static_cast<unsigned>(units < di.sms ? units : di.sms);      // persistent CTAs
+    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, heads, seq, q_per_kv,
+                                                     static_cast<const __half*>(d_q), scale, d_scores);
     return check_launch();
 }
 
