@@ -38,13 +38,14 @@ METRIC, UNIT = "decompress_output_GBps", "GB/s"
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg5"],
-                    help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg5: long-context GQA K cache "
-                         "[16][8][32768][128] (decompress + attention scores with 8 query heads per KV head)")
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5"],
+                    help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg4: 70B-shaped MLP weights + stream-size "
+                         "sweep; cfg5: long-context GQA K cache [16][8][32768][128] (decompress + attention scores with 8 "
+                         "query heads per KV head)")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -191,6 +192,37 @@ def cpu_baseline(layer, c: int):
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
+WORKLOADS = {
+    "cfg2": dict(label="cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
+                       "+ cfg3 K cache [8][32][4096][128]",
+                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1",
+                 l2="inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
+    "cfg4": dict(label="cfg4 llama-70b-shaped MLP weights (gate, up 28672x8192; down 8192x28672; 5,505,024 groups)",
+                 step="decompress x3, gemv batch 1 x3; plus a decompress sweep over 64 MiB .. 4 GiB streams (stream_sweep)",
+                 l2="inputs larger than L2: each step streams 336 MiB of blocks and writes 1.3 GiB"),
+    "cfg5": dict(label="cfg5 long-context GQA K cache [16][8][32768][128] (4,194,304 groups)",
+                 step="decompress x1, attn_scores x1 (8 query heads per KV head)",
+                 l2="inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB"),
+    "small": dict(label="reduced (profiling): q + gate of cfg2, K cache [2][32][4096][128]",
+                  step="decompress x2, gemv batch 1 x2, gemv batch 8 x2, attn_scores x1",
+                  l2="inputs larger than L2 except the q projection"),
+}
+
+
+def build_workload(name, workloads):
+    """-> (weight tensors, kv tensor or None, q_per_kv, decompress_kv, default segments)."""
+    if name == "cfg5":
+        (kt,) = workloads.config5(which=("K",))
+        return [], kt, 8, True, ["decompress", "attn"]
+    if name == "cfg4":
+        return workloads.config4(), None, 1, False, ["decompress", "gemv1"]
+    if name == "small":
+        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, workloads.calibrate_kv(3, 32))
+        return workloads.config2(names=("q", "gate")), kt, 1, False, ["decompress", "gemv1", "gemv8", "attn"]
+    (kt,) = workloads.config3(which=("K",))
+    return workloads.config2(), kt, 1, False, ["decompress", "gemv1", "gemv8", "attn"]
+
+
 def run_ours(args):
     import torch
 
@@ -209,74 +241,63 @@ def run_ours(args):
     B.lib()
 
     # ---- workload (the same seeded tensors on every rank)
-    q_per_kv = 1
-    if args.workload == "cfg5":
-        (kt,) = workloads.config5(which=("K",))
-        layer, q_per_kv = [], 8
-    elif args.small:
-        layer = workloads.config2(names=("q", "gate"))
-        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, workloads.calibrate_kv(3, 32))
-    else:
-        layer = workloads.config2()
-        (kt,) = workloads.config3(which=("K",))
-    kb, kh, kseq, _ = kt.shape
+    wname = "small" if args.small else args.workload
+    weights, kt, q_per_kv, decompress_kv, default_segs = build_workload(wname, workloads)
+    segs = [s for s in args.only.split(",") if s] or default_segs
     stream = torch.cuda.current_stream()
-    dl = []
-    for t in layer:
+    need8 = "gemv8" in segs
+    mats = []                                       # weight matrices: decompress + GEMV targets
+    for t in weights:
         n_out, k = t.shape
-        wsb = B.ecco_gemv_workspace_bytes(n_out, k, 8)
-        dl.append(dict(t=t, n=t.n_groups, n_out=n_out, k=k, meta=B.meta_to_device(t.meta), blocks=torch.from_numpy(t.blocks).cuda(),
-                       out=torch.empty(t.n_groups * G, dtype=torch.float16, device="cuda"),
-                       x1=torch.from_numpy(synth.activations(1, k, 11)).cuda(), x8=torch.from_numpy(synth.activations(8, k, 12)).cuda(),
-                       y1=torch.empty((1, n_out), dtype=torch.float32, device="cuda"),
-                       y8=torch.empty((8, n_out), dtype=torch.float32, device="cuda"),
-                       ws=torch.empty(wsb, dtype=torch.uint8, device="cuda"), wsb=wsb))
-    k_meta, k_blocks = B.meta_to_device(kt.meta), torch.from_numpy(kt.blocks).cuda()
-    q = torch.from_numpy(synth.queries(kb, kh * q_per_kv, 13)).cuda()
-    scores = torch.empty((kb, kh * q_per_kv, kseq), dtype=torch.float32, device="cuda")
-    if args.workload == "cfg5":          # the cache itself is the tensor to decompress; no weight matrices, no GEMV
-        dl.append(dict(t=kt, n=kt.n_groups, meta=k_meta, blocks=k_blocks,
-                       out=torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")))
-    segs = [s for s in args.only.split(",") if s] or (["decompress", "attn"] if args.workload == "cfg5" else
-                                                         ["decompress", "gemv1", "gemv8", "attn"])
+        wsb = B.ecco_gemv_workspace_bytes(n_out, k, 8 if need8 else 1)
+        mats.append(dict(t=t, n=t.n_groups, n_out=n_out, k=k, meta=B.meta_to_device(t.meta), blocks=torch.from_numpy(t.blocks).cuda(),
+                         out=torch.empty(t.n_groups * G, dtype=torch.float16, device="cuda"),
+                         x1=torch.from_numpy(synth.activations(1, k, 11)).cuda(), x8=torch.from_numpy(synth.activations(8, k, 12)).cuda(),
+                         y1=torch.empty((1, n_out), dtype=torch.float32, device="cuda"),
+                         y8=torch.empty((8, n_out), dtype=torch.float32, device="cuda"),
+                         ws=torch.empty(wsb, dtype=torch.uint8, device="cuda"), wsb=wsb))
+    dec = list(mats)                                # decompress targets
+    kv = None
+    if kt is not None:
+        kb, kh, kseq, _ = kt.shape
+        kv = dict(t=kt, n=kt.n_groups, meta=B.meta_to_device(kt.meta), blocks=torch.from_numpy(kt.blocks).cuda(),
+                  q=torch.from_numpy(synth.queries(kb, kh * q_per_kv, 13)).cuda(),
+                  scores=torch.empty((kb, kh * q_per_kv, kseq), dtype=torch.float32, device="cuda"))
+        if decompress_kv:
+            kv["out"] = torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")
+            dec.append(kv)
 
-    def step():
-        if "decompress" in segs:
-            for d in dl:
-                B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
-        if "gemv1" in segs:
-            for d in dl:
-                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1"], 1, d["y1"], d["ws"], d["wsb"], stream)
-        if "gemv8" in segs:
-            for d in dl:
-                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
-        if "attn" in segs:
-            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, q_per_kv, q, 128 ** -0.5, scores, stream)
+    def seg_decompress():
+        for d in dec:
+            B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
 
-    def timed_step(ev):
-        ev[0].record(stream)
-        if "decompress" in segs:
-            for d in dl:
-                B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
-        ev[1].record(stream)
-        if "gemv1" in segs:
-            for d in dl:
-                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1"], 1, d["y1"], d["ws"], d["wsb"], stream)
-        ev[2].record(stream)
-        if "gemv8" in segs:
-            for d in dl:
-                B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x8"], 8, d["y8"], d["ws"], d["wsb"], stream)
-        ev[3].record(stream)
-        if "attn" in segs:
-            B.ecco_attn_scores(k_meta, k_blocks, kb, kh, kseq, q_per_kv, q, 128 ** -0.5, scores, stream)
-        ev[4].record(stream)
+    def seg_gemv(b):
+        for d in mats:
+            B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1" if b == 1 else "x8"], b, d["y1" if b == 1 else "y8"],
+                        d["ws"], d["wsb"], stream)
+
+    def seg_attn():
+        if kv is not None:
+            B.ecco_attn_scores(kv["meta"], kv["blocks"], kb, kh, kseq, q_per_kv, kv["q"], 128 ** -0.5, kv["scores"], stream)
+
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        if "decompress" in segs: seg_decompress()
+        if ev: ev[1].record(stream)
+        if "gemv1" in segs: seg_gemv(1)
+        if ev: ev[2].record(stream)
+        if "gemv8" in segs: seg_gemv(8)
+        if ev: ev[3].record(stream)
+        if "attn" in segs: seg_attn()
+        if ev: ev[4].record(stream)
 
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
         step()
     events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     sampler = ClockSampler(local)
@@ -285,7 +306,7 @@ def run_ours(args):
     launches0 = B.ecco_kernel_launch_count()
     barrier()
     for ev in events:
-        timed_step(ev)
+        step(ev)
     barrier()
     launches = B.ecco_kernel_launch_count() - launches0
     clocks = sampler.stop()
@@ -295,18 +316,18 @@ def run_ours(args):
     seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(4)]
     total_ms, dec_ms, g1_ms, g8_ms, at_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
 
-    groups = sum(d["n"] for d in dl)
+    groups = sum(d["n"] for d in dec)
     out_bytes = groups * G * 2
     value = world * out_bytes * args.steps / (dec_ms / 1e3) / 1e9 if dec_ms > 0 else 0.0
 
     # ---- end to end through the C ABI with host buffers: H2D of the blocks, decompress, D2H of the fp16
     e2e = None
-    if "decompress" in segs:
-        h_in = [torch.from_numpy(d["t"].blocks).pin_memory() for d in dl]
-        h_out = [torch.empty(d["n"] * G, dtype=torch.float16).pin_memory() for d in dl]
+    if "decompress" in segs and dec:
+        h_in = [torch.from_numpy(d["t"].blocks).pin_memory() for d in dec]
+        h_out = [torch.empty(d["n"] * G, dtype=torch.float16).pin_memory() for d in dec]
 
         def e2e_step():
-            for d, hi, ho in zip(dl, h_in, h_out):
+            for d, hi, ho in zip(dec, h_in, h_out):
                 d["blocks"].copy_(hi, non_blocking=True)
                 B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
                 ho.copy_(d["out"], non_blocking=True)
@@ -324,6 +345,31 @@ def run_ours(args):
         (ems,) = distutil.max_over_ranks([e0.elapsed_time(e1)], dist, "cuda")
         e2e = {"value": world * out_bytes * esteps / (ems / 1e3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": groups * BLOCK, "d2h_bytes_per_step": out_bytes, "steps": esteps}
+        del h_in, h_out
+
+    # ---- cfg4 only: standalone decompress over streams of 64 MiB .. 4 GiB (the gate matrix's blocks, tiled)
+    sweep = None
+    if wname == "cfg4" and rank == 0 and "decompress" in segs:
+        gate = mats[0]
+        sweep = []
+        for mib in (64, 256, 1024, 4096):
+            n = mib * (1 << 20) // BLOCK
+            reps = -(-n // gate["n"])
+            blocks = gate["blocks"].repeat(reps, 1)[:n].contiguous()
+            out = torch.empty(n * G, dtype=torch.float16, device="cuda")
+            for _ in range(2):
+                B.ecco_decompress(gate["meta"], blocks, n, out, stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps_t = 5
+            e0.record(stream)
+            for _ in range(reps_t):
+                B.ecco_decompress(gate["meta"], blocks, n, out, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps_t
+            sweep.append({"compressed_MiB": mib, "groups": n, "us": us, "output_GBps": n * G * 2 / us / 1e3,
+                          "hbm_frac": n * (BLOCK + G * 2) / us / 1e3 / measured_peaks()[0]})
+            del blocks, out
 
     if rank != 0:
         if dist is not None:
@@ -331,7 +377,7 @@ def run_ours(args):
         return
 
     peak, peak_kind = measured_peaks()
-    n_launch = len(dl)
+    n_launch = max(1, len(dec))
     avg_launch_s = dec_ms / 1e3 / (args.steps * n_launch) if dec_ms > 0 else float("nan")
     alg_bytes_per_launch = groups * (BLOCK + G * 2) / n_launch
     achieved = alg_bytes_per_launch / avg_launch_s / 1e9 if dec_ms > 0 else 0.0
@@ -340,29 +386,47 @@ def run_ours(args):
     if os.path.exists(tp):
         with open(tp) as f:
             traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
+    # the fused kernels against the same HBM peak (algorithmic bytes: blocks + vectors + results); what bounds them
+    # is the SM load/store pipe, so the symbol rate is reported next to the HBM fraction
+    seg_total = dec_ms + g1_ms + g8_ms + at_ms
+    kernels = []
+
+    def kernel_entry(name, ms, alg_bytes_per_step, symbols_per_step):
+        if ms <= 0 or symbols_per_step == 0:
+            return
+        sec = ms / 1e3 / args.steps
+        kernels.append({"kernel": name, "share_of_step": ms / seg_total, "us_per_step": sec * 1e6,
+                        "hbm_GBps": alg_bytes_per_step / sec / 1e9, "hbm_frac": alg_bytes_per_step / sec / 1e9 / peak,
+                        "Gsymbols_per_s": symbols_per_step / sec / 1e9})
+
+    w_groups = sum(d["n"] for d in mats)
+    gemv_vec = lambda b: sum(2 * b * d["k"] + 4 * b * d["n_out"] for d in mats)
+    kernel_entry("ecco_decompress", dec_ms if "decompress" in segs else 0, groups * (BLOCK + G * 2), groups * G)
+    kernel_entry("ecco_gemv batch 1", g1_ms if "gemv1" in segs else 0, w_groups * BLOCK + gemv_vec(1), w_groups * G)
+    kernel_entry("ecco_gemv batch 8", g8_ms if "gemv8" in segs else 0, w_groups * BLOCK + gemv_vec(8), w_groups * G)
+    if kv is not None:
+        kernel_entry(f"ecco_attn_scores q_per_kv {q_per_kv}", at_ms if "attn" in segs else 0, kv["n"] * (BLOCK + 4 * q_per_kv), kv["n"] * G)
+    info = WORKLOADS[wname]
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
         "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic",
-        "config": {"workload": ("cfg5 long-context GQA K cache [16][8][32768][128] (4,194,304 groups)" if args.workload == "cfg5" else
-                                "reduced (profiling): q+gate, K cache batch 2" if args.small else
-                                "cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
-                                "+ cfg3 K cache [8][32][4096][128]"),
-                   "step": ("decompress x1, attn_scores x1 (8 query heads per KV head)" if args.workload == "cfg5" else
-                            "decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1"),
-                   "l2": ("inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB" if args.workload == "cfg5" else
-                          "inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
+        "config": {"workload": info["label"], "step": info["step"], "segments": segs, "l2": info["l2"],
                    "format": "S=64, H=4, group 128, 64-byte blocks"},
-        "segments_us_per_step": {"decompress_layer": dec_ms / args.steps * 1e3, "gemv_layer_batch1": g1_ms / args.steps * 1e3,
-                                 "gemv_layer_batch8": g8_ms / args.steps * 1e3, "attn_scores_cfg3": at_ms / args.steps * 1e3},
-        "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3,
+        "segments_us_per_step": {"decompress": dec_ms / args.steps * 1e3, "gemv_batch1": g1_ms / args.steps * 1e3,
+                                 "gemv_batch8": g8_ms / args.steps * 1e3, "attn_scores": at_ms / args.steps * 1e3},
+        "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3 if wname == "cfg2" else None,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
-        "roofline": {"kernel": "ecco_decompress_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
-                     "algorithmic_bytes_per_launch": alg_bytes_per_launch, "avg_launch_us": avg_launch_s * 1e6},
+                     "algorithmic_bytes_per_launch": alg_bytes_per_launch, "avg_launch_us": avg_launch_s * 1e6,
+                     "note": "kernel of the headline metric; limited by the SM load/store pipe, see kernels[] and profiles/"},
+        "kernels": kernels,
     }
-    if world == 1 and not args.no_cpu_baseline:
-        line["cpu_baseline"] = cpu_baseline([d["t"] for d in dl], cores())
+    if sweep is not None:
+        line["stream_sweep"] = sweep
+    if world == 1 and not args.no_cpu_baseline and dec:
+        line["cpu_baseline"] = cpu_baseline([d["t"] for d in dec], cores())
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
