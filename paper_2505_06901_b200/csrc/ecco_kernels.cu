@@ -261,7 +261,7 @@ __device__ __forceinline__ uint32_t read_pad(const WarpSmem& ws, int j)
 template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
-                       uint16_t* __restrict__ d_out)
+                       uint16_t* __restrict__ d_out, uint32_t active_warps)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ uint64_t bar;
@@ -275,8 +275,11 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
     sts_u32(ws.bits + 17 * 128, 0u);
 
     const uint64_t n_tiles = (n_groups + 31) / 32;
-    const uint64_t tile_stride = static_cast<uint64_t>(gridDim.x) * kWarps;
-    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;   // warps of one CTA take tiles far apart
+    // the host picks active_warps so that every working warp gets the same number of tiles (+-1 over
+    // the whole grid); warp ids interleave over the CTAs, so every SM keeps the same number busy
+    const uint64_t tile_stride = active_warps;
+    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
+    if (tile >= tile_stride) tile = n_tiles;               // this warp sits the launch out (after the table barrier)
     Block blk;
     // lanes past the end of the tensor decode the last group again and store nothing
     if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
@@ -319,7 +322,7 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
 template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
-                           uint16_t* __restrict__ d_out, const __grid_constant__ CUtensorMap out_map)
+                           uint16_t* __restrict__ d_out, uint32_t active_warps, const __grid_constant__ CUtensorMap out_map)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ uint64_t bar;
@@ -337,8 +340,9 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
     const uint32_t my_row = stage + lane * 32;
 
     const uint64_t n_tiles = (n_groups + 31) / 32;
-    const uint64_t tile_stride = static_cast<uint64_t>(gridDim.x) * kWarps;
+    const uint64_t tile_stride = active_warps;             // see ecco_decompress_kernel
     uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
+    if (tile >= tile_stride) tile = n_tiles;
     Block blk;
     if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
     if (!stage_tables(smem, d_meta, &bar)) return;
@@ -612,7 +616,7 @@ template <int kV, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
                       const __half* __restrict__ d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
-                      unsigned int* __restrict__ d_tickets)
+                      unsigned int* __restrict__ d_tickets, int active_warps)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     __shared__ uint64_t bar;
@@ -623,11 +627,12 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     const uint32_t xs = smem_base + kSmemWarpBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
 
-    const int wg = static_cast<int>(blockIdx.x) * kWarps + warp;
+    // W working warps (chosen by the host so that they all get the same number of units, and never
+    // more than there are units); warp ids interleave over the CTAs; the other warps idle
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
     const int tiles = (n_out + 31) / 32;
     const int64_t U = static_cast<int64_t>(tiles) * kblocks;
-    // never more working warps than units: every warp in [0, W) owns at least one unit, the rest idle
-    const int W = static_cast<int>(min(static_cast<int64_t>(gridDim.x) * kWarps, U));
+    const int W = active_warps;
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     const int k = kblocks * kGroup;
     auto block_ptr = [&](int64_t u) {
@@ -666,9 +671,18 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
             if (row_ok) {
 #pragma unroll
                 for (int b = 0; b < kV; ++b) {
+                    // slots are added in warp order whatever the arrival order; loads go out sixteen at a time
+                    const float* slot = d_partial + (static_cast<size_t>(w_lo + tile) * kV + b) * 32 + lane;
                     float sum = 0.0f;
-                    for (int ww = w_lo; ww <= w_hi; ++ww)
-                        sum += __ldcg(d_partial + (static_cast<size_t>(ww + tile) * kV + b) * 32 + lane);
+                    int ww = w_lo;
+                    for (; ww + 16 <= w_hi + 1; ww += 16, slot += 16 * kV * 32) {
+                        float v[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = __ldcg(slot + i * kV * 32);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) sum += v[i];
+                    }
+                    for (; ww <= w_hi; ++ww, slot += kV * 32) sum += __ldcg(slot);
                     d_y[static_cast<size_t>(b) * n_out + row] = sum;
                 }
             }
@@ -676,9 +690,18 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         }
     };
 
+    // x for a unit is fetched one unit ahead, like the block
+    uint2 xraw[kV];
+    auto load_x = [&](int64_t u) {
+        const int kb = static_cast<int>(u % kblocks);
+#pragma unroll
+        for (int b = 0; b < kV; ++b)
+            xraw[b] = __ldg(reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4));
+    };
+    if (u0 < u1) load_x(u0);
     int cur_tile = static_cast<int>(u0 / kblocks);
     for (int64_t u = u0; u < u1; ++u) {
-        const int tile = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
+        const int tile = static_cast<int>(u / kblocks);
         if (tile != cur_tile) { flush(cur_tile); acc.clear(); cur_tile = tile; }
         // this warp's slice: lane l converts x[b][kb*128 + 4l .. 4l+3] to fp32, layout xs[i][b]
         __syncwarp();
@@ -686,8 +709,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
             float v[kV][4];
 #pragma unroll
             for (int b = 0; b < kV; ++b) {
-                const uint2 raw = *reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4);
-                const __half2 h0 = *reinterpret_cast<const __half2*>(&raw.x), h1 = *reinterpret_cast<const __half2*>(&raw.y);
+                const __half2 h0 = *reinterpret_cast<const __half2*>(&xraw[b].x), h1 = *reinterpret_cast<const __half2*>(&xraw[b].y);
                 v[b][0] = __low2float(h0); v[b][1] = __high2float(h0); v[b][2] = __low2float(h1); v[b][3] = __high2float(h1);
             }
             if constexpr (kV == 1) {
@@ -699,7 +721,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         }
         __syncwarp();
         const Block cur = blk;
-        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_x(u + 1); }
         fused_group<kV>(cur, smem_base, ws, T, xs, acc);
     }
     if (u0 < u1) flush(cur_tile);
@@ -765,6 +787,14 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
 // ---------------------------------------------------------------------------------------------
 // host-side launch helpers
 // ---------------------------------------------------------------------------------------------
+// number of working warps <= w_max such that `units` split evenly: all get ceil(units / w_max) or one less
+inline uint32_t balanced_warps(uint64_t units, uint32_t w_max)
+{
+    if (units <= w_max) return static_cast<uint32_t>(units);
+    const uint64_t per_warp = (units + w_max - 1) / w_max;
+    return static_cast<uint32_t>((units + per_warp - 1) / per_warp);
+}
+
 struct DeviceInfo {
     int device = -1, sms = 0, cc_major = 0;
     bool ok = false;
@@ -823,7 +853,7 @@ GemvPlan gemv_plan(int n_out, int kblocks, int vpad, int ctas_max)
     const int kFusedRows = fused_warps(vpad) * 32;
     p.row_tiles = (n_out + kFusedRows - 1) / kFusedRows;
     const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
-    p.grid = static_cast<int>(units < ctas_max ? units : ctas_max);
+    p.grid = static_cast<int>(balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(ctas_max)));   // same units per CTA
     p.partial_bytes = static_cast<size_t>(p.grid + p.row_tiles) * vpad * kFusedRows * sizeof(float);
     p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
     p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
@@ -923,8 +953,9 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
         }
         const uint64_t cta_tiles = (n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
         const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
+        const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kDecompressTmaWarps);
         kernel<<<grid, kDecompressTmaWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-            static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), map);
+            static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), active, map);
         return check_launch();
     }
     auto kernel = ecco_decompress_kernel<kDecompressWarps>;
@@ -937,7 +968,8 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     const uint64_t cta_tiles = (n_groups + kDecompressWarps * 32 - 1) / (kDecompressWarps * 32);   // one tile per warp
     const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
     kernel<<<grid, kDecompressWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out));
+        static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out),
+        balanced_warps((n_groups + 31) / 32, grid * kDecompressWarps));
     return check_launch();
 }
 
@@ -997,8 +1029,9 @@ static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
     cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
     if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kFusedWarps));
     kernel<<<p.grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
-                                                       static_cast<const __half*>(d_x), d_y, partial, tickets);
+                                                       static_cast<const __half*>(d_x), d_y, partial, tickets, active);
     return check_launch();
 }
 
@@ -1081,7 +1114,7 @@ static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* 
     }
     const int heads = batch * n_kv_heads;
     const int64_t units = static_cast<int64_t>(heads) * ((seq + kFusedRows - 1) / kFusedRows);
-    const unsigned grid = static_cast<unsigned>(units < di.sms ? units : di.sms);      // persistent CTAs
+    const unsigned grid = balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(di.sms));   // persistent CTAs, same units each
     kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, heads, seq, q_per_kv,
                                                      static_cast<const __half*>(d_q), scale, d_scores);
     return check_launch();
