@@ -42,10 +42,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5", "act2x"],
                     help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg4: 70B-shaped MLP weights + stream-size "
                          "sweep; cfg5: long-context GQA K cache [16][8][32768][128] (decompress + attention scores with 8 "
-                         "query heads per KV head)")
+                         "query heads per KV head); act2x: the 2x activation codec on a [32768][8192] fp16 tensor")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -432,9 +432,113 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_act2x(args):
+    """2x activation codec (Sec. 3.2): one step = compress + decompress of a [32768][8192] fp16 N(0,1) tensor."""
+    import torch
+
+    from paper_2505_06901_b200 import binding as B
+    from paper_2505_06901_b200 import distutil, synth
+
+    rank, world, local = distutil.rank_info()
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    rows, cols = 32768, 8192
+    x = synth.activations(rows, cols, 1006)
+    n = rows * cols // 64
+    d_x = torch.from_numpy(x).cuda()
+    d_blocks = torch.empty((n, 64), dtype=torch.uint8, device="cuda")
+    d_out = torch.empty_like(d_x)
+    stream = torch.cuda.current_stream()
+    warmup = max(args.warmup, 3)
+    for _ in range(warmup):
+        B.ecco_act_compress(d_x, n, d_blocks, stream)
+        B.ecco_act_decompress(d_blocks, n, d_out, stream)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    l0 = B.ecco_kernel_launch_count()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    for e in ev:
+        e[0].record(stream)
+        B.ecco_act_compress(d_x, n, d_blocks, stream)
+        e[1].record(stream)
+        B.ecco_act_decompress(d_blocks, n, d_out, stream)
+        e[2].record(stream)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches = B.ecco_kernel_launch_count() - l0
+    clocks = sampler.stop()
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    c_ms = sum(e[0].elapsed_time(e[1]) for e in ev)
+    d_ms = sum(e[1].elapsed_time(e[2]) for e in ev)
+    total_ms, c_ms, d_ms = distutil.max_over_ranks([total_ms, c_ms, d_ms], dist, "cuda")
+    # end to end: blocks from pinned host memory, fp16 back to pinned host memory
+    h_in, h_out = torch.empty((n, 64), dtype=torch.uint8).pin_memory(), torch.empty((rows, cols), dtype=torch.float16).pin_memory()
+    h_in.copy_(d_blocks)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    esteps = 5
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(esteps):
+        d_blocks.copy_(h_in, non_blocking=True)
+        B.ecco_act_decompress(d_blocks, n, d_out, stream)
+        h_out.copy_(d_out, non_blocking=True)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    (ems,) = distutil.max_over_ranks([e0.elapsed_time(e1)], dist, "cuda")
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peaks()
+    out_bytes = n * 128
+    dec_s = d_ms / 1e3 / args.steps
+    achieved = n * 192 / dec_s / 1e9
+    line = {
+        "metric": "act2x_decompress_output_GBps", "value": world * out_bytes / dec_s / 1e9, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "2x activation codec, fp16 N(0,1) [32768][8192] (4,194,304 groups of 64)",
+                   "step": "ecco_act_compress x1, ecco_act_decompress x1",
+                   "l2": "inputs larger than L2: 512 MiB of fp16, 256 MiB of blocks"},
+        "segments_us_per_step": {"act_compress": c_ms / args.steps * 1e3, "act_decompress": d_ms / args.steps * 1e3},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": world * out_bytes * esteps / (ems / 1e3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": n * 64,
+                "d2h_bytes_per_step": out_bytes, "steps": esteps},
+        "roofline": {"kernel": "ecco_act_decompress_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": n * 192, "avg_launch_us": dec_s * 1e6},
+        "kernels": [{"kernel": "ecco_act_compress", "us_per_step": c_ms / args.steps * 1e3,
+                     "hbm_GBps": n * 192 / (c_ms / 1e3 / args.steps) / 1e9, "hbm_frac": n * 192 / (c_ms / 1e3 / args.steps) / 1e9 / peak},
+                    {"kernel": "ecco_act_decompress", "us_per_step": dec_s * 1e6, "hbm_GBps": achieved, "hbm_frac": achieved / peak}],
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import ecco_oracle as eo
+
+        blocks = d_blocks[: 1 << 20].cpu().numpy()
+        t0 = time.perf_counter()
+        eo.act_decode(blocks)
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": blocks.shape[0] * 128 / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"first {blocks.shape[0]} groups, one pass on one thread"}
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 if __name__ == "__main__":
     a = parse_args()
     if a.impl == "reference":
         run_reference(a)
+    elif a.workload == "act2x":
+        run_act2x(a)
     else:
         run_ours(a)

@@ -159,6 +159,21 @@ int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, int32_t n_o
 int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
                      int32_t q_per_kv, const void* d_q_fp16, float scale, float* d_scores, void* stream);
 
+/* ---------------------------------------------------------------- 2x activation format (device) */
+
+/* Sec. 3.2 "Activation Compression", Sec. 4.2 / 4.3 low-ratio (de)compressor: 64 fp16 values <-> one
+ * 64-byte block.  Byte i holds the 7-bit two's-complement quantised value q_i (-64..63) in bits 0..6
+ * and one metadata bit in bit 7; metadata bits 0..15 are the fp16 scale, 16..31 the fp16 zero point
+ * (both least-significant bit first), 32..63 zero.  (The field widths are the paper's; the order
+ * is this library's definition.)  Compression: scale = fp16((max - min) / 127), zero point =
+ * fp16(min + 64 * scale), q = clamp(round_to_nearest_even((x - zero) * (1 / scale)), -64, 63) in fp32;
+ * a zero scale stores q = 0.  Decompression: fp16_rn(fma(q, scale, zero)) in fp32.  Inputs must be
+ * finite (non-finite values give unspecified bytes, never a fault).  Blocks 16-byte aligned, fp16
+ * buffers 32-byte aligned.  Both calls are asynchronous on `stream`. */
+#define ECCO_ACT_GROUP 64
+int ecco_act_compress(const void* d_x_fp16, uint64_t n_groups, uint8_t* d_blocks, void* stream);
+int ecco_act_decompress(const uint8_t* d_blocks, uint64_t n_groups, void* d_out_fp16, void* stream);
+
 /* ---------------------------------------------------------------- diagnostics */
 const char* ecco_error_string(int code);
 int ecco_last_cuda_error(void);        /* cudaError_t of the last ECCO_ERR_CUDA on this thread */

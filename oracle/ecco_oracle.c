@@ -898,3 +898,74 @@ int eo_set_exponent(eo_meta* M, const uint16_t* x16, uint64_t n_values) { return
 int eo_sizeof_meta(void) { return (int)sizeof(eo_meta); }
 int eo_sizeof_stats(void) { return (int)sizeof(eo_stats); }
 int eo_sizeof_info(void) { return (int)sizeof(eo_group_info); }
+
+/* ------------------------------------------------------------------------------------ */
+/* 2x activation format (Sec. 3.2 "Activation Compression", Sec. 4.2/4.3 low-ratio units): */
+/* 64 values -> 64 bytes; every byte holds a 7-bit quantised value, the eighth bit of the   */
+/* bytes carries a 16-bit scale factor and a 16-bit zero point, one bit per byte.           */
+/* reading (the paper gives the field widths only): byte i = q_i in its low 7 bits          */
+/* (two's complement, -64..63: the decompressor sign-extends 7 -> 8 bits) and metadata bit  */
+/* i in bit 7; metadata bits 0..15 = fp16 scale (lsb first), 16..31 = fp16 zero point,       */
+/* 32..63 = 0.  scale = fp16((max - min) / 127), zero = fp16(min + 64 * scale) (so q = -64   */
+/* is the group minimum), q = clamp(rint((x - zero) * (1 / scale)), -64, 63) in fp32 with    */
+/* the rounded scale and zero -- a multiply by the reciprocal, as in the compressor's        */
+/* "multiply-and-round circuit" (Sec. 4.3, low-ratio compressor); 1 / scale is one fp32      */
+/* division per group; a zero scale stores q = 0.  Dequantisation is one fp32 fused          */
+/* multiply-add rounded to fp16 (the "two operations" of the decompressor): q * scale + zero. */
+/* Parity unpinned: these choices are this build's definition.  Inputs must be finite.      */
+/* ------------------------------------------------------------------------------------ */
+#define EO_ACT_G 64
+
+int eo_act_encode_group(const uint16_t* x16, uint8_t* blk)
+{
+    float x[EO_ACT_G], lo = INFINITY, hi = -INFINITY;
+    for (int i = 0; i < EO_ACT_G; ++i) {
+        x[i] = eo_fp16_to_f32(x16[i]);
+        if (!isfinite(x[i])) return EO_ERR_NONFINITE;
+        if (x[i] < lo) lo = x[i];
+        if (x[i] > hi) hi = x[i];
+    }
+    uint16_t scale16 = eo_f32_to_fp16((hi - lo) / 127.0f);
+    float scale = eo_fp16_to_f32(scale16);
+    uint16_t zero16 = eo_f32_to_fp16(lo + 64.0f * scale);
+    float zero = eo_fp16_to_f32(zero16);
+    uint32_t meta_lo = (uint32_t)scale16 | ((uint32_t)zero16 << 16);
+    for (int i = 0; i < EO_ACT_G; ++i) {
+        int q = 0;
+        if (scale > 0.0f && isfinite(scale)) {
+            float inv = 1.0f / scale;
+            float r = rintf((x[i] - zero) * inv);
+            q = r < -64.0f ? -64 : r > 63.0f ? 63 : (int)r;
+        }
+        int mbit = (i < 32) ? (int)((meta_lo >> i) & 1u) : 0;
+        blk[i] = (uint8_t)(((unsigned)q & 0x7fu) | ((unsigned)mbit << 7));
+    }
+    return EO_OK;
+}
+
+void eo_act_decode_group(const uint8_t* blk, uint16_t* out16)
+{
+    uint32_t meta_lo = 0;
+    for (int i = 0; i < 32; ++i) meta_lo |= (uint32_t)(blk[i] >> 7) << i;
+    float scale = eo_fp16_to_f32((uint16_t)(meta_lo & 0xffffu));
+    float zero = eo_fp16_to_f32((uint16_t)(meta_lo >> 16));
+    for (int i = 0; i < EO_ACT_G; ++i) {
+        int q = blk[i] & 0x7f;
+        if (q & 0x40) q -= 128;                 /* sign extension of the 7-bit value */
+        out16[i] = eo_f32_to_fp16(fmaf((float)q, scale, zero));
+    }
+}
+
+int eo_act_encode(const uint16_t* x16, uint64_t n_groups, uint8_t* blocks)
+{
+    for (uint64_t g = 0; g < n_groups; ++g) {
+        int rc = eo_act_encode_group(x16 + g * EO_ACT_G, blocks + g * 64);
+        if (rc) return rc;
+    }
+    return EO_OK;
+}
+
+void eo_act_decode(const uint8_t* blocks, uint64_t n_groups, uint16_t* out16)
+{
+    for (uint64_t g = 0; g < n_groups; ++g) eo_act_decode_group(blocks + g * 64, out16 + g * EO_ACT_G);
+}

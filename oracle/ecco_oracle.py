@@ -334,3 +334,25 @@ def attn_scores(meta: Meta, kblocks, batch: int, n_kv_heads: int, seq: int, q_pe
     _check(lib().eo_attn_scores(C.byref(meta), _p(b, C.c_uint8), batch, n_kv_heads, seq, q_per_kv, _p(q, C.c_uint16),
                                 C.c_double(scale), _p(s, C.c_double), _p(sa, C.c_double)), "attn_scores")
     return s, sa
+
+
+# ---------------------------------------------------------------- 2x activation format
+ACT_G = 64
+
+
+def act_encode(x16) -> np.ndarray:
+    """fp16 [n_groups*64] -> uint8 [n_groups][64]."""
+    x = _u16(x16).reshape(-1)
+    assert x.size % ACT_G == 0
+    n = x.size // ACT_G
+    blocks = np.zeros((n, 64), dtype=np.uint8)
+    _check(lib().eo_act_encode(_p(x, C.c_uint16), C.c_uint64(n), _p(blocks, C.c_uint8)), "act_encode")
+    return blocks
+
+
+def act_decode(blocks) -> np.ndarray:
+    """uint8 [n_groups][64] -> fp16 [n_groups][64]."""
+    b = np.ascontiguousarray(blocks, dtype=np.uint8).reshape(-1, 64)
+    out = np.zeros((b.shape[0], ACT_G), dtype=np.uint16)
+    lib().eo_act_decode(_p(b, C.c_uint8), C.c_uint64(b.shape[0]), _p(out, C.c_uint16))
+    return out.view(np.float16)

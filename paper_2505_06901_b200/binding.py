@@ -33,7 +33,7 @@ ERR_DEVICE_TIMEOUT = -8
 EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
-    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
+    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
 
@@ -89,6 +89,8 @@ def lib():
         L.ecco_gemv.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, vp]
         L.ecco_gemv_static_ws.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
         L.ecco_attn_scores.argtypes = [vp, vp, i32, i32, i32, i32, vp, C.c_float, vp, vp]
+        L.ecco_act_compress.argtypes = [vp, u64, vp, vp]
+        L.ecco_act_decompress.argtypes = [vp, u64, vp, vp]
         L.ecco_error_string.argtypes = [C.c_int]
         L.ecco_error_string.restype = C.c_char_p
         L.ecco_last_cuda_error.restype = C.c_int
@@ -252,6 +254,15 @@ def ecco_attn_scores(d_meta, d_kblocks, batch: int, n_kv_heads: int, seq: int, q
                      d_scores, stream=None) -> None:
     _check(lib().ecco_attn_scores(_ptr(d_meta), _ptr(d_kblocks), batch, n_kv_heads, seq, q_per_kv, _ptr(d_q_fp16),
                                   C.c_float(scale), _ptr(d_scores), _stream(stream)), "ecco_attn_scores")
+
+
+def ecco_act_compress(d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:
+    """2x activation format: 64 fp16 values -> 64 bytes per group (device to device)."""
+    _check(lib().ecco_act_compress(_ptr(d_x_fp16), n_groups, _ptr(d_blocks), _stream(stream)), "ecco_act_compress")
+
+
+def ecco_act_decompress(d_blocks, n_groups: int, d_out_fp16, stream=None) -> None:
+    _check(lib().ecco_act_decompress(_ptr(d_blocks), n_groups, _ptr(d_out_fp16), _stream(stream)), "ecco_act_decompress")
 
 
 def ecco_device_status() -> int:

@@ -349,3 +349,34 @@ def test_config5_long_context_gqa_full_size(B, eo, W, synth):
     assert t.n_groups == 16 * 8 * 32768
     check_full_decompress(B, eo, t)
     check_full_attn(B, eo, synth, t, 8)
+
+
+# ------------------------------------------------------------------ 2x activation codec
+@pytest.mark.parametrize("n_groups", [0, 1, 7, 8, 9, 1000, 4097, 1 << 16])
+def test_act2x_compress_and_decompress_match_oracle(B, eo, synth, n_groups):
+    x = synth.activations(max(n_groups, 1), 64, 300 + n_groups % 97)[:n_groups]
+    if n_groups > 8:
+        x[3] = np.float16(-0.75)                     # constant group: zero scale
+        x[5] = (x[5].astype(np.float32) * 1000).astype(np.float16)
+        x[6] = (x[6].astype(np.float32) * 1e-4).astype(np.float16)   # subnormal-sized steps
+    d_x = torch.from_numpy(np.ascontiguousarray(x)).cuda() if n_groups else torch.empty(64, dtype=torch.float16, device="cuda")
+    d_blocks = torch.full((max(n_groups, 1), 64), 0xEE, dtype=torch.uint8, device="cuda")
+    B.ecco_act_compress(d_x, n_groups, d_blocks)
+    d_out = torch.empty((max(n_groups, 1), 64), dtype=torch.float16, device="cuda")
+    B.ecco_act_decompress(d_blocks, n_groups, d_out)
+    torch.cuda.synchronize()
+    if n_groups == 0:
+        return
+    want_blocks = eo.act_encode(x)
+    got_blocks = d_blocks.cpu().numpy()
+    bad = np.nonzero((got_blocks != want_blocks).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} blocks differ, first {bad[:4]}"
+    assert np.array_equal(d_out.cpu().numpy().view(np.uint16), eo.act_decode(want_blocks).view(np.uint16))
+    # decompression is total: random bytes decode like the oracle says
+    rb = synth.random_blocks(n_groups, 17)
+    d_rb = torch.from_numpy(rb).cuda()
+    B.ecco_act_decompress(d_rb, n_groups, d_out)
+    torch.cuda.synchronize()
+    got, want = d_out.cpu().numpy().view(np.uint16), eo.act_decode(rb).view(np.uint16)
+    finite = np.isfinite(eo.act_decode(rb).astype(np.float32))       # NaN payloads may differ, everything else may not
+    assert np.array_equal(got[finite], want[finite])
