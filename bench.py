@@ -194,17 +194,17 @@ def cpu_baseline(layer, c: int):
 # ------------------------------------------------------------------------------------------------
 WORKLOADS = {
     "cfg2": dict(label="cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
-                       "+ cfg3 K cache [8][32][4096][128]",
-                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1",
+                       "+ cfg3 K and V caches [8][32][4096][128]",
+                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache)",
                  l2="inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
     "cfg4": dict(label="cfg4 llama-70b-shaped MLP weights (gate, up 28672x8192; down 8192x28672; 5,505,024 groups)",
                  step="decompress x3, gemv batch 1 x3; plus a decompress sweep over 64 MiB .. 4 GiB streams (stream_sweep)",
                  l2="inputs larger than L2: each step streams 336 MiB of blocks and writes 1.3 GiB"),
-    "cfg5": dict(label="cfg5 long-context GQA K cache [16][8][32768][128] (4,194,304 groups)",
-                 step="decompress x1, attn_scores x1 (8 query heads per KV head)",
+    "cfg5": dict(label="cfg5 long-context GQA K and V caches [16][8][32768][128] (4,194,304 groups each)",
+                 step="decompress x1 (K), attn_scores x1 and attn_values x1 (8 query heads per KV head)",
                  l2="inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB"),
     "small": dict(label="reduced (profiling): q + gate of cfg2, K cache [2][32][4096][128]",
-                  step="decompress x2, gemv batch 1 x2, gemv batch 8 x2, attn_scores x1",
+                  step="decompress x2, gemv batch 1 x2, gemv batch 8 x2, attn_scores x1, attn_values x1",
                   l2="inputs larger than L2 except the q projection"),
 }
 
@@ -212,15 +212,17 @@ WORKLOADS = {
 def build_workload(name, workloads):
     """-> (weight tensors, kv tensor or None, q_per_kv, decompress_kv, default segments)."""
     if name == "cfg5":
-        (kt,) = workloads.config5(which=("K",))
-        return [], kt, 8, True, ["decompress", "attn"]
+        kt, vt = workloads.config5(which=("K", "V"))
+        return [], (kt, vt), 8, True, ["decompress", "attn", "attnv"]
     if name == "cfg4":
         return workloads.config4(), None, 1, False, ["decompress", "gemv1"]
     if name == "small":
-        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, workloads.calibrate_kv(3, 32))
-        return workloads.config2(names=("q", "gate")), kt, 1, False, ["decompress", "gemv1", "gemv8", "attn"]
-    (kt,) = workloads.config3(which=("K",))
-    return workloads.config2(), kt, 1, False, ["decompress", "gemv1", "gemv8", "attn"]
+        base = workloads.calibrate_kv(3, 32)
+        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, base)
+        vt = workloads.kv_tensor("V", 2, 32, 4096, 1003 * 16 + 1, 3003, base)
+        return workloads.config2(names=("q", "gate")), (kt, vt), 1, False, ["decompress", "gemv1", "gemv8", "attn", "attnv"]
+    kt, vt = workloads.config3(which=("K", "V"))
+    return workloads.config2(), (kt, vt), 1, False, ["decompress", "gemv1", "gemv8", "attn", "attnv"]
 
 
 def run_ours(args):
@@ -242,7 +244,8 @@ def run_ours(args):
 
     # ---- workload (the same seeded tensors on every rank)
     wname = "small" if args.small else args.workload
-    weights, kt, q_per_kv, decompress_kv, default_segs = build_workload(wname, workloads)
+    weights, kvt, q_per_kv, decompress_kv, default_segs = build_workload(wname, workloads)
+    kt, vt = kvt if kvt is not None else (None, None)
     segs = [s for s in args.only.split(",") if s] or default_segs
     stream = torch.cuda.current_stream()
     need8 = "gemv8" in segs
@@ -263,6 +266,10 @@ def run_ours(args):
         kv = dict(t=kt, n=kt.n_groups, meta=B.meta_to_device(kt.meta), blocks=torch.from_numpy(kt.blocks).cuda(),
                   q=torch.from_numpy(synth.queries(kb, kh * q_per_kv, 13)).cuda(),
                   scores=torch.empty((kb, kh * q_per_kv, kseq), dtype=torch.float32, device="cuda"))
+        avb = B.ecco_attn_values_workspace_bytes(kb, kh, kseq, q_per_kv)
+        kv.update(v_meta=B.meta_to_device(vt.meta), v_blocks=torch.from_numpy(vt.blocks).cuda(),
+                  attn_out=torch.empty((kb, kh * q_per_kv, G), dtype=torch.float32, device="cuda"),
+                  av_ws=torch.empty(avb, dtype=torch.uint8, device="cuda"), av_wsb=avb)
         if decompress_kv:
             kv["out"] = torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")
             dec.append(kv)
@@ -280,6 +287,11 @@ def run_ours(args):
         if kv is not None:
             B.ecco_attn_scores(kv["meta"], kv["blocks"], kb, kh, kseq, q_per_kv, kv["q"], 128 ** -0.5, kv["scores"], stream)
 
+    def seg_attnv():
+        if kv is not None:
+            B.ecco_attn_values(kv["v_meta"], kv["v_blocks"], kb, kh, kseq, q_per_kv, kv["scores"], kv["attn_out"], kv["av_ws"],
+                               kv["av_wsb"], stream)
+
     def step(ev=None):
         if ev: ev[0].record(stream)
         if "decompress" in segs: seg_decompress()
@@ -290,6 +302,8 @@ def run_ours(args):
         if ev: ev[3].record(stream)
         if "attn" in segs: seg_attn()
         if ev: ev[4].record(stream)
+        if "attnv" in segs: seg_attnv()
+        if ev: ev[5].record(stream)
 
     def barrier():
         if dist is not None:
@@ -299,7 +313,7 @@ def run_ours(args):
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
         step()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
@@ -312,9 +326,9 @@ def run_ours(args):
     clocks = sampler.stop()
     assert B.ecco_device_status() == 0, "a kernel reported a device-side timeout"
 
-    total_ms = events[0][0].elapsed_time(events[-1][4])
-    seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(4)]
-    total_ms, dec_ms, g1_ms, g8_ms, at_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
+    total_ms = events[0][0].elapsed_time(events[-1][5])
+    seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(5)]
+    total_ms, dec_ms, g1_ms, g8_ms, at_ms, av_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
 
     groups = sum(d["n"] for d in dec)
     out_bytes = groups * G * 2
@@ -388,7 +402,7 @@ def run_ours(args):
             traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
     # the fused kernels against the same HBM peak (algorithmic bytes: blocks + vectors + results); what bounds them
     # is the SM load/store pipe, so the symbol rate is reported next to the HBM fraction
-    seg_total = dec_ms + g1_ms + g8_ms + at_ms
+    seg_total = dec_ms + g1_ms + g8_ms + at_ms + av_ms
     kernels = []
 
     def kernel_entry(name, ms, alg_bytes_per_step, symbols_per_step):
@@ -406,6 +420,7 @@ def run_ours(args):
     kernel_entry("ecco_gemv batch 8", g8_ms if "gemv8" in segs else 0, w_groups * BLOCK + gemv_vec(8), w_groups * G)
     if kv is not None:
         kernel_entry(f"ecco_attn_scores q_per_kv {q_per_kv}", at_ms if "attn" in segs else 0, kv["n"] * (BLOCK + 4 * q_per_kv), kv["n"] * G)
+        kernel_entry(f"ecco_attn_values q_per_kv {q_per_kv}", av_ms if "attnv" in segs else 0, kv["n"] * (BLOCK + 4 * q_per_kv), kv["n"] * G)
     info = WORKLOADS[wname]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -414,7 +429,8 @@ def run_ours(args):
         "config": {"workload": info["label"], "step": info["step"], "segments": segs, "l2": info["l2"],
                    "format": "S=64, H=4, group 128, 64-byte blocks"},
         "segments_us_per_step": {"decompress": dec_ms / args.steps * 1e3, "gemv_batch1": g1_ms / args.steps * 1e3,
-                                 "gemv_batch8": g8_ms / args.steps * 1e3, "attn_scores": at_ms / args.steps * 1e3},
+                                 "gemv_batch8": g8_ms / args.steps * 1e3, "attn_scores": at_ms / args.steps * 1e3,
+                                 "attn_values": av_ms / args.steps * 1e3},
         "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3 if wname == "cfg2" else None,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",

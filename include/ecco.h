@@ -159,6 +159,20 @@ int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, int32_t n_o
 int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
                      int32_t q_per_kv, const void* d_q_fp16, float scale, float* d_scores, void* stream);
 
+/* Attention output over a compressed V cache (Eq. 3: softmax(Q K^T / sqrt(d_k)) V):
+ * out[b][hq][d] = sum_t p[b][hq][t] * V~[b][hq / q_per_kv][t][d] with p = softmax over t of
+ * scores[b][hq][:] (fp32 logits, e.g. the output of ecco_attn_scores).  Blocks are ordered
+ * [batch][n_kv_heads][seq], one group = one token's 128-wide head vector; out is fp32
+ * [batch][n_kv_heads*q_per_kv][128]; q_per_kv in 1..8; seq >= 1.  The sum over tokens runs on the
+ * tensor cores with fp32 accumulation; outlier corrections are added in an order that may vary from
+ * run to run (last-bit differences).  d_workspace: at least ecco_attn_values_workspace_bytes(...)
+ * bytes, 16-byte aligned, contents irrelevant before and undefined after; calls sharing a workspace
+ * must not overlap. */
+size_t ecco_attn_values_workspace_bytes(int32_t batch, int32_t n_kv_heads, int32_t seq, int32_t q_per_kv);
+int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
+                     int32_t q_per_kv, const float* d_scores, float* d_out, void* d_workspace, size_t workspace_bytes,
+                     void* stream);
+
 /* ---------------------------------------------------------------- 2x activation format (device) */
 
 /* Sec. 3.2 "Activation Compression", Sec. 4.2 / 4.3 low-ratio (de)compressor: 64 fp16 values <-> one

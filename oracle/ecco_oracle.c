@@ -969,3 +969,49 @@ void eo_act_decode(const uint8_t* blocks, uint64_t n_groups, uint16_t* out16)
 {
     for (uint64_t g = 0; g < n_groups; ++g) eo_act_decode_group(blocks + g * 64, out16 + g * EO_ACT_G);
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Attention output over a compressed V cache (Eq. 3: softmax(QK^T / sqrt(d_k)) V):       */
+/* out[b][hq][d] = sum_t softmax_t(scores[b][hq][:])[t] * V~[b][hq / q_per_kv][t][d], in   */
+/* fp64 over the decompressed fp16 values.  scores are the fp32 logits (already scaled).   */
+/* outabs receives sum_t p_t |V~| for the error metric.                                    */
+/* ------------------------------------------------------------------------------------ */
+int eo_attn_values(const eo_meta* M, const uint8_t* vblocks, int batch, int n_kv_heads, int seq, int q_per_kv,
+                   const float* scores, double* out, double* outabs)
+{
+    int rc = eo_meta_check(M);
+    if (rc) return rc;
+    int n_q = n_kv_heads * q_per_kv;
+    uint16_t v16[EO_G];
+    double* p = (double*)malloc(sizeof(double) * (size_t)seq * (size_t)q_per_kv);
+    for (int b = 0; b < batch; ++b)
+        for (int h = 0; h < n_kv_heads; ++h) {
+            for (int r = 0; r < q_per_kv; ++r) {
+                const float* s = scores + ((size_t)b * n_q + h * q_per_kv + r) * (size_t)seq;
+                double mx = -INFINITY, sum = 0.0;
+                for (int t = 0; t < seq; ++t) if (s[t] > mx) mx = s[t];
+                for (int t = 0; t < seq; ++t) { p[(size_t)r * seq + t] = exp((double)s[t] - mx); sum += p[(size_t)r * seq + t]; }
+                for (int t = 0; t < seq; ++t) p[(size_t)r * seq + t] /= sum;
+                double* o = out + ((size_t)b * n_q + h * q_per_kv + r) * EO_G;
+                double* oa = outabs ? outabs + ((size_t)b * n_q + h * q_per_kv + r) * EO_G : NULL;
+                for (int d = 0; d < EO_G; ++d) { o[d] = 0.0; if (oa) oa[d] = 0.0; }
+            }
+            for (int t = 0; t < seq; ++t) {
+                size_t g = ((size_t)b * n_kv_heads + h) * (size_t)seq + t;
+                rc = eo_decode_block(M, vblocks + g * EO_BLOCK, v16, NULL, NULL);
+                if (rc) { free(p); return rc; }
+                for (int r = 0; r < q_per_kv; ++r) {
+                    double* o = out + ((size_t)b * n_q + h * q_per_kv + r) * EO_G;
+                    double* oa = outabs ? outabs + ((size_t)b * n_q + h * q_per_kv + r) * EO_G : NULL;
+                    double pt = p[(size_t)r * seq + t];
+                    for (int d = 0; d < EO_G; ++d) {
+                        double v = (double)eo_fp16_to_f32(v16[d]);
+                        o[d] += pt * v;
+                        if (oa) oa[d] += pt * fabs(v);
+                    }
+                }
+            }
+        }
+    free(p);
+    return EO_OK;
+}

@@ -356,3 +356,17 @@ def act_decode(blocks) -> np.ndarray:
     out = np.zeros((b.shape[0], ACT_G), dtype=np.uint16)
     lib().eo_act_decode(_p(b, C.c_uint8), C.c_uint64(b.shape[0]), _p(out, C.c_uint16))
     return out.view(np.float16)
+
+
+def attn_values(meta: Meta, vblocks, batch: int, n_kv_heads: int, seq: int, q_per_kv: int, scores):
+    """softmax(scores) . V~ -> (out fp64 [batch][n_kv_heads*q_per_kv][128], sum_t p_t |V~| of the same shape)."""
+    b = np.ascontiguousarray(vblocks, dtype=np.uint8).reshape(-1)
+    assert b.size == batch * n_kv_heads * seq * BLOCK
+    s = np.ascontiguousarray(scores, dtype=np.float32)
+    nq = n_kv_heads * q_per_kv
+    assert s.shape == (batch, nq, seq)
+    out = np.zeros((batch, nq, G), dtype=np.float64)
+    oa = np.zeros((batch, nq, G), dtype=np.float64)
+    _check(lib().eo_attn_values(C.byref(meta), _p(b, C.c_uint8), batch, n_kv_heads, seq, q_per_kv, _p(s, C.c_float),
+                                _p(out, C.c_double), _p(oa, C.c_double)), "attn_values")
+    return out, oa

@@ -33,7 +33,8 @@ ERR_DEVICE_TIMEOUT = -8
 EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
-    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
+    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
+    "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
 
@@ -89,6 +90,9 @@ def lib():
         L.ecco_gemv.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, vp]
         L.ecco_gemv_static_ws.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
         L.ecco_attn_scores.argtypes = [vp, vp, i32, i32, i32, i32, vp, C.c_float, vp, vp]
+        L.ecco_attn_values_workspace_bytes.argtypes = [i32, i32, i32, i32]
+        L.ecco_attn_values_workspace_bytes.restype = sz
+        L.ecco_attn_values.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.ecco_act_compress.argtypes = [vp, u64, vp, vp]
         L.ecco_act_decompress.argtypes = [vp, u64, vp, vp]
         L.ecco_error_string.argtypes = [C.c_int]
@@ -254,6 +258,18 @@ def ecco_attn_scores(d_meta, d_kblocks, batch: int, n_kv_heads: int, seq: int, q
                      d_scores, stream=None) -> None:
     _check(lib().ecco_attn_scores(_ptr(d_meta), _ptr(d_kblocks), batch, n_kv_heads, seq, q_per_kv, _ptr(d_q_fp16),
                                   C.c_float(scale), _ptr(d_scores), _stream(stream)), "ecco_attn_scores")
+
+
+def ecco_attn_values_workspace_bytes(batch: int, n_kv_heads: int, seq: int, q_per_kv: int) -> int:
+    return int(lib().ecco_attn_values_workspace_bytes(batch, n_kv_heads, seq, q_per_kv))
+
+
+def ecco_attn_values(d_meta, d_vblocks, batch: int, n_kv_heads: int, seq: int, q_per_kv: int, d_scores, d_out, d_workspace,
+                     workspace_bytes: int, stream=None) -> None:
+    """softmax(scores) . V~ over a compressed V cache -> fp32 [batch][n_kv_heads*q_per_kv][128]."""
+    _check(lib().ecco_attn_values(_ptr(d_meta), _ptr(d_vblocks), batch, n_kv_heads, seq, q_per_kv, _ptr(d_scores), _ptr(d_out),
+                                  _ptr(d_workspace) if d_workspace is not None else None, workspace_bytes, _stream(stream)),
+           "ecco_attn_values")
 
 
 def ecco_act_compress(d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:

@@ -330,11 +330,27 @@ def check_full_attn(B, eo, synth, t, qpk):
     assert np.isfinite(s).all()
 
 
+def check_full_attn_values(B, eo, t, qpk, n_heads_checked=3):
+    batch, heads, seq, _ = t.shape
+    om = oracle_meta_from_lib(eo, t.meta)
+    rng = np.random.Generator(np.random.PCG64(seq * 3 + qpk))
+    scores = (rng.standard_normal((batch, heads * qpk, seq)) * 2.0).astype(np.float32)
+    got = gpu_attn_values(B, t.meta, t.blocks, batch, heads, seq, qpk, scores)
+    assert np.isfinite(got).all()
+    for _ in range(n_heads_checked):
+        b, h = int(rng.integers(batch)), int(rng.integers(heads))
+        g0 = (b * heads + h) * seq
+        ref, refabs = eo.attn_values(om, t.blocks[g0:g0 + seq], 1, 1, seq, qpk, scores[b:b + 1, h * qpk:(h + 1) * qpk])
+        check_fused(got[b, h * qpk:(h + 1) * qpk], ref[0], refabs[0])
+
+
 def test_config3_kv_cache_full_size(B, eo, W, synth):
-    (t,) = W.config3(which=("K",))
-    assert t.n_groups == 8 * 32 * 4096
-    check_full_decompress(B, eo, t)
-    check_full_attn(B, eo, synth, t, 1)
+    k, v = W.config3(which=("K", "V"))
+    assert k.n_groups == 8 * 32 * 4096
+    check_full_decompress(B, eo, k)
+    check_full_attn(B, eo, synth, k, 1)
+    check_full_decompress(B, eo, v)
+    check_full_attn_values(B, eo, v, 1)
 
 
 def test_config4_llama70b_mlp_full_size(B, eo, W, synth):
@@ -345,10 +361,11 @@ def test_config4_llama70b_mlp_full_size(B, eo, W, synth):
 
 
 def test_config5_long_context_gqa_full_size(B, eo, W, synth):
-    (t,) = W.config5(which=("K",))
-    assert t.n_groups == 16 * 8 * 32768
-    check_full_decompress(B, eo, t)
-    check_full_attn(B, eo, synth, t, 8)
+    k, v = W.config5(which=("K", "V"))
+    assert k.n_groups == 16 * 8 * 32768
+    check_full_decompress(B, eo, k)
+    check_full_attn(B, eo, synth, k, 8)
+    check_full_attn_values(B, eo, v, 8, n_heads_checked=2)
 
 
 # ------------------------------------------------------------------ 2x activation codec
@@ -380,3 +397,41 @@ def test_act2x_compress_and_decompress_match_oracle(B, eo, synth, n_groups):
     got, want = d_out.cpu().numpy().view(np.uint16), eo.act_decode(rb).view(np.uint16)
     finite = np.isfinite(eo.act_decode(rb).astype(np.float32))       # NaN payloads may differ, everything else may not
     assert np.array_equal(got[finite], want[finite])
+
+
+# ------------------------------------------------------------------ fused attention output (softmax . V)
+def gpu_attn_values(B, lmeta, blocks, batch, heads, seq, qpk, scores):
+    d_meta, d_blocks, d_s = B.meta_to_device(lmeta), dev(blocks), dev(scores)
+    d_o = torch.full((batch, heads * qpk, 128), float("nan"), dtype=torch.float32, device="cuda")
+    wsb = B.ecco_attn_values_workspace_bytes(batch, heads, seq, qpk)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    ws.fill_(0xCD)
+    B.ecco_attn_values(d_meta, d_blocks, batch, heads, seq, qpk, d_s, d_o, ws, wsb)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    return d_o.cpu().numpy().astype(np.float64)
+
+
+@pytest.mark.parametrize("batch,heads,seq,qpk", [(2, 4, 256, 1), (2, 4, 256, 8), (1, 3, 77, 4), (1, 1, 1, 1), (2, 2, 1300, 3),
+                                                 (1, 2, 5000, 2)])
+def test_attn_values_match_oracle(B, eo, kv_small, synth, batch, heads, seq, qpk):
+    meta = kv_small["meta"]
+    n = batch * heads * seq
+    blocks = np.tile(kv_small["blocks"], (-(-n // 2048), 1))[:n]
+    rng = np.random.Generator(np.random.PCG64(seq * 7 + qpk))
+    scores = (rng.standard_normal((batch, heads * qpk, seq)) * 2.5).astype(np.float32)
+    got = gpu_attn_values(B, lib_meta_from_oracle(B, meta), blocks, batch, heads, seq, qpk, scores)
+    ref, refabs = eo.attn_values(meta, blocks, batch, heads, seq, qpk, scores)
+    check_fused(got, ref, refabs)
+
+
+def test_attn_values_on_garbage_blocks_and_peaked_softmax(B, eo, kv_small, synth):
+    meta = kv_small["meta"]
+    rb = synth.random_blocks(2 * 2 * 700, 321)             # duplicate pad locations, clips, 16-pad groups
+    rng = np.random.Generator(np.random.PCG64(5))
+    scores = (rng.standard_normal((2, 4, 700)) * 2).astype(np.float32)
+    scores[0, 1, :] = -50.0
+    scores[0, 1, 333] = 10.0                               # one-hot softmax
+    got = gpu_attn_values(B, lib_meta_from_oracle(B, meta), rb, 2, 2, 700, 2, scores)
+    ref, refabs = eo.attn_values(meta, rb, 2, 2, 700, 2, scores)
+    check_fused(got, ref, refabs)

@@ -291,3 +291,22 @@ def test_compression_quality_on_the_synthetic_distributions(eo, cfg1_small, kv_s
     # threaded driver gives the same bytes as the single-threaded loop
     a = eo.decode_threads(kv_small["meta"], kv_small["blocks"], 3)
     assert np.array_equal(a.view(np.uint16), eo.decode(kv_small["meta"], kv_small["blocks"]).view(np.uint16))
+
+
+def test_attention_output_reduces_to_textbook_softmax_times_v(eo, kv_small, synth):
+    km, kb = kv_small["meta"], kv_small["blocks"]
+    V = eo.decode(km, kb).reshape(2, 4, 256, 128).astype(np.float64)
+    rng = np.random.Generator(np.random.PCG64(31))
+    scores = (rng.standard_normal((2, 8, 256)) * 3).astype(np.float32)
+    out, oa = eo.attn_values(km, kb, 2, 4, 256, 2, scores)
+    s = scores.astype(np.float64)
+    p = np.exp(s - s.max(-1, keepdims=True))
+    p /= p.sum(-1, keepdims=True)
+    ref = np.einsum("bhrt,bhtd->bhrd", p.reshape(2, 4, 2, 256), V).reshape(2, 8, 128)
+    assert np.allclose(out, ref, rtol=1e-12, atol=1e-14)
+    assert np.all(oa >= np.abs(out) - 1e-12)
+    # a one-hot softmax (one logit far above the rest) returns that token's decompressed vector
+    scores[:] = -1e4
+    scores[:, :, 17] = 0.0
+    out, _ = eo.attn_values(km, kb, 2, 4, 256, 2, scores)
+    assert np.allclose(out.reshape(2, 4, 2, 128), V[:, :, 17][:, :, None, :], rtol=1e-12)
