@@ -164,8 +164,8 @@ int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch
  * scores[b][hq][:] (fp32 logits, e.g. the output of ecco_attn_scores).  Blocks are ordered
  * [batch][n_kv_heads][seq], one group = one token's 128-wide head vector; out is fp32
  * [batch][n_kv_heads*q_per_kv][128]; q_per_kv in 1..8; seq >= 1.  The sum over tokens runs on the
- * tensor cores with fp32 accumulation; outlier corrections are added in an order that may vary from
- * run to run (last-bit differences).  d_workspace: at least ecco_attn_values_workspace_bytes(...)
+ * tensor cores with fp32 accumulation, in an order fixed by the shapes (results are reproducible).
+ * d_workspace: at least ecco_attn_values_workspace_bytes(...)
  * bytes, 16-byte aligned, contents irrelevant before and undefined after; calls sharing a workspace
  * must not overlap. */
 size_t ecco_attn_values_workspace_bytes(int32_t batch, int32_t n_kv_heads, int32_t seq, int32_t q_per_kv);

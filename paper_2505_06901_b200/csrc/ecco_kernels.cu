@@ -205,11 +205,11 @@ __device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t sme
 }
 
 // Decodes the 128 indices of the lane's group (Sec. 4.2, Huffman decode) and hands each value to
-// sink(n, value_bits, symbol).  A codeword that would cross bit 512 ends the group: that and all
+// sink(n, value_bits, symbol, alive) (kLookup = false skips the value lookup and passes 0).  A codeword that would cross bit 512 ends the group: that and all
 // later positions are delivered as zero (clipped).  Returns the end bit if all 128 fitted, else 0.
 // Must be called by all 32 lanes of the warp.  Four symbols are decoded per window refill; the
 // per-symbol clip test runs only in steps where some lane of the warp reaches bit 512.
-template <class Sink>
+template <bool kLookup = true, class Sink>
 __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const WarpSmem& ws, Sink&& sink)
 {
     uint32_t pos = h.pos;
@@ -231,12 +231,13 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 alive = alive && (end[j] <= limit);
-                const uint32_t v = lds_u32(ws.tab + (e[j] & 15u) * 128);
-                sink(step * 4 + j, alive ? v : 0u, e[j] & 15u);
+                const uint32_t v = kLookup ? lds_u32(ws.tab + (e[j] & 15u) * 128) : 0u;
+                sink(step * 4 + j, alive ? v : 0u, e[j] & 15u, alive);
             }
         } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) sink(step * 4 + j, lds_u32(ws.tab + (e[j] & 15u) * 128), e[j] & 15u);
+            for (int j = 0; j < 4; ++j)
+                sink(step * 4 + j, kLookup ? lds_u32(ws.tab + (e[j] & 15u) * 128) : 0u, e[j] & 15u, true);
         }
         pos += acc;
     }
@@ -295,7 +296,7 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
             ldg_block(blk, d_blocks + min(tn * 32 + lane, n_groups - 1) * kBlockBytes);
         uint16_t* out = d_out + min(g, n_groups - 1) * kGroup;
         uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t) {
+        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
             const int slot = (n & 15) >> 1;
             if (n & 1) r[slot] |= v << 16; else r[slot] = v;
             if ((n & 15) == 15 && store) stg_v8(out + (n - 15), r);
@@ -367,7 +368,7 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
             __syncwarp();
             if (lane == 0) { tma_store_2d(&out_map, stage, chunk * 16, row0); bulk_commit(); }
         };
-        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t) {
+        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
             const int slot = (n & 15) >> 1;
             if (n & 1) r[slot] |= v << 16; else r[slot] = v;
             if ((n & 15) == 15 && n != 127) { stage_rows(); send_tile(n >> 4); }
@@ -457,7 +458,7 @@ __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base
 {
     const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
     uint32_t packed = 0;
-    const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym) {
+    const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
         acc.fma(n, __uint_as_float(v), xs);
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
@@ -788,13 +789,14 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
 // K5: attention output over a compressed V cache (Eq. 3: softmax(QK^T / sqrt(d_k)) V).
 // out[b][hq][d] = sum_t p[b][hq][t] * V~[b][hq / q_per_kv][t][d] with p = softmax_t(scores).
 // A thread owns one token (one group) as in K3, but here the sum runs over tokens, i.e. across
-// lanes.  Every 16 decoded values per lane go to a [32 tokens][16 dims] fp16 tile in shared memory
-// (same swizzle as the decompress staging tile) and the tile is contracted on the tensor cores:
-// (V tile)^T [16 dims x 32 tokens] x P^T [32 tokens x 8 heads] with mma.m16n8k16, fp32
-// accumulators (4 registers per 16 dims, 32 for the 128 dims).  p is split into an fp16 head and
-// an fp16 remainder (two MMAs) so that its rounding does not show in the result.  Outliers: those
-// of the last 16 dims are patched in the tile; the earlier ones are added as corrections
-// (outlier - mapped) * p through shared-memory float adds.
+// lanes.  Pass 1 runs the serial Huffman chain and keeps only the 4-bit indices (syms[16][32]);
+// by then the end bit, hence the outliers, are known.  Pass 2 walks the eight 16-dim chunks: map
+// the indices through the lane's table, stage them in a [32 tokens][16 dims] fp16 tile (same
+// swizzle as the decompress staging tile), overwrite the outliers of that chunk in the tile, and
+// contract the tile on the tensor cores: (V tile)^T [16 dims x 32 tokens] x P^T [32 tokens x 8
+// heads] with mma.m16n8k16, fp32 accumulators (4 registers per 16 dims, 32 for the 128 dims).  p is
+// split into an fp16 head and an fp16 remainder (two MMAs) so that its rounding does not show.
+// The result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 ecco_softmax_stats_kernel(const float* __restrict__ d_scores, int rows, int seq, float2* __restrict__ d_stats)
@@ -852,8 +854,6 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
     float* out_s = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kAvWarpBytes);    // [128 dims][8 heads]
-    float* corr_s = out_s + kGroup * 8;                                                       // outlier corrections
-    const uint32_t corr_addr = smem_u32(corr_s);
 
     const int G = gridDim.x, c = blockIdx.x;
     const int chunks = (seq + kTokens - 1) / kTokens;
@@ -877,7 +877,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     };
     clear_acc();
 
-    // all tokens of head bh seen by this CTA are in acc / corr_s: reduce over the warps in warp order, then
+    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in warp order, then
     // either store (this CTA owns the whole head) or hand a partial to the slot-and-ticket reduction
     auto flush = [&](int bh) {
         for (int i = tid; i < kGroup * 8; i += kTokens) out_s[i] = 0.0f;
@@ -895,8 +895,6 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             }
             __syncthreads();
         }
-        for (int i = tid; i < kGroup * 8; i += kTokens) out_s[i] += corr_s[i];
-        __syncthreads();
         const int c_lo = unit_owner(U, G, static_cast<int64_t>(bh) * chunks);
         const int c_hi = unit_owner(U, G, static_cast<int64_t>(bh + 1) * chunks - 1);
         if (c_lo == c_hi) {
@@ -933,7 +931,6 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int t = tile_base + static_cast<int>(lane);
         if (bh != cur_bh) {
             if (cur_bh >= 0) { flush(cur_bh); clear_acc(); }
-            for (int i = tid; i < kGroup * 8; i += kTokens) corr_s[i] = 0.0f;
             if (tid < 8) stats_s[tid] = tid < q_per_kv ? d_stats[static_cast<size_t>(bh) * q_per_kv + tid] : make_float2(0.0f, 0.0f);
             __syncthreads();
             cur_bh = bh;
@@ -948,8 +945,8 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             for (int j = 0; j < 4; ++j) {
                 const int tk = tile_base + static_cast<int>(lane & 3u) * 2 + 8 * j;
                 float p0 = 0.0f, p1 = 0.0f;
-                if (r < q_per_kv && tk < seq) p0 = expf(srow[tk] - st.x) * st.y;
-                if (r < q_per_kv && tk + 1 < seq) p1 = expf(srow[tk + 1] - st.x) * st.y;
+                if (r < q_per_kv && tk < seq) p0 = __expf(srow[tk] - st.x) * st.y;
+                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(srow[tk + 1] - st.x) * st.y;
                 const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
                 const __half l0 = __float2half_rn(p0 - __half2float(h0)), l1 = __float2half_rn(p1 - __half2float(h1));
                 p_hi[j] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);
@@ -960,14 +957,47 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         const bool valid = t < seq;                        // lanes past the end stage zeros (their p is zero too)
         const GroupHeader h = open_group<false>(cur, smem_base, ws, T);
-        uint32_t r8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
         uint32_t packed = 0;
-        auto stage_rows = [&]() {
+        int n_fit = kGroup;
+        const uint32_t end = decode_symbols<false>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+            if (!alive) n_fit = min(n_fit, n);             // only the clip path can see alive == false
+            packed |= sym << ((n & 7) * 4);
+            if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+        });
+        if (!valid) n_fit = 0;
+        // outliers of a complete group: which 16-dim chunks they fall into
+        const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
+        uint64_t pads_lo = 0, pads_hi = 0;                 // 16 bits per chunk: which pads fall into it
+        for (int j = 0; j < n_pad; ++j) {
+            const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
+            const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
+            if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+        }
+        // pass 2: per 16-dim chunk map the indices, patch the outliers in the tile, contract on the tensor cores
+        for (int ch = 0; ch < 8; ++ch) {
+            uint32_t r8[8];
+            const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
+            const bool whole = ch * 16 + 16 <= n_fit;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
+                uint32_t v = lds_u32(ws.tab + sym * 128);
+                if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;      // clipped positions (and lanes past the end) are +0
+                if (i & 1) r8[i >> 1] |= v << 16; else r8[i >> 1] = v;
+            }
             __syncwarp();                                  // the previous tile has been read
             sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
             sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
-        };
-        auto contract = [&](int ch) {
+            uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
+            while (mine) {                                 // ascending: a later pad overrides an earlier one
+                const int j = __ffs(static_cast<int>(mine)) - 1;
+                mine &= mine - 1;
+                const uint32_t f = read_pad(ws, j);
+                const uint32_t byte = (f & 15u) * 2;
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
+                             "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
+            }
             __syncwarp();                                  // tile complete
             uint32_t a[2][4];
 #pragma unroll
@@ -975,8 +1005,8 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                 const uint32_t tok = (lane >> 4) * 8 + (lane & 7u) + 16 * ks, half = (lane >> 3) & 1u;
                 ldmatrix_x4_trans(a[ks], stage + tok * 32 + ((half ^ ((tok >> 2) & 1u)) << 4));
             }
-            // ch is uniform but not a compile-time constant inside the decode loop: pick the accumulator set by
-            // a chain of uniform branches so that it stays in registers
+            // ch is uniform but not a compile-time constant: pick the accumulator set by uniform branches so
+            // that it stays in registers
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 if (ch == k) {
@@ -987,49 +1017,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                     }
                 }
             }
-        };
-        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym) {
-            const int slot = (n & 15) >> 1;
-            v = valid ? v : 0u;
-            if (n & 1) r8[slot] |= v << 16; else r8[slot] = v;
-            packed |= sym << ((n & 7) * 4);
-            if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
-            if ((n & 15) == 15 && n != 127) { stage_rows(); contract(n >> 4); }
-        });
-        stage_rows();                                      // dims 112..127
-        const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
-        if (n_pad > 0) {
-            float pown[8];                                 // this token's weight under each query head
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                const float2 st = stats_s[r];
-                pown[r] = r < q_per_kv ? expf(d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] - st.x) * st.y : 0.0f;
-            }
-            uint64_t seen_lo = 0, seen_hi = 0;
-            for (int j = n_pad - 1; j >= 0; --j) {         // the last pad wins on a duplicate location
-                const uint32_t f = read_pad(ws, j);
-                const uint32_t loc = f & 127u;
-                const uint64_t bit = 1ull << (loc & 63u);
-                const bool upper = loc >= 64u;
-                if ((upper ? seen_hi : seen_lo) & bit) continue;
-                if (upper) seen_hi |= bit; else seen_lo |= bit;
-                const uint32_t val16 = f2h_bits(fp8_to_float(f >> 7) * T);
-                if (loc >= 112u) {
-                    const uint32_t byte = (loc - 112u) * 2;
-                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
-                                 "h"(static_cast<unsigned short>(val16)) : "memory");
-                } else {
-                    const uint32_t word = lds_u32(ws.syms + (loc >> 3) * 128);
-                    const uint32_t sym = (word >> ((loc & 7u) * 4)) & 15u;
-                    const float mapped = __half2float(__ushort_as_half(static_cast<unsigned short>(lds_u32(ws.tab + sym * 128))));
-                    const float delta = __half2float(__ushort_as_half(static_cast<unsigned short>(val16))) - mapped;
-#pragma unroll
-                    for (int r = 0; r < 8; ++r)
-                        asm volatile("red.shared.add.f32 [%0], %1;" ::"r"(corr_addr + (loc * 8 + r) * 4), "f"(delta * pown[r]) : "memory");
-                }
-            }
         }
-        contract(7);
     }
     if (cur_bh >= 0) flush(cur_bh);
 }
@@ -1394,7 +1382,7 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
 // ecco_attn_values
 // ---------------------------------------------------------------------------------------------
 namespace {
-constexpr int kAvWarps = 18;
+constexpr int kAvWarps = 16;    // 512 tokens per unit: divides the usual sequence lengths
 struct AvPlan { int grid; size_t stats_bytes, partial_bytes, ticket_bytes; };
 AvPlan av_plan(int batch, int n_kv_heads, int seq, int q_per_kv, int ctas_max)
 {
@@ -1434,7 +1422,7 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     if (!d_workspace || !aligned16(d_workspace)) return d_workspace ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (workspace_bytes < p.stats_bytes + p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     auto kernel = ecco_attn_values_kernel<kAvWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kAvWarps) * kAvWarpBytes + 2 * kGroup * 8 * sizeof(float);
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kAvWarps) * kAvWarpBytes + kGroup * 8 * sizeof(float);
     static thread_local bool configured[64] = {};
     if (!configured[di.device]) {
         rc = set_smem(kernel, smem);
