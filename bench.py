@@ -195,13 +195,13 @@ def cpu_baseline(layer, c: int):
 WORKLOADS = {
     "cfg2": dict(label="cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
                        "+ cfg3 K and V caches [8][32][4096][128]",
-                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache)",
+                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache); --only kvcomp times ecco_kv_compress over the whole K cache",
                  l2="inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
     "cfg4": dict(label="cfg4 llama-70b-shaped MLP weights (gate, up 28672x8192; down 8192x28672; 5,505,024 groups)",
                  step="decompress x3, gemv batch 1 x3; plus a decompress sweep over 64 MiB .. 4 GiB streams (stream_sweep)",
                  l2="inputs larger than L2: each step streams 336 MiB of blocks and writes 1.3 GiB"),
     "cfg5": dict(label="cfg5 long-context GQA K and V caches [16][8][32768][128] (4,194,304 groups each)",
-                 step="decompress x1 (K), attn_scores x1 and attn_values x1 (8 query heads per KV head)",
+                 step="decompress x1 (K), attn_scores x1 and attn_values x1 (8 query heads per KV head); --only kvcomp times ecco_kv_compress over the whole K cache",
                  l2="inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB"),
     "small": dict(label="reduced (profiling): q + gate of cfg2, K cache [2][32][4096][128]",
                   step="decompress x2, gemv batch 1 x2, gemv batch 8 x2, attn_scores x1, attn_values x1",
@@ -212,16 +212,18 @@ WORKLOADS = {
 def build_workload(name, workloads):
     """-> (weight tensors, kv tensor or None, q_per_kv, decompress_kv, default segments)."""
     if name == "cfg5":
-        kt, vt = workloads.config5(which=("K", "V"))
+        kt, vt = workloads.config5(which=("K", "V"), keep_source=True)
+        vt.source = None
         return [], (kt, vt), 8, True, ["decompress", "attn", "attnv"]
     if name == "cfg4":
         return workloads.config4(), None, 1, False, ["decompress", "gemv1"]
     if name == "small":
         base = workloads.calibrate_kv(3, 32)
-        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, base)
+        kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, base, keep_source=True)
         vt = workloads.kv_tensor("V", 2, 32, 4096, 1003 * 16 + 1, 3003, base)
         return workloads.config2(names=("q", "gate")), (kt, vt), 1, False, ["decompress", "gemv1", "gemv8", "attn", "attnv"]
-    kt, vt = workloads.config3(which=("K", "V"))
+    kt, vt = workloads.config3(which=("K", "V"), keep_source=True)
+    vt.source = None
     return workloads.config2(), (kt, vt), 1, False, ["decompress", "gemv1", "gemv8", "attn", "attnv"]
 
 
@@ -270,6 +272,8 @@ def run_ours(args):
         kv.update(v_meta=B.meta_to_device(vt.meta), v_blocks=torch.from_numpy(vt.blocks).cuda(),
                   attn_out=torch.empty((kb, kh * q_per_kv, G), dtype=torch.float32, device="cuda"),
                   av_ws=torch.empty(avb, dtype=torch.uint8, device="cuda"), av_wsb=avb)
+        if "kvcomp" in segs:
+            kv.update(x=torch.from_numpy(kt.source.reshape(-1)).cuda(), cblocks=torch.empty((kt.n_groups, BLOCK), dtype=torch.uint8, device="cuda"))
         if decompress_kv:
             kv["out"] = torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")
             dec.append(kv)
@@ -292,6 +296,10 @@ def run_ours(args):
             B.ecco_attn_values(kv["v_meta"], kv["v_blocks"], kb, kh, kseq, q_per_kv, kv["scores"], kv["attn_out"], kv["av_ws"],
                                kv["av_wsb"], stream)
 
+    def seg_kvcomp():
+        if kv is not None:
+            B.ecco_kv_compress(kv["meta"], kv["x"], kv["n"], kv["cblocks"], stream)
+
     def step(ev=None):
         if ev: ev[0].record(stream)
         if "decompress" in segs: seg_decompress()
@@ -304,6 +312,8 @@ def run_ours(args):
         if ev: ev[4].record(stream)
         if "attnv" in segs: seg_attnv()
         if ev: ev[5].record(stream)
+        if "kvcomp" in segs: seg_kvcomp()
+        if ev: ev[6].record(stream)
 
     def barrier():
         if dist is not None:
@@ -313,7 +323,7 @@ def run_ours(args):
     warmup = max(args.warmup, 3)
     for _ in range(warmup):
         step()
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(6)] for _ in range(args.steps)]
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(7)] for _ in range(args.steps)]
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
@@ -326,9 +336,9 @@ def run_ours(args):
     clocks = sampler.stop()
     assert B.ecco_device_status() == 0, "a kernel reported a device-side timeout"
 
-    total_ms = events[0][0].elapsed_time(events[-1][5])
-    seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(5)]
-    total_ms, dec_ms, g1_ms, g8_ms, at_ms, av_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
+    total_ms = events[0][0].elapsed_time(events[-1][6])
+    seg_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) for i in range(6)]
+    total_ms, dec_ms, g1_ms, g8_ms, at_ms, av_ms, kc_ms = distutil.max_over_ranks([total_ms] + seg_ms, dist, "cuda")   # slowest rank decides
 
     groups = sum(d["n"] for d in dec)
     out_bytes = groups * G * 2
@@ -402,7 +412,7 @@ def run_ours(args):
             traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
     # the fused kernels against the same HBM peak (algorithmic bytes: blocks + vectors + results); what bounds them
     # is the SM load/store pipe, so the symbol rate is reported next to the HBM fraction
-    seg_total = dec_ms + g1_ms + g8_ms + at_ms + av_ms
+    seg_total = dec_ms + g1_ms + g8_ms + at_ms + av_ms + kc_ms
     kernels = []
 
     def kernel_entry(name, ms, alg_bytes_per_step, symbols_per_step):
@@ -421,6 +431,7 @@ def run_ours(args):
     if kv is not None:
         kernel_entry(f"ecco_attn_scores q_per_kv {q_per_kv}", at_ms if "attn" in segs else 0, kv["n"] * (BLOCK + 4 * q_per_kv), kv["n"] * G)
         kernel_entry(f"ecco_attn_values q_per_kv {q_per_kv}", av_ms if "attnv" in segs else 0, kv["n"] * (BLOCK + 4 * q_per_kv), kv["n"] * G)
+        kernel_entry("ecco_kv_compress", kc_ms if "kvcomp" in segs else 0, kv["n"] * (BLOCK + 2 * G), kv["n"] * G)
     info = WORKLOADS[wname]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
@@ -430,7 +441,7 @@ def run_ours(args):
                    "format": "S=64, H=4, group 128, 64-byte blocks"},
         "segments_us_per_step": {"decompress": dec_ms / args.steps * 1e3, "gemv_batch1": g1_ms / args.steps * 1e3,
                                  "gemv_batch8": g8_ms / args.steps * 1e3, "attn_scores": at_ms / args.steps * 1e3,
-                                 "attn_values": av_ms / args.steps * 1e3},
+                                 "attn_values": av_ms / args.steps * 1e3, "kv_compress": kc_ms / args.steps * 1e3},
         "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3 if wname == "cfg2" else None,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",

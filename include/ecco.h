@@ -173,6 +173,14 @@ int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, int32_t batch
                      int32_t q_per_kv, const float* d_scores, float* d_out, void* d_workspace, size_t workspace_bytes,
                      void* stream);
 
+/* Online 4x compressor for the KV cache (Sec. 4.3: sorter, min/max pattern selector, four encoders,
+ * pack and clip): n_groups*128 fp16 device values -> n_groups*64 bytes at d_blocks, with the
+ * patterns, codebooks and exponent of d_meta (the device image, which also carries the encoder
+ * tables).  The blocks are byte-identical to ecco_encode_host(meta, x, n_groups,
+ * ECCO_SELECT_MINMAX | ECCO_KEEP_EXPONENT, ...).  Inputs must be finite (non-finite values give
+ * unspecified blocks, never a fault); values above 448 * 2^e saturate. */
+int ecco_kv_compress(const void* d_meta, const void* d_x_fp16, uint64_t n_groups, uint8_t* d_blocks, void* stream);
+
 /* ---------------------------------------------------------------- 2x activation format (device) */
 
 /* Sec. 3.2 "Activation Compression", Sec. 4.2 / 4.3 low-ratio (de)compressor: 64 fp16 values <-> one

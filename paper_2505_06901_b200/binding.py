@@ -34,7 +34,7 @@ EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
     "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
-    "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
+    "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
 
@@ -93,6 +93,7 @@ def lib():
         L.ecco_attn_values_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.ecco_attn_values_workspace_bytes.restype = sz
         L.ecco_attn_values.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.ecco_kv_compress.argtypes = [vp, vp, u64, vp, vp]
         L.ecco_act_compress.argtypes = [vp, u64, vp, vp]
         L.ecco_act_decompress.argtypes = [vp, u64, vp, vp]
         L.ecco_error_string.argtypes = [C.c_int]
@@ -270,6 +271,11 @@ def ecco_attn_values(d_meta, d_vblocks, batch: int, n_kv_heads: int, seq: int, q
     _check(lib().ecco_attn_values(_ptr(d_meta), _ptr(d_vblocks), batch, n_kv_heads, seq, q_per_kv, _ptr(d_scores), _ptr(d_out),
                                   _ptr(d_workspace) if d_workspace is not None else None, workspace_bytes, _stream(stream)),
            "ecco_attn_values")
+
+
+def ecco_kv_compress(d_meta, d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:
+    """Online 4x compressor (min/max pattern selection, calibrated exponent): fp16 device tensor -> 64-byte blocks."""
+    _check(lib().ecco_kv_compress(_ptr(d_meta), _ptr(d_x_fp16), n_groups, _ptr(d_blocks), _stream(stream)), "ecco_kv_compress")
 
 
 def ecco_act_compress(d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:

@@ -22,7 +22,7 @@ constexpr int kExpMin = -32, kExpMax = 16;
 // Device image of the per-tensor metadata.  The tables follow the 64-byte header back to back
 // so that one bulk copy brings them into shared memory.
 constexpr uint32_t kDevMagic = 0x4F434345u;  // "ECCO"
-constexpr uint32_t kDevVersion = 1;
+constexpr uint32_t kDevVersion = 2;
 struct DevHeader {
     uint32_t magic, version;
     int32_t S, H, e;
@@ -38,8 +38,14 @@ constexpr uint32_t kOffKpLut = kOffPattern + kPatternBytes;           // [4096] 
 constexpr uint32_t kKpLutBytes = (1u << kKpMaxLen) * 2;
 constexpr uint32_t kOffSymLut = kOffKpLut + kKpLutBytes;              // [S*H = 256][256] u8: len << 4 | sym
 constexpr uint32_t kSymLutBytes = kMaxPatterns * kCodebooks * 256;
-constexpr uint32_t kDevBytes = kOffSymLut + kSymLutBytes;             // 75840
-constexpr uint32_t kTableBytes = kDevBytes - kOffPattern;             // 75776, a multiple of 16
+constexpr uint32_t kTableBytes = kOffSymLut + kSymLutBytes - kOffPattern;   // 75776: what the decoders stage, a multiple of 16
+// encoder tables for the device-side compressor, after the decode tables
+constexpr uint32_t kOffEncCb = kOffSymLut + kSymLutBytes;             // [256][16] u16: stream-order codeword | length << 8
+constexpr uint32_t kEncCbBytes = kMaxPatterns * kCodebooks * kSymbols * 2;
+constexpr uint32_t kOffEncKp = kOffEncCb + kEncCbBytes;               // [64] u16: stream-order ID_KP codeword | length << 12
+constexpr uint32_t kEncKpBytes = kMaxPatterns * 2;
+constexpr uint32_t kDevBytes = kOffEncKp + kEncKpBytes;               // 84160
+constexpr uint32_t kEncBytes = kEncCbBytes + kEncKpBytes;             // 8320, a multiple of 16
 // Both lookup tables are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.
 //

@@ -794,6 +794,16 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
                     t[(tmp.cb_rev[k][c][s] | (hi << L)) ^ rot] = static_cast<uint8_t>((L << 4) | s);
             }
         }
+    // encoder tables: codeword in stream order (first code bit in bit 0) and its length
+    uint16_t* ecb = reinterpret_cast<uint16_t*>(base + kOffEncCb);
+    uint16_t* ekp = reinterpret_cast<uint16_t*>(base + kOffEncKp);
+    for (int k = 0; k < tmp.S; ++k) {
+        ekp[k] = static_cast<uint16_t>(tmp.kp_rev[k] | (tmp.kp_len[k] << 12));
+        for (int c = 0; c < kCodebooks; ++c)
+            for (int s = 0; s < kSymbols; ++s)
+                ecb[(static_cast<size_t>(k) * kCodebooks + c) * kSymbols + s] =
+                    static_cast<uint16_t>(tmp.cb_rev[k][c][s] | (tmp.cb_len[k][c][s] << 8));
+    }
     // unused pattern rows (S < 64) decode with 4-bit codes so that every table entry is valid
     for (int k = tmp.S; k < kMaxPatterns; ++k)
         for (int c = 0; c < kCodebooks; ++c) {

@@ -435,3 +435,64 @@ def test_attn_values_on_garbage_blocks_and_peaked_softmax(B, eo, kv_small, synth
     got = gpu_attn_values(B, lib_meta_from_oracle(B, meta), rb, 2, 2, 700, 2, scores)
     ref, refabs = eo.attn_values(meta, rb, 2, 2, 700, 2, scores)
     check_fused(got, ref, refabs)
+
+
+# ------------------------------------------------------------------ online KV compressor
+def gpu_kv_compress(B, lmeta, x):
+    n = x.size // 128
+    d_meta = B.meta_to_device(lmeta)
+    d_x = dev(x.reshape(-1)) if n else torch.empty(128, dtype=torch.float16, device="cuda")
+    d_blocks = torch.full((max(n, 1), 64), 0xEE, dtype=torch.uint8, device="cuda")
+    B.ecco_kv_compress(d_meta, d_x, n, d_blocks)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    return d_blocks.cpu().numpy()[:n]
+
+
+def assert_blocks_equal(got, want):
+    bad = np.nonzero((got != want).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} of {got.shape[0]} blocks differ; first {bad[:5]}"
+
+
+@pytest.mark.parametrize("n_groups", [0, 1, 7, 8, 9, 2048])
+def test_kv_compress_matches_oracle_encoder(B, eo, kv_small, n_groups):
+    meta = kv_small["meta"]
+    x = kv_small["k"].reshape(-1, 128)[:n_groups]
+    got = gpu_kv_compress(B, lib_meta_from_oracle(B, meta), x)
+    if n_groups:
+        assert_blocks_equal(got, kv_small["blocks"][:n_groups])
+
+
+def test_kv_compress_edge_groups_and_s16(B, eo, kv_small, synth):
+    meta = kv_small["meta"]
+    rng = np.random.Generator(np.random.PCG64(77))
+    groups = [np.zeros(128), np.full(128, 0.5), np.full(128, -3.0), np.concatenate([np.full(64, 1.0), np.full(64, -1.0)]),
+              np.full(128, 2.0 ** -24), rng.standard_normal(128) * 1e-3, rng.standard_normal(128) * 300,   # saturating scales
+              np.where(np.arange(128) % 2 == 0, 5.0, -5.0), np.arange(128) - 64.0, rng.choice([-2.0, 0.0, 2.0], 128)]
+    for _ in range(200):
+        g = rng.standard_normal(128) * rng.choice([0.1, 1.0, 10.0])
+        g[rng.integers(128)] *= rng.choice([1.0, 20.0])
+        if rng.random() < 0.3:
+            g[rng.integers(128, size=5)] = g[rng.integers(128)]            # ties in |x|
+        groups.append(g)
+    x = np.array(groups, dtype=np.float16)
+    want, st = eo.encode(meta, x, eo.SELECT_MINMAX)
+    assert st.clipped_groups > 0 and st.padded_groups > 0
+    assert_blocks_equal(gpu_kv_compress(B, lib_meta_from_oracle(B, meta), x), want)
+    # the paper's hardware compressor works with 16 patterns
+    cal = synth.kv_cache(1, 4, 512, 2003, 3003)
+    m16 = eo.calibrate(cal, S=16, H=4, seed=3, select=eo.SELECT_MINMAX)
+    want, _ = eo.encode(m16, kv_small["k"], eo.SELECT_MINMAX)
+    assert_blocks_equal(gpu_kv_compress(B, lib_meta_from_oracle(B, m16), kv_small["k"]), want)
+    # a skewed codebook: long streams (heavy clipping) and short ones (16 pads)
+    skew = make_meta(eo, skew_lens, seed=3)
+    xs = (rng.standard_t(3, size=(512, 128)) * 0.05).astype(np.float16)
+    want, st = eo.encode(skew, xs, eo.SELECT_MINMAX)
+    assert_blocks_equal(gpu_kv_compress(B, lib_meta_from_oracle(B, skew), xs), want)
+
+
+def test_kv_compress_full_size_round_trip(B, eo, W, synth):
+    """cfg 3 K cache: GPU-compressed blocks equal the host encoder's, and decompress to the same fp16."""
+    (t,) = W.config3(which=("K",), keep_source=True)
+    got = gpu_kv_compress(B, t.meta, t.source)
+    assert_blocks_equal(got, t.blocks)

@@ -160,14 +160,17 @@ def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
     ometa = cfg1_small["meta"]
     lm = lib_meta_from_oracle(binding, ometa)
     img = binding.ecco_meta_serialize_device(lm)
-    assert img.size == binding.ecco_meta_device_bytes(lm) == 75840
+    assert img.size == binding.ecco_meta_device_bytes(lm) == 84160
     hdr = img[:64].view(np.uint32)
     assert hdr[0] == 0x4F434345 and hdr[2] == 64 and hdr[3] == 4 and hdr[4:5].view(np.int32)[0] == ometa.e
     assert img[20:24].view(np.float32)[0] == 2.0 ** ometa.e
     pat = img[64:64 + 2048].view(np.float16).reshape(64, 16)
     assert np.array_equal(pat[:, :15].view(np.uint16), ometa.patterns().view(np.uint16)) and np.all(pat[:, 15] == 0)
     kpl = img[64 + 2048:64 + 2048 + 8192].view(np.uint16)
-    syml = img[64 + 2048 + 8192:].reshape(256, 256)
+    syml = img[64 + 2048 + 8192:64 + 2048 + 8192 + 65536].reshape(256, 256)
+    enc = img[75840:75840 + 8192].view(np.uint16).reshape(64, 4, 16)
+    assert np.array_equal(enc >> 8, ometa.cb_lengths())                  # encoder table: lengths per (pattern, codebook, symbol)
+    assert np.array_equal(img[84032:84160].view(np.uint16) >> 12, ometa.kp_lengths())
     assert np.all((syml >> 4) >= 2) and np.all((syml >> 4) <= 8)
     for g in range(0, 2048, 41):
         blk = cfg1_small["blocks"][g]
