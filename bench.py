@@ -42,10 +42,11 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
-    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5", "act2x"],
+    ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5", "act2x", "var"],
                     help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg4: 70B-shaped MLP weights + stream-size "
                          "sweep; cfg5: long-context GQA K cache [16][8][32768][128] (decompress + attention scores with 8 "
-                         "query heads per KV head); act2x: the 2x activation codec on a [32768][8192] fp16 tensor")
+                         "query heads per KV head); act2x: the 2x activation codec on a [32768][8192] fp16 tensor; var: the "
+                         "variable-length container on the cfg2 gate/up/down matrices")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -459,6 +460,87 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_var(args):
+    """Variable-length container: one step = ecco_var_decompress of the cfg-2 gate, up and down matrices."""
+    import torch
+
+    from paper_2505_06901_b200 import binding as B
+    from paper_2505_06901_b200 import distutil, workloads
+
+    rank, world, local = distutil.rank_info()
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    mats = []
+    for t in workloads.config2(names=("gate", "up", "down"), keep_source=True):
+        stream, index, total = B.ecco_var_encode_host(t.meta, t.source, B.SELECT_MSE | B.KEEP_EXPONENT)
+        mats.append(dict(n=t.n_groups, meta=B.meta_to_device(t.meta), stream=torch.from_numpy(stream).cuda(), index=torch.from_numpy(index).cuda(),
+                         blocks=torch.from_numpy(t.blocks).cuda(), out=torch.empty(t.n_groups * G, dtype=torch.float16, device="cuda"),
+                         stream_bytes=stream.size, index_bytes=index.size, total_bits=total))
+        t.source = None
+    st = torch.cuda.current_stream()
+    warmup = max(args.warmup, 3)
+
+    def step(ev=None):
+        if ev: ev[0].record(st)
+        for d in mats:
+            B.ecco_var_decompress(d["meta"], d["stream"], d["index"], d["n"], d["out"], st)
+        if ev: ev[1].record(st)
+        for d in mats:
+            B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], st)
+        if ev: ev[2].record(st)
+
+    for _ in range(warmup):
+        step()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    l0 = B.ecco_kernel_launch_count()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    for e in ev:
+        step(e)
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    launches = B.ecco_kernel_launch_count() - l0
+    clocks = sampler.stop()
+    v_ms = sum(e[0].elapsed_time(e[1]) for e in ev)
+    b_ms = sum(e[1].elapsed_time(e[2]) for e in ev)
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    total_ms, v_ms, b_ms = distutil.max_over_ranks([total_ms, v_ms, b_ms], dist, "cuda")
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peaks()
+    groups = sum(d["n"] for d in mats)
+    alg = sum(d["stream_bytes"] + 4 * d["n"] + d["n"] * G * 2 for d in mats)     # stream + 4-byte start per group + fp16 out
+    v_s = v_ms / 1e3 / args.steps
+    line = {
+        "metric": "var_decompress_output_GBps", "value": world * groups * G * 2 / v_s / 1e9, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "variable-length container of the cfg2 gate, up (11008x4096) and down (4096x11008) matrices",
+                   "step": "ecco_var_decompress x3, then ecco_decompress x3 of the same matrices as 64-byte blocks (for comparison)",
+                   "l2": "inputs larger than L2: 63 MiB of stream and 258 MiB of output per segment",
+                   "mean_bits_per_group": sum(d["total_bits"] for d in mats) / groups},
+        "segments_us_per_step": {"var_decompress": v_ms / args.steps * 1e3, "block_decompress": b_ms / args.steps * 1e3},
+        "clocks": clocks, "gpu_launches": int(launches), "e2e": None,
+        "roofline": {"kernel": "ecco_var_decompress_kernel", "bound": "hbm", "achieved": alg / v_s / 1e9, "peak": peak, "unit": "GB/s",
+                     "frac": alg / v_s / 1e9 / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": alg / len(mats), "avg_launch_us": v_s * 1e6 / len(mats)},
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 def run_act2x(args):
     """2x activation codec (Sec. 3.2): one step = compress + decompress of a [32768][8192] fp16 N(0,1) tensor."""
     import torch
@@ -567,5 +649,7 @@ if __name__ == "__main__":
         run_reference(a)
     elif a.workload == "act2x":
         run_act2x(a)
+    elif a.workload == "var":
+        run_var(a)
     else:
         run_ours(a)

@@ -181,6 +181,25 @@ int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, int32_t batch
  * unspecified blocks, never a fault); values above 448 * 2^e saturate. */
 int ecco_kv_compress(const void* d_meta, const void* d_x_fp16, uint64_t n_groups, uint8_t* d_blocks, void* stream);
 
+/* ---------------------------------------------------------------- variable-length container */
+
+/* The same per-group fields as the 64-byte block (scale byte, ID_HF, ID_KP codeword, 128 codewords;
+ * Sec. 3.2) written back to back into one bit stream: nothing is clipped, nothing is padded, and
+ * a side index says where every group starts.  (The paper has only the fixed block; this layout
+ * trades the fixed 4x ratio for the absence of clipping loss.)  Stream bit k = bit k&7 of byte k>>3.
+ * Index (host and device, 8-byte aligned): u64 total_bits | u64 chunk_base[ceil(n/4096)] | u32
+ * offset[n]; group g starts at bit chunk_base[g >> 12] + offset[g] and sees the stream up to the
+ * start of group g+1 (zeros after that).  ecco_var_encode_host quantises exactly like
+ * ecco_encode_host (same flags) and needs stream_capacity >= 16 * ceil(total_bits / 128), at most
+ * ecco_var_stream_bytes_bound(n_groups).  ecco_var_decompress: d_stream 16-byte aligned and a
+ * multiple of 16 bytes long, d_index 8-byte aligned, output as ecco_decompress. */
+size_t ecco_var_stream_bytes_bound(uint64_t n_groups);
+size_t ecco_var_index_bytes(uint64_t n_groups);
+int ecco_var_encode_host(ecco_meta* meta, const uint16_t* src_fp16, uint64_t n_groups, uint32_t flags, uint8_t* dst_stream,
+                         size_t stream_capacity, void* dst_index, size_t index_capacity, uint64_t* total_bits_out);
+int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, const void* d_index, uint64_t n_groups, void* d_out_fp16,
+                        void* stream);
+
 /* ---------------------------------------------------------------- 2x activation format (device) */
 
 /* Sec. 3.2 "Activation Compression", Sec. 4.2 / 4.3 low-ratio (de)compressor: 64 fp16 values <-> one

@@ -1015,3 +1015,95 @@ int eo_attn_values(const eo_meta* M, const uint8_t* vblocks, int batch, int n_kv
     free(p);
     return EO_OK;
 }
+
+/* ------------------------------------------------------------------------------------ */
+/* Variable-length container (the alternative layout without clipping and padding): the    */
+/* same per-group fields -- scale byte, ID_HF, ID_KP codeword, 128 codewords (Sec. 3.2) -- */
+/* written back to back into one bit stream, plus an index of where every group starts.    */
+/* reading (the paper only has the fixed 64-byte block; this layout is this build's):      */
+/* stream bit k = bit k&7 of byte k>>3 as in the block; the groups of one chunk of 4096    */
+/* groups follow each other without gaps; offsets[g] is the absolute start bit of group g  */
+/* and offsets[n_groups] the total length.  Nothing is clipped and nothing is padded.      */
+/* The decoder of group g sees the stream bits in [offsets[g], offsets[g+1]) and zeros      */
+/* after them, so any stream and any offsets decode to something.                           */
+/* ------------------------------------------------------------------------------------ */
+#define EO_VAR_MAX_BITS (10 + EO_KP_MAXLEN + EO_G * 8)
+
+static int eo_sget_bit(const uint8_t* s, uint64_t k) { return (s[k >> 3] >> (k & 7)) & 1; }
+static void eo_sset_bit(uint8_t* s, uint64_t k, int b) { if (b) s[k >> 3] |= (uint8_t)(1u << (k & 7)); }
+
+/* stream must be zero-initialised and hold (total bits + 7) / 8 bytes; returns the bit count through offsets */
+int eo_var_encode(const eo_meta* M, const uint16_t* x16, uint64_t n_groups, int select, uint8_t* stream, uint64_t* offsets)
+{
+    int rc = eo_meta_check(M);
+    if (rc) return rc;
+    uint16_t kpcode[EO_MAXS], code[EO_NSYM];
+    eo_canonical_codes(M->kp_len, M->S, EO_KP_MAXLEN, kpcode, NULL);
+    uint64_t pos = 0;
+    for (uint64_t g = 0; g < n_groups; ++g) {
+        float u[EO_G]; uint8_t sym[EO_G]; int32_t p, kp; uint8_t qs;
+        rc = eo_quantize_group(M, x16 + g * EO_G, select, &p, &qs, u, &kp, sym, NULL);
+        if (rc) return rc;
+        int hf = 0, best_len = 1 << 30;
+        for (int h = 0; h < EO_H; ++h) {
+            int L = 0;
+            for (int i = 0; i < EO_G; ++i) L += M->cb_len[kp][h][sym[i]];
+            if (L < best_len) { best_len = L; hf = h; }
+        }
+        eo_canonical_codes(M->cb_len[kp][hf], EO_NSYM, 8, code, NULL);
+        offsets[g] = pos;
+        for (int i = 0; i < 8; ++i) eo_sset_bit(stream, pos++, (qs >> i) & 1);
+        for (int i = 0; i < 2; ++i) eo_sset_bit(stream, pos++, (hf >> i) & 1);
+        for (int i = 0; i < M->kp_len[kp]; ++i) eo_sset_bit(stream, pos++, (kpcode[kp] >> (M->kp_len[kp] - 1 - i)) & 1);
+        for (int n = 0; n < EO_G; ++n) {
+            int L = M->cb_len[kp][hf][sym[n]];
+            for (int i = 0; i < L; ++i) eo_sset_bit(stream, pos++, (code[sym[n]] >> (L - 1 - i)) & 1);
+        }
+    }
+    offsets[n_groups] = pos;
+    return EO_OK;
+}
+
+/* group g reads bits below offsets[g+1] (and below the total length); everything else reads as 0 */
+int eo_var_decode(const eo_meta* M, const uint8_t* stream, const uint64_t* offsets, uint64_t n_groups, uint16_t* out16)
+{
+    int rc = eo_meta_check(M);
+    if (rc) return rc;
+    float T = (float)ldexp(1.0, M->e);
+    uint16_t kpcode[EO_MAXS], code[EO_NSYM];
+    eo_canonical_codes(M->kp_len, M->S, EO_KP_MAXLEN, kpcode, NULL);
+    uint64_t total = offsets[n_groups];
+#define EO_SBIT(k) ((k) < limit ? eo_sget_bit(stream, (k)) : 0)
+    for (uint64_t g = 0; g < n_groups; ++g) {
+        uint64_t pos = offsets[g];
+        uint64_t limit = offsets[g + 1] < total ? offsets[g + 1] : total;
+        uint32_t qs = 0, hf = 0;
+        for (int i = 0; i < 8; ++i) qs |= (uint32_t)EO_SBIT(pos + i) << i;
+        for (int i = 0; i < 2; ++i) hf |= (uint32_t)EO_SBIT(pos + 8 + i) << i;
+        pos += 10;
+        int kp = -1;
+        for (int k = 0; k < M->S && kp < 0; ++k) {
+            int ok = 1;
+            for (int i = 0; i < M->kp_len[k] && ok; ++i) ok = EO_SBIT(pos + i) == (int)((kpcode[k] >> (M->kp_len[k] - 1 - i)) & 1);
+            if (ok) kp = k;
+        }
+        if (kp < 0) return EO_ERR_META;
+        pos += M->kp_len[kp];
+        float s = fabsf(eo_e4m3_to_f32((uint8_t)qs)) * T;
+        eo_canonical_codes(M->cb_len[kp][hf], EO_NSYM, 8, code, NULL);
+        for (int n = 0; n < EO_G; ++n) {
+            int found = -1;
+            for (int c = 0; c < EO_NSYM && found < 0; ++c) {
+                int L = M->cb_len[kp][hf][c], ok = 1;
+                for (int i = 0; i < L && ok; ++i) ok = EO_SBIT(pos + i) == (int)((code[c] >> (L - 1 - i)) & 1);
+                if (ok) found = c;
+            }
+            if (found < 0) return EO_ERR_META;
+            pos += M->cb_len[kp][hf][found];
+            out16[g * EO_G + n] = found == 15 ? eo_f32_to_fp16(eo_e4m3_to_f32((uint8_t)qs) * T)
+                                             : eo_f32_to_fp16(eo_fp16_to_f32(M->pattern[kp][found]) * s);
+        }
+    }
+#undef EO_SBIT
+    return EO_OK;
+}

@@ -370,3 +370,29 @@ def attn_values(meta: Meta, vblocks, batch: int, n_kv_heads: int, seq: int, q_pe
     _check(lib().eo_attn_values(C.byref(meta), _p(b, C.c_uint8), batch, n_kv_heads, seq, q_per_kv, _p(s, C.c_float),
                                 _p(out, C.c_double), _p(oa, C.c_double)), "attn_values")
     return out, oa
+
+
+# ---------------------------------------------------------------- variable-length container
+VAR_MAX_BITS = 10 + 12 + 128 * 8
+
+
+def var_encode(meta: Meta, x16, select: int = SELECT_MSE):
+    """-> (stream uint8, offsets uint64 [n_groups + 1]) : the groups' fields back to back, nothing clipped or padded."""
+    x = _u16(x16).reshape(-1)
+    assert x.size % G == 0
+    n = x.size // G
+    stream = np.zeros((n * VAR_MAX_BITS + 7) // 8 + 8, dtype=np.uint8)
+    offsets = np.zeros(n + 1, dtype=np.uint64)
+    _check(lib().eo_var_encode(C.byref(meta), _p(x, C.c_uint16), C.c_uint64(n), select, _p(stream, C.c_uint8),
+                               _p(offsets, C.c_uint64)), "var_encode")
+    return stream[: (int(offsets[n]) + 7) // 8].copy(), offsets
+
+
+def var_decode(meta: Meta, stream, offsets) -> np.ndarray:
+    s = np.ascontiguousarray(stream, dtype=np.uint8)
+    o = np.ascontiguousarray(offsets, dtype=np.uint64)
+    n = o.size - 1
+    assert (int(o[n]) + 7) // 8 <= s.size
+    out = np.zeros((n, G), dtype=np.uint16)
+    _check(lib().eo_var_decode(C.byref(meta), _p(s, C.c_uint8), _p(o, C.c_uint64), C.c_uint64(n), _p(out, C.c_uint16)), "var_decode")
+    return out.view(np.float16)

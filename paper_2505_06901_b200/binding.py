@@ -34,7 +34,8 @@ EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
     "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
-    "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
+    "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress",
+    "ecco_var_stream_bytes_bound", "ecco_var_index_bytes", "ecco_var_encode_host", "ecco_var_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
 
@@ -94,6 +95,12 @@ def lib():
         L.ecco_attn_values_workspace_bytes.restype = sz
         L.ecco_attn_values.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.ecco_kv_compress.argtypes = [vp, vp, u64, vp, vp]
+        L.ecco_var_stream_bytes_bound.argtypes = [u64]
+        L.ecco_var_stream_bytes_bound.restype = sz
+        L.ecco_var_index_bytes.argtypes = [u64]
+        L.ecco_var_index_bytes.restype = sz
+        L.ecco_var_encode_host.argtypes = [vp, vp, u64, C.c_uint32, vp, sz, vp, sz, C.POINTER(u64)]
+        L.ecco_var_decompress.argtypes = [vp, vp, vp, u64, vp, vp]
         L.ecco_act_compress.argtypes = [vp, u64, vp, vp]
         L.ecco_act_decompress.argtypes = [vp, u64, vp, vp]
         L.ecco_error_string.argtypes = [C.c_int]
@@ -201,6 +208,21 @@ def ecco_meta_serialize_device(meta: Meta) -> np.ndarray:
     return buf
 
 
+def ecco_var_encode_host(meta: Meta, src_fp16, flags: int = SELECT_MSE):
+    """Variable-length container: -> (stream uint8, a multiple of 16 bytes; index uint8; total_bits)."""
+    x = _host_u16(src_fp16).reshape(-1)
+    if x.size % GROUP:
+        raise ValueError("tensor is not a whole number of 128-value groups")
+    n = x.size // GROUP
+    stream = np.empty(int(lib().ecco_var_stream_bytes_bound(n)), dtype=np.uint8)
+    index = np.zeros(int(lib().ecco_var_index_bytes(n)), dtype=np.uint8)
+    total = C.c_uint64(0)
+    _check(lib().ecco_var_encode_host(meta.handle, x.ctypes.data, n, flags, stream.ctypes.data, stream.size, index.ctypes.data,
+                                      index.size, C.byref(total)), "ecco_var_encode_host")
+    used = (total.value + 127) // 128 * 16
+    return stream[:used].copy(), index, total.value
+
+
 # ------------------------------------------------------------------ device calls
 def _ptr(t) -> int:
     """Raw device pointer of a CUDA torch tensor (or an int that already is one)."""
@@ -276,6 +298,12 @@ def ecco_attn_values(d_meta, d_vblocks, batch: int, n_kv_heads: int, seq: int, q
 def ecco_kv_compress(d_meta, d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:
     """Online 4x compressor (min/max pattern selection, calibrated exponent): fp16 device tensor -> 64-byte blocks."""
     _check(lib().ecco_kv_compress(_ptr(d_meta), _ptr(d_x_fp16), n_groups, _ptr(d_blocks), _stream(stream)), "ecco_kv_compress")
+
+
+def ecco_var_decompress(d_meta, d_stream, d_index, n_groups: int, d_out_fp16, stream=None) -> None:
+    """Decompress the variable-length container (see ecco_var_encode_host) to fp16 [n_groups][128]."""
+    _check(lib().ecco_var_decompress(_ptr(d_meta), _ptr(d_stream), _ptr(d_index), n_groups, _ptr(d_out_fp16), _stream(stream)),
+           "ecco_var_decompress")
 
 
 def ecco_act_compress(d_x_fp16, n_groups: int, d_blocks, stream=None) -> None:

@@ -60,4 +60,10 @@ constexpr uint32_t kEncBytes = kEncCbBytes + kEncKpBytes;             // 8320, a
 #endif
 ECCO_HD constexpr uint32_t lut_rotation(uint32_t cb) { return ((cb * 11u + (cb >> 3)) & 31u) << 2; }
 
+// Variable-length container: index = u64 total_bits | u64 chunk_base[ceil(n / 4096)] | u32 offset[n];
+// group g starts at stream bit chunk_base[g >> 12] + offset[g].
+constexpr int kVarChunkShift = 12;
+constexpr int kVarMaxBits = kHeaderBits + kKpMaxLen + kGroup * kMaxLen;      // 1046
+ECCO_HD constexpr uint64_t var_chunks(uint64_t n_groups) { return (n_groups + (1ull << kVarChunkShift) - 1) >> kVarChunkShift; }
+
 }  // namespace ecco

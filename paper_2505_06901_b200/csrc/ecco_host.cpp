@@ -628,6 +628,105 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
 }
 
 // ---------------------------------------------------------------------------------------------
+// C ABI: variable-length container (no clipping, no padding; groups back to back + start index)
+// ---------------------------------------------------------------------------------------------
+extern "C" size_t ecco_var_stream_bytes_bound(uint64_t n_groups)
+{
+    return static_cast<size_t>(((n_groups * kVarMaxBits + 127) / 128) * 16 + 16);
+}
+extern "C" size_t ecco_var_index_bytes(uint64_t n_groups)
+{
+    return static_cast<size_t>((8 + 8 * var_chunks(n_groups) + 4 * n_groups + 15) & ~15ull);
+}
+
+extern "C" int ecco_var_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_groups, uint32_t flags, uint8_t* dst_stream,
+                                    size_t stream_capacity, void* dst_index, size_t index_capacity, uint64_t* total_bits_out)
+{
+    if (!m || !dst_index || (n_groups && (!src || !dst_stream))) return ECCO_ERR_INVALID_ARG;
+    if (flags & ~(ECCO_SELECT_MINMAX | ECCO_KEEP_EXPONENT)) return ECCO_ERR_INVALID_ARG;
+    if (index_capacity < ecco_var_index_bytes(n_groups)) return ECCO_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dst_stream) | reinterpret_cast<uintptr_t>(dst_index)) & 7u) return ECCO_ERR_ALIGNMENT;
+    ensure_tables();
+    if (!(flags & ECCO_KEEP_EXPONENT)) {
+        int rc = fit_exponent(src, n_groups * kGroup, 0, &m->e);
+        if (rc) return rc;
+    }
+    int rc = derive(m);
+    if (rc) return rc;
+    const uint32_t select = flags & ECCO_SELECT_MINMAX;
+    const float T = std::ldexp(1.0f, m->e);
+    const int threads = available_cores();
+    // pass 1: the bit length of every group
+    std::vector<uint16_t> bits(static_cast<size_t>(n_groups));
+    std::atomic<int> err{0};
+    auto group_fields = [&](uint64_t g, Scratch& s, Quantized& q, int& hf) -> int {
+        int r = quantize_group(*m, src + g * kGroup, select, T, s, q);
+        if (r) return -1;
+        int total[kCodebooks] = {0, 0, 0, 0};
+        for (int i = 0; i < kGroup; ++i)
+            for (int h = 0; h < kCodebooks; ++h) total[h] += m->cb_len[q.kp][h][q.sym[i]];
+        hf = 0;
+        for (int h = 1; h < kCodebooks; ++h)
+            if (total[h] < total[hf]) hf = h;
+        return kHeaderBits + m->kp_len[q.kp] + total[hf];
+    };
+    parallel_ranges(n_groups, threads, [&](int, uint64_t lo, uint64_t hi) {
+        Scratch s;
+        Quantized q;
+        int hf;
+        for (uint64_t g = lo; g < hi && !err.load(std::memory_order_relaxed); ++g) {
+            int L = group_fields(g, s, q, hf);
+            if (L < 0) { err = ECCO_ERR_NONFINITE_INPUT; break; }
+            bits[g] = static_cast<uint16_t>(L);
+        }
+    });
+    if (err) return err;
+    // index
+    uint64_t* idx64 = static_cast<uint64_t*>(dst_index);
+    uint32_t* off32 = reinterpret_cast<uint32_t*>(idx64 + 1 + var_chunks(n_groups));
+    std::vector<uint64_t> start(static_cast<size_t>(n_groups) + 1);
+    uint64_t pos = 0;
+    for (uint64_t g = 0; g < n_groups; ++g) {
+        if ((g & ((1ull << kVarChunkShift) - 1)) == 0) idx64[1 + (g >> kVarChunkShift)] = pos;
+        off32[g] = static_cast<uint32_t>(pos - idx64[1 + (g >> kVarChunkShift)]);
+        start[g] = pos;
+        pos += bits[g];
+    }
+    start[n_groups] = pos;
+    idx64[0] = pos;
+    if (total_bits_out) *total_bits_out = pos;
+    const size_t need = static_cast<size_t>(((pos + 127) / 128) * 16);
+    if (stream_capacity < need) return ECCO_ERR_INVALID_ARG;
+    std::memset(dst_stream, 0, need);
+    // pass 2: write the fields; neighbouring threads may share a 64-bit word at their range boundary
+    uint64_t* words = reinterpret_cast<uint64_t*>(dst_stream);
+    auto put = [&](uint64_t p, uint64_t v, int nbits) {
+        const uint64_t w = p >> 6;
+        const int off = static_cast<int>(p & 63);
+        __atomic_fetch_or(&words[w], v << off, __ATOMIC_RELAXED);
+        if (off + nbits > 64) __atomic_fetch_or(&words[w + 1], v >> (64 - off), __ATOMIC_RELAXED);
+    };
+    parallel_ranges(n_groups, threads, [&](int, uint64_t lo, uint64_t hi) {
+        Scratch s;
+        Quantized q;
+        int hf = 0;
+        for (uint64_t g = lo; g < hi; ++g) {
+            group_fields(g, s, q, hf);
+            uint64_t p = start[g];
+            put(p, q.qs | (static_cast<uint64_t>(hf) << 8) | (static_cast<uint64_t>(m->kp_rev[q.kp]) << kHeaderBits),
+                kHeaderBits + m->kp_len[q.kp]);
+            p += kHeaderBits + m->kp_len[q.kp];
+            for (int i = 0; i < kGroup; ++i) {
+                const int L = m->cb_len[q.kp][hf][q.sym[i]];
+                put(p, m->cb_rev[q.kp][hf][q.sym[i]], L);
+                p += L;
+            }
+        }
+    });
+    return ECCO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // C ABI: calibration
 // ---------------------------------------------------------------------------------------------
 extern "C" int ecco_calibrate_host(const uint16_t* calib, uint64_t n_groups, const float* weights,

@@ -172,21 +172,20 @@ struct GroupHeader {
     uint32_t lut;       // shared address of the symbol table of (ID_KP, ID_HF), OR-ed with its index rotation
 };
 
-// Pattern retriever (Sec. 4.2): scale byte, ID_HF, Huffman-coded ID_KP; writes the lane's 16
-// dequantised values (fp16 bits, or fp32 bits when kFloatTab) and the transposed bit stream.
+// Pattern retriever (Sec. 4.2): scale byte, ID_HF, Huffman-coded ID_KP from the group's first 22
+// stream bits (hdr, first bit in bit 0); writes the lane's 16 dequantised values (fp16 bits, or
+// fp32 bits when kFloatTab).  first_bit = position of the group's first bit in the lane's staged
+// bit stream.
 template <bool kFloatTab>
-__device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T)
+__device__ __forceinline__ GroupHeader open_header(uint32_t hdr, uint32_t first_bit, uint32_t smem_base, const WarpSmem& ws, float T)
 {
-    const uint32_t (&w)[16] = blk.w;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) sts_u32(ws.bits + i * 128, w[i]);
-    const uint32_t qs = w[0] & 0xffu, hf = (w[0] >> 8) & 3u;
-    const uint32_t kpw = __funnelshift_r(w[0], w[1], 10) & 0xfffu;
+    const uint32_t qs = hdr & 0xffu, hf = (hdr >> 8) & 3u;
+    const uint32_t kpw = (hdr >> kHeaderBits) & 0xfffu;
     uint32_t kpe;
     asm volatile("ld.shared.u16 %0, [%1];" : "=r"(kpe) : "r"(smem_base + kSmemKpLut + kpw * 2));
     const uint32_t kp = kpe & 0xffu;
     GroupHeader h;
-    h.pos = kHeaderBits + (kpe >> 8);
+    h.pos = first_bit + kHeaderBits + (kpe >> 8);
     const uint32_t cb = kp * kCodebooks + hf;
     h.lut = (smem_base + kSmemSymLut + cb * 256) | lut_rotation(cb);   // table rows are 256-byte aligned
     const float top = fp8_to_float(qs) * T;           // FP8 -> FP16 range by the power-of-two factor
@@ -205,19 +204,30 @@ __device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t sme
     return h;
 }
 
+// 64-byte block: stage the 16 words in the lane's column of the transposed bit-stream array, then the header
+template <bool kFloatTab>
+__device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T)
+{
+#pragma unroll
+    for (int i = 0; i < 16; ++i) sts_u32(ws.bits + i * 128, blk.w[i]);
+    return open_header<kFloatTab>(blk.w[0], 0u, smem_base, ws, T);
+}
+
 // Decodes the 128 indices of the lane's group (Sec. 4.2, Huffman decode) and hands each value to
 // sink(n, value_bits, symbol, alive) (kLookup = false skips the value lookup and passes 0).  A codeword that would cross bit 512 ends the group: that and all
 // later positions are delivered as zero (clipped).  Returns the end bit if all 128 fitted, else 0.
 // Must be called by all 32 lanes of the warp.  Four symbols are decoded per window refill; the
 // per-symbol clip test runs only in steps where some lane of the warp reaches bit 512.
-template <bool kLookup = true, class Sink>
+// kLastRow / kEndBit: last data row of the lane's staged stream (two zero rows follow) and the bit
+// at which the stream ends (16 and 512 for the 64-byte block).
+template <bool kLookup = true, uint32_t kLastRow = 16, uint32_t kEndBit = kBlockBits, class Sink>
 __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const WarpSmem& ws, Sink&& sink)
 {
     uint32_t pos = h.pos;
     bool alive = true;
 #pragma unroll 4
     for (int step = 0; step < 32; ++step) {
-        const uint32_t wi = min(pos >> 5, 16u);
+        const uint32_t wi = min(pos >> 5, kLastRow);
         const uint32_t lo = lds_u32(ws.bits + wi * 128), hi = lds_u32(ws.bits + wi * 128 + 128);
         const uint32_t win = __funnelshift_r(lo, hi, pos);           // 32 stream bits from pos
         uint32_t e[4], end[4], acc = 0;
@@ -227,8 +237,8 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
             acc += e[j] >> 4;
             end[j] = acc;
         }
-        if (__any_sync(0xffffffffu, pos + acc > static_cast<uint32_t>(kBlockBits))) {
-            const uint32_t limit = kBlockBits - min(pos, static_cast<uint32_t>(kBlockBits));
+        if (__any_sync(0xffffffffu, pos + acc > kEndBit)) {
+            const uint32_t limit = kEndBit - min(pos, kEndBit);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 alive = alive && (end[j] <= limit);
@@ -395,6 +405,96 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
         send_tile(7);
     }
     if (lane == 0) bulk_wait_all();                        // shared memory must outlive the engine's reads
+}
+
+// ---------------------------------------------------------------------------------------------
+// K1v: decompress of the variable-length container (groups back to back in one bit stream, start
+// index on the side; nothing clipped, nothing padded).  Same thread-per-group decode and the same
+// TMA tile store as K1; the difference is the front end: a lane copies the 16-byte chunks that
+// cover its group (on average 5) into its column of a 40-row transposed array, masks the bits
+// that belong to the next group, and starts decoding at bit (start mod 128).
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kVarRows = 40;                        // 10 chunks: 127 + 1046 bits at most, plus slack
+constexpr uint32_t kVarBitsBytes = kVarRows * 128;
+
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __restrict__ d_stream,
+                           const uint64_t* __restrict__ d_index, uint64_t n_groups, uint16_t* __restrict__ d_out,
+                           uint32_t active_warps, const __grid_constant__ CUtensorMap out_map)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t smem_base = smem_u32(smem);
+    constexpr uint32_t kStageBase = (kSmemWarpBase + kWarps * (kVarBitsBytes + kTabBytes) + 1023u) & ~1023u;
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * (kVarBitsBytes + kTabBytes) + lane * 4;
+    ws.tab = ws.bits + kVarBitsBytes;
+    ws.syms = 0;
+    for (uint32_t r = 0; r < kVarRows; ++r) sts_u32(ws.bits + r * 128, 0u);
+    const uint32_t stage = smem_base + kStageBase + warp * 1024;
+    const uint32_t swz = ((lane >> 2) & 1u) << 4;
+    const uint32_t my_row = stage + lane * 32;
+
+    const uint64_t total_bits = d_index[0];
+    const uint64_t stream_chunks = (total_bits + 127) >> 7;
+    const uint64_t* chunk_base = d_index + 1;
+    const uint32_t* off32 = reinterpret_cast<const uint32_t*>(d_index + 1 + var_chunks(n_groups));
+    auto start_of = [&](uint64_t g) { return g < n_groups ? chunk_base[g >> kVarChunkShift] + off32[g] : total_bits; };
+
+    const uint64_t n_tiles = (n_groups + 31) / 32;
+    const uint64_t tile_stride = active_warps;
+    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
+    if (tile >= tile_stride) tile = n_tiles;
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    uint32_t dirty_rows = 0;                               // rows of this lane's column that hold a previous group
+
+    for (; tile < n_tiles; tile += tile_stride) {
+        const uint64_t g = min(tile * 32 + lane, n_groups - 1);
+        const uint64_t start = min(start_of(g), total_bits);
+        const uint64_t end = max(min(start_of(g + 1), total_bits), start);   // the group sees [start, end), zeros after
+        const uint64_t c0 = start >> 7;
+        const uint32_t nc = static_cast<uint32_t>(min(static_cast<uint64_t>(kVarRows / 4), ((end + 127) >> 7) - c0));
+        for (uint32_t c = 0; c < nc; ++c) {
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (c0 + c < stream_chunks) asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d_stream + c0 + c));
+            uint32_t w[4] = {v.x, v.y, v.z, v.w};
+            const uint64_t first = (c0 + c) << 7;          // stream bit of w[0] bit 0
+            if (first + 128 > end) {                       // bits of the next group read as zero
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const uint64_t wb = first + 32 * k;
+                    w[k] = wb >= end ? 0u : (end - wb >= 32 ? w[k] : (w[k] & ((1u << static_cast<uint32_t>(end - wb)) - 1u)));
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sts_u32(ws.bits + (4 * c + k) * 128, w[k]);
+        }
+        for (uint32_t r = 4 * nc; r < dirty_rows; ++r) sts_u32(ws.bits + r * 128, 0u);
+        dirty_rows = 4 * nc;
+        const uint32_t first_bit = static_cast<uint32_t>(start & 127u);
+        const uint32_t hw = first_bit >> 5;
+        const uint32_t hdr = __funnelshift_r(lds_u32(ws.bits + hw * 128), lds_u32(ws.bits + hw * 128 + 128), first_bit);
+        const GroupHeader h = open_header<false>(hdr, first_bit, smem_base, ws, T);
+        const int row0 = static_cast<int>(tile * 32);
+        uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        decode_symbols<true, kVarRows - 2, kVarRows * 32>(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
+            const int slot = (n & 15) >> 1;
+            if (n & 1) r[slot] |= v << 16; else r[slot] = v;
+            if ((n & 15) == 15) {
+                if (lane == 0) bulk_wait_read0();          // the engine has read the previous tile
+                __syncwarp();
+                sts_v4(my_row + swz, r[0], r[1], r[2], r[3]);
+                sts_v4(my_row + (swz ^ 16u), r[4], r[5], r[6], r[7]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) { tma_store_2d(&out_map, stage, (n >> 4) * 16, row0); bulk_commit(); }
+            }
+        });
+    }
+    if (lane == 0) bulk_wait_all();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1209,6 +1309,40 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     kernel<<<grid, kDecompressWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out),
         balanced_warps((n_groups + 31) / 32, grid * kDecompressWarps));
+    return check_launch();
+}
+
+constexpr int kVarWarps = 18;
+
+extern "C" int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, const void* d_index, uint64_t n_groups, void* d_out,
+                                   void* stream)
+{
+    if (n_groups == 0) return ECCO_OK;
+    if (!d_meta || !d_stream || !d_index || !d_out) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_stream) || !aligned16(d_out) || (reinterpret_cast<uintptr_t>(d_index) & 7u)) return ECCO_ERR_ALIGNMENT;
+    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    // the tile store needs 32 rows: pad the logical row count of tiny tensors is not possible, so they are refused
+    CUtensorMap map;
+    if (!make_out_map(&map, d_out, n_groups)) return ECCO_ERR_CUDA;
+    auto kernel = ecco_var_decompress_kernel<kVarWarps>;
+    constexpr size_t smem =
+        ((kSmemWarpBase + static_cast<size_t>(kVarWarps) * (kVarBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
+        static_cast<size_t>(kVarWarps) * 1024;
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    const uint64_t cta_tiles = (n_groups + kVarWarps * 32 - 1) / (kVarWarps * 32);
+    const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
+    const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kVarWarps);
+    kernel<<<grid, kVarWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const uint8_t*>(d_meta), reinterpret_cast<const uint4*>(d_stream), static_cast<const uint64_t*>(d_index),
+        n_groups, static_cast<uint16_t*>(d_out), active, map);
     return check_launch();
 }
 

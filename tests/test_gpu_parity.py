@@ -496,3 +496,68 @@ def test_kv_compress_full_size_round_trip(B, eo, W, synth):
     (t,) = W.config3(which=("K",), keep_source=True)
     got = gpu_kv_compress(B, t.meta, t.source)
     assert_blocks_equal(got, t.blocks)
+
+
+# ------------------------------------------------------------------ variable-length container
+def oracle_offsets_from_index(index, n):
+    nc = (n + 4095) // 4096
+    idx64 = index[: 8 * (1 + nc)].view(np.uint64)
+    off32 = index[8 * (1 + nc): 8 * (1 + nc) + 4 * n].view(np.uint32)
+    return np.concatenate([idx64[1:][np.arange(n) >> 12] + off32, idx64[:1]]).astype(np.uint64)
+
+
+def gpu_var_decompress(B, lmeta, stream, index, n):
+    d_out = torch.full((n, 128), float("nan"), dtype=torch.float16, device="cuda")
+    B.ecco_var_decompress(B.meta_to_device(lmeta), dev(stream), dev(index), n, d_out)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    return d_out.cpu().numpy()
+
+
+@pytest.mark.parametrize("n_groups", [1, 31, 33, 1000, 2048])
+def test_var_decompress_matches_oracle(B, eo, cfg1_small, n_groups):
+    meta = cfg1_small["meta"]
+    lm = lib_meta_from_oracle(B, meta)
+    x = cfg1_small["w"].reshape(-1, 128)[:n_groups]
+    stream, index, total = B.ecco_var_encode_host(lm, x, B.SELECT_MSE | B.KEEP_EXPONENT)
+    got = gpu_var_decompress(B, lm, stream, index, n_groups)
+    assert_bit_exact(got, eo.var_decode(meta, stream, oracle_offsets_from_index(index, n_groups)))
+
+
+def test_var_decompress_is_total_on_garbage(B, eo, cfg1_small, synth):
+    """Random stream bytes with a valid-looking but arbitrary index: overlapping, empty and over-long groups."""
+    meta = cfg1_small["meta"]
+    lm = lib_meta_from_oracle(B, meta)
+    n = 4096 + 100
+    rng = np.random.Generator(np.random.PCG64(12))
+    stream = synth.random_blocks(4096, 5).reshape(-1)                      # 256 KiB of noise, a multiple of 16
+    total = stream.size * 8 - 37
+    starts = np.sort(rng.integers(0, total, n)).astype(np.uint64)
+    starts[5] = starts[4]                                                   # empty group
+    nc = (n + 4095) // 4096
+    index = np.zeros((8 * (1 + nc) + 4 * n + 15) // 16 * 16, dtype=np.uint8)
+    idx64 = index[: 8 * (1 + nc)].view(np.uint64)
+    idx64[0] = total
+    for c in range(nc):
+        idx64[1 + c] = starts[c * 4096]
+    index[8 * (1 + nc): 8 * (1 + nc) + 4 * n].view(np.uint32)[:] = (starts - idx64[1:][np.arange(n) >> 12]).astype(np.uint32)
+    got = gpu_var_decompress(B, lm, stream, index, n)
+    assert_bit_exact(got, eo.var_decode(meta, stream, np.concatenate([starts, [np.uint64(total)]]).astype(np.uint64)))
+
+
+def test_var_decompress_config2_gate_full_size(B, eo, W, synth):
+    (t,) = W.config2(names=("gate",), keep_source=True)
+    stream, index, total = B.ecco_var_encode_host(t.meta, t.source, B.SELECT_MSE | B.KEEP_EXPONENT)
+    n = t.n_groups
+    d_out = torch.empty((n, 128), dtype=torch.float16, device="cuda")
+    B.ecco_var_decompress(B.meta_to_device(t.meta), dev(stream), dev(index), n, d_out)
+    torch.cuda.synchronize()
+    om = oracle_meta_from_lib(eo, t.meta)
+    offs = oracle_offsets_from_index(index, n)
+    # sampled runs of consecutive groups (the oracle needs each group's end = the next group's start)
+    rng = np.random.Generator(np.random.PCG64(2))
+    for g0 in [0, n - 512] + [int(v) for v in rng.integers(0, n - 512, 6)]:
+        want = eo.var_decode(om, stream, np.concatenate([offs[g0:g0 + 512], offs[g0 + 512:g0 + 513]]))
+        assert_bit_exact(d_out[g0:g0 + 512].cpu().numpy(), want)
+    assert bool(torch.isfinite(d_out).all())
+    assert total / n < 512                                                  # on average the stream is shorter than the blocks

@@ -191,3 +191,34 @@ def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
             pos += t >> 4
             n += 1
         assert n == info.n_fit and pos == info.end_bit
+
+
+def test_variable_length_host_encoder_matches_oracle(binding, eo, cfg1_small, kv_small):
+    for fx, key, flags in ((cfg1_small, "w", binding.SELECT_MSE), (kv_small, "k", binding.SELECT_MINMAX | binding.KEEP_EXPONENT)):
+        ometa, x = fx["meta"], fx[key]
+        lm = lib_meta_from_oracle(binding, ometa)
+        stream, index, total = binding.ecco_var_encode_host(lm, x, flags)
+        want_stream, want_off = eo.var_encode(ometa, x, flags & 1)
+        n = x.size // 128
+        assert total == int(want_off[n]) and stream.size % 16 == 0
+        assert np.array_equal(stream[: want_stream.size], want_stream) and not stream[want_stream.size:].any()
+        idx64 = index[: 8 * (1 + (n + 4095) // 4096)].view(np.uint64)
+        off32 = index[8 * (1 + (n + 4095) // 4096): 8 * (1 + (n + 4095) // 4096) + 4 * n].view(np.uint32)
+        assert idx64[0] == total
+        starts = idx64[1:][np.arange(n) >> 12] + off32
+        assert np.array_equal(starts, want_off[:n])
+        # no clipping: positions the fixed block had to drop (decoded as +0 there) carry their mapped value here
+        out = eo.var_decode(ometa, want_stream, want_off)
+        groups = x.reshape(-1, 128)
+        seen = 0
+        for g in range(0, n, 7):
+            _, _, info = eo.decode_block(ometa, fx["blocks"][g])
+            if info.n_fit < 128:
+                q = eo.quantize_group(ometa, groups[g], flags & 1)
+                tail = out[g, info.n_fit:].astype(np.float32)
+                pat = ometa.patterns()[q["kp"]].astype(np.float32)
+                s = np.float32(abs(eo.e4m3_to_f32(q["qs"]))) * np.float32(2.0 ** ometa.e)
+                want = np.array([pat[sy] * s if sy < 15 else eo.e4m3_to_f32(q["qs"]) * 2.0 ** ometa.e for sy in q["sym"][info.n_fit:]])
+                assert np.array_equal(tail, want.astype(np.float16).astype(np.float32))
+                seen += 1
+        assert seen > 3

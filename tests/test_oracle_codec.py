@@ -310,3 +310,41 @@ def test_attention_output_reduces_to_textbook_softmax_times_v(eo, kv_small, synt
     scores[:, :, 17] = 0.0
     out, _ = eo.attn_values(km, kb, 2, 4, 256, 2, scores)
     assert np.allclose(out.reshape(2, 4, 2, 128), V[:, :, 17][:, :, None, :], rtol=1e-12)
+
+
+def test_variable_length_container_round_trip(eo, cfg1_small):
+    """No clipping, no padding: every group decodes to exactly the mapped values of its 128 symbols, the
+    stream is the concatenation of the groups' bit strings, and groups that fit a block agree with it."""
+    meta, w = cfg1_small["meta"], cfg1_small["w"]
+    stream, off = eo.var_encode(meta, w[:64], eo.SELECT_MSE)
+    n = 64 * 1024 // 128
+    assert off.size == n + 1 and off[0] == 0 and np.all(np.diff(off.astype(np.int64)) >= 10 + 1 + 256)
+    out = eo.var_decode(meta, stream, off)
+    cb, kl, pats = meta.cb_lengths(), meta.kp_lengths(), meta.patterns().astype(np.float32)
+    T = np.float32(2.0 ** meta.e)
+    blocks = cfg1_small["blocks"]
+    n_unclipped = 0
+    for g in range(n):
+        q = eo.quantize_group(meta, w.reshape(-1, 128)[g], eo.SELECT_MSE)
+        totals = cb[q["kp"]][:, q["sym"]].astype(np.int64).sum(axis=1)
+        hf = int(totals.argmin())
+        assert int(off[g + 1] - off[g]) == 10 + int(kl[q["kp"]]) + int(totals[hf])          # bit-exact length
+        s = np.float32(abs(eo.e4m3_to_f32(q["qs"]))) * T
+        want = np.array([np.float16(np.float32(eo.e4m3_to_f32(q["qs"])) * T) if sy == 15 else np.float16(pats[q["kp"]][sy] * s)
+                         for sy in q["sym"]], dtype=np.float16)
+        assert np.array_equal(out[g].view(np.uint16), want.view(np.uint16))
+        # the group's bits are the block's bits when the block was neither clipped nor padded past them
+        _, _, info = eo.decode_block(meta, blocks[g])
+        if info.n_fit == 128:
+            n_unclipped += 1
+            L = int(off[g + 1] - off[g])
+            bits_blk = int.from_bytes(blocks[g].tobytes(), "little") & ((1 << L) - 1)
+            big = int.from_bytes(stream[int(off[g]) // 8: int(off[g]) // 8 + 140].tobytes(), "little") >> (int(off[g]) % 8)
+            assert big & ((1 << L) - 1) == bits_blk
+    assert n_unclipped > n // 2
+    # totality: garbage stream, arbitrary (even overlapping) offsets
+    rng = np.random.Generator(np.random.PCG64(3))
+    junk = rng.integers(0, 256, 4096, dtype=np.uint8)
+    joff = np.sort(rng.integers(0, 4096 * 8, 33)).astype(np.uint64)
+    joff[-1] = 4096 * 8
+    assert np.isfinite(eo.var_decode(meta, junk, joff).astype(np.float32)).all()
