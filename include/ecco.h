@@ -140,7 +140,7 @@ int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_
  * of ECCO_STATIC_WORKSPACE_BYTES inside the library's device image (every GPU that loads the
  * library carries it until the process exits) instead of a caller buffer.  The call allocates
  * nothing.  A shape whose plan needs more scratch than that is refused with ECCO_ERR_WORKSPACE
- * before anything is launched (for scale: batch 8 on an 11008 x 4096 matrix needs about 3.7 MB).
+ * before anything is launched (for scale: batch 8 on an 11008 x 4096 matrix needs about 3.3 MB).
  * The first call on each device looks up the array's device address (with that device current);
  * make that first call outside any stream capture.  All calls on a device share the one array:
  * it still holds the previous call's values when the next call starts (each call clears the part

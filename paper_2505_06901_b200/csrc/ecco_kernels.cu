@@ -608,112 +608,14 @@ __device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
     return ws;
 }
 
-// K2: y[b][n] = sum_k W~[n][k] x[b][k].  A work unit is (row tile of kWarps*32 rows, one k-block);
-// units are numbered row tile major and dealt to the persistent CTAs in contiguous runs, so a
-// thread (= one row) keeps its partial sums in registers across the k-blocks of its run.  When a
-// row tile is shared by several CTAs each writes its partial sums to its own workspace slot and
-// the last to arrive (ticket counter) adds the slots in CTA order: the result does not depend on
-// scheduling.  Workspace: partial[slot][kV][rows per tile] floats, then one ticket per row tile.
-template <int kV, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
-ecco_gemv_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                 const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
-                 unsigned int* __restrict__ d_tickets)
-{
-    extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    __shared__ unsigned int ticket;
-    constexpr int kRows = kWarps * 32;
-    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
-    constexpr uint32_t kXsBytes = kGroup * kV * 4;
-    const uint32_t smem_base = smem_u32(smem);
-    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
-    float* xs_ptr = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);   // two slices
-    const uint32_t xs_base = smem_u32(xs_ptr);
-
-    const int G = gridDim.x, c = blockIdx.x;
-    const int row_tiles = (n_out + kRows - 1) / kRows;
-    const int64_t U = static_cast<int64_t>(row_tiles) * kblocks;
-    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
-    const int k = kblocks * kGroup;
-    const int tid = static_cast<int>(threadIdx.x);
-
-    // rows past the end of the matrix decode the last row again and store nothing
-    auto block_ptr = [&](int64_t u) {
-        const int rt = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
-        const int row = min(rt * kRows + tid, n_out - 1);
-        return d_blocks + (static_cast<uint64_t>(row) * kblocks + kb) * kBlockBytes;
-    };
-    Block blk;
-    if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!stage_tables(smem, d_meta, &bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
-
-    Accum<kV> acc;
-    acc.clear();
-    auto flush = [&](int rt) {
-        const int row = rt * kRows + tid;
-        const bool row_ok = row < n_out;
-        const int c_lo = unit_owner(U, G, static_cast<int64_t>(rt) * kblocks);
-        const int c_hi = unit_owner(U, G, static_cast<int64_t>(rt + 1) * kblocks - 1);
-        if (c_lo == c_hi) {                                // this CTA owns the whole row tile
-            if (row_ok) {
-#pragma unroll
-                for (int b = 0; b < kV; ++b)
-                    if (b < batch) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
-            }
-            return;
-        }
-        // staircase of (CTA, row tile) pairs: slot = c + rt is unique
-        float* mine = d_partial + static_cast<size_t>(c + rt) * kV * kRows;
-#pragma unroll
-        for (int b = 0; b < kV; ++b) mine[b * kRows + tid] = acc.a[b];
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) ticket = atomicAdd(&d_tickets[rt], 1u);
-        __syncthreads();
-        if (ticket == static_cast<unsigned int>(c_hi - c_lo)) {   // last of the CTAs that share this row tile
-            __threadfence();
-            if (row_ok) {
-#pragma unroll
-                for (int b = 0; b < kV; ++b) {
-                    if (b >= batch) continue;
-                    float sum = 0.0f;
-                    for (int cc = c_lo; cc <= c_hi; ++cc)
-                        sum += __ldcg(d_partial + (static_cast<size_t>(cc + rt) * kV + b) * kRows + tid);
-                    d_y[static_cast<size_t>(b) * n_out + row] = sum;
-                }
-            }
-            if (tid == 0) d_tickets[rt] = 0;               // ready for the next call on this workspace
-        }
-        __syncthreads();                                   // `ticket` may be rewritten by the next flush
-    };
-
-    int cur_rt = static_cast<int>(u0 / kblocks);
-    for (int64_t u = u0; u < u1; ++u) {
-        const int rt = static_cast<int>(u / kblocks), kb = static_cast<int>(u % kblocks);
-        if (rt != cur_rt) { flush(cur_rt); acc.clear(); cur_rt = rt; }
-        // stage x[b][kb*128 .. +128) as fp32 xs[i][b] (rows beyond `batch` are zero)
-        const int buf = static_cast<int>((u - u0) & 1);
-        float* xs = xs_ptr + buf * (kGroup * kV);
-        for (int i = tid; i < kGroup * kV; i += kRows) {
-            const int b = i % kV, e = i / kV;
-            xs[i] = (b < batch) ? __half2float(d_x[static_cast<size_t>(b) * k + kb * kGroup + e]) : 0.0f;
-        }
-        __syncthreads();                                   // slice visible; the other slice is free again
-        const Block cur = blk;
-        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
-        fused_group<kV>(cur, smem_base, ws, T, xs_base + buf * kXsBytes, acc);
-    }
-    if (u0 < u1) flush(cur_rt);
-}
-
 // K2 for one or two rows of x: the slice is small enough (512 B or 1 KB) for every warp to keep
 // its own, so warps never meet at a barrier.  A work unit is (32 consecutive rows, one k-block),
-// numbered row-tile major; every warp of the grid owns a contiguous run of units, keeps its rows'
-// partial sums in registers along k, and shares a row tile with the neighbouring warps through
-// the same slot-and-ticket scheme as above (slot = global warp id + row tile, 32 floats per row
-// of x).  Workspace: partial[slot][kV][32] floats, then one ticket per 32-row tile.
+// numbered row-tile major; every working warp owns a contiguous run of units and keeps its rows'
+// partial sums in registers along k.  When a row tile is shared by several warps each writes its
+// partial sums to its own workspace slot (slot = global warp id + row tile: unique along the
+// staircase of (warp, tile) pairs) and the last to arrive (ticket counter) adds the slots in warp
+// order: the result does not depend on scheduling.  Workspace: partial[slot][kV][32] floats, then
+// one ticket per 32-row tile.
 template <int kV, int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
@@ -1124,6 +1026,247 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
 }
 
 // ---------------------------------------------------------------------------------------------
+// K2m / K3m: the fused consumers for 3 to 8 dot products per group (rows of x, query heads) on the
+// tensor cores.  With eight products per weight the scalar path spends four shared-memory
+// wavefronts and eight FMAs per symbol on the vector operand alone.  Here a group is decoded in
+// two passes as in K5 (indices first; then per 16 values: map, stage a [32 rows][16 k] fp16 tile,
+// patch its outliers) and each tile is contracted against the fp16 vector fragments, which stay
+// in registers for the whole group: C[32 rows][8] += tile[32 x 16] * V[16 x 8], two
+// mma.m16n8k16 per tile, fp32 accumulate (fp16 x fp16 products are exact in fp32).  A warp is
+// independent of the others: no vector slice in shared memory, no block barrier.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
+}
+
+// Position i (0..15) of a 16-value chunk is staged in tile column 2q + (j & 1) + 8 (j >> 1) with i = 4q + j.  The
+// contraction index of an MMA may be permuted freely as long as both operands agree, and with this
+// order the four vector elements a lane needs per chunk (columns 2q, 2q+1, 2q+8, 2q+9) are the
+// contiguous k = 4q .. 4q+3: one 8-byte load instead of two 4-byte ones.
+__host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i & 1) + 8 * ((i >> 1) & 1); }
+
+// vfrag[2c], vfrag[2c+1]: B fragments of chunk c (tile columns (lane%4)*2 + {0,1}, and + 8), vector lane/4
+// acc[0] / acc[1]: C fragments of rows 0..15 / 16..31 of the warp's 32 groups
+__device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base, const WarpSmem& ws, uint32_t stage, float T,
+                                            bool valid, const uint32_t (&vfrag)[16], float (&acc)[2][4])
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = stage + lane * 32;
+    const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
+    uint32_t packed = 0;
+    int n_fit = kGroup;
+    const uint32_t end = decode_symbols<false>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+        if (!alive) n_fit = min(n_fit, n);
+        packed |= sym << ((n & 7) * 4);
+        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+    });
+    if (!valid) n_fit = 0;                                 // rows past the end contribute zeros
+    const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
+    uint64_t pads_lo = 0, pads_hi = 0;                     // 16 bits per chunk: which pads fall into it
+    for (int j = 0; j < n_pad; ++j) {
+        const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
+        const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
+        if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+    }
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        uint32_t r8[8];
+        const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
+        const bool whole = ch * 16 + 16 <= n_fit;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
+            uint32_t v = lds_u32(ws.tab + sym * 128);
+            if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;
+            const int col = tile_column(i);                // see load_vfrag
+            if (col & 1) r8[col >> 1] |= v << 16; else r8[col >> 1] = v;
+        }
+        __syncwarp();                                      // the previous tile has been read
+        sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
+        sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
+        uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
+        while (mine) {                                     // ascending: a later pad overrides an earlier one
+            const int j = __ffs(static_cast<int>(mine)) - 1;
+            mine &= mine - 1;
+            const uint32_t f = read_pad(ws, j);
+            const uint32_t byte = static_cast<uint32_t>(tile_column(static_cast<int>(f & 15u))) * 2;
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
+                         "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
+        }
+        __syncwarp();                                      // tile complete
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const uint32_t row = ((lane >> 3) & 1u) * 8 + (lane & 7u) + 16 * mt, half = lane >> 4;
+            uint32_t a[4];
+            ldmatrix_x4(a, stage + row * 32 + ((half ^ ((row >> 2) & 1u)) << 4));
+            mma_16816(acc[mt], a, vfrag[2 * ch], vfrag[2 * ch + 1]);
+        }
+    }
+}
+
+// fragments of eight fp16 vectors v[col][k0 .. k0+127] (col = lane/4; columns >= n_cols are zero)
+__device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols)
+{
+    const int lane = static_cast<int>(threadIdx.x & 31u), col = lane >> 2;
+    const uint2* p = reinterpret_cast<const uint2*>(base + static_cast<size_t>(min(col, n_cols - 1)) * col_stride) + (lane & 3);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint2 v = col < n_cols ? __ldg(p + c * 4) : make_uint2(0u, 0u);     // k = 16c + 4 (lane%4) .. + 3
+        vfrag[2 * c] = v.x;                                // tile columns 2q, 2q+1
+        vfrag[2 * c + 1] = v.y;                            // tile columns 2q+8, 2q+9
+    }
+}
+
+// K2m: y[b][n] = sum_k W~[n][k] x[b][k] for 3..8 rows of x.  Units, ownership and the slot-and-ticket
+// reduction are those of the per-warp kernel (unit = 32 rows x one k-block).
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                     const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+                     unsigned int* __restrict__ d_tickets, int active_warps)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t smem_base = smem_u32(smem);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int tiles = (n_out + 31) / 32;
+    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    const int W = active_warps;
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    const int k = kblocks * kGroup;
+    auto block_ptr = [&](int64_t u) {
+        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
+        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
+    };
+    Block blk;
+    uint32_t vnext[16];
+    if (u0 < u1) { ldg_block(blk, block_ptr(u0)); load_vfrag(vnext, d_x + static_cast<int>(u0 % kblocks) * kGroup, k, batch); }
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // C fragment element (mt, i): row = 16 mt + lane/4 + 8 (i >= 2), column b = (lane%4)*2 + (i & 1)
+    auto flush = [&](int tile) {
+        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
+        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
+        float* mine = d_partial + static_cast<size_t>(wg + tile) * 8 * 32;
+        if (w_lo != w_hi) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    mine[((lane & 3) * 2 + (i & 1)) * 32 + 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0)] = acc[mt][i];
+            __threadfence();
+            __syncwarp();
+            unsigned int t = 0;
+            if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            if (t != static_cast<unsigned int>(w_hi - w_lo)) return;
+            __threadfence();
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0), b = (lane & 3) * 2 + (i & 1);
+                const int row = tile * 32 + r;
+                float sum = acc[mt][i];
+                if (w_lo != w_hi) {                        // slots in warp order, whatever the arrival order
+                    sum = 0.0f;
+                    for (int ww = w_lo; ww <= w_hi; ++ww) sum += __ldcg(d_partial + (static_cast<size_t>(ww + tile) * 8 + b) * 32 + r);
+                }
+                if (row < n_out && b < batch) d_y[static_cast<size_t>(b) * n_out + row] = sum;
+            }
+        if (w_lo != w_hi && lane == 0) d_tickets[tile] = 0;
+    };
+
+    int cur_tile = static_cast<int>(u0 / kblocks);
+    for (int64_t u = u0; u < u1; ++u) {
+        const int tile = static_cast<int>(u / kblocks);
+        if (tile != cur_tile) {
+            flush(cur_tile);
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.0f;
+            cur_tile = tile;
+        }
+        const Block cur = blk;
+        uint32_t vfrag[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) vfrag[i] = vnext[i];
+        if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_vfrag(vnext, d_x + static_cast<int>((u + 1) % kblocks) * kGroup, k, batch); }
+        row_dot_mma(cur, smem_base, ws, stage, T, tile * 32 + lane < n_out, vfrag, acc);
+    }
+    if (u0 < u1) flush(cur_tile);
+}
+
+// K3m: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for 3..8 query heads per KV head.
+// Unit = (one (batch, kv head), 32 tokens); every working warp owns a contiguous run of units.
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
+                            int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores,
+                            int active_warps)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t smem_base = smem_u32(smem);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int tiles = (seq + 31) / 32;
+    const int64_t U = static_cast<int64_t>(heads) * tiles;
+    const int W = active_warps;
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    auto block_ptr = [&](int64_t u) {
+        const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    };
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!stage_tables(smem, d_meta, &bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    uint32_t vfrag[16];
+    int cur_bh = -1;
+    for (int64_t u = u0; u < u1; ++u) {
+        const int bh = static_cast<int>(u / tiles), t0 = static_cast<int>(u % tiles) * 32;
+        if (bh != cur_bh) { load_vfrag(vfrag, d_q + static_cast<size_t>(bh) * q_per_kv * kGroup, kGroup, q_per_kv); cur_bh = bh; }
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        row_dot_mma(cur, smem_base, ws, stage, T, t0 + lane < seq, vfrag, acc);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = t0 + 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0), r = (lane & 3) * 2 + (i & 1);
+                if (t < seq && r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = scale * acc[mt][i];
+            }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // host-side launch helpers
 // ---------------------------------------------------------------------------------------------
 // number of working warps <= w_max such that `units` split evenly: all get ceil(units / w_max) or one less
@@ -1176,28 +1319,12 @@ int check_launch()
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 constexpr int kDecompressWarps = 32;
-// warps per CTA of the fused kernels: as many as shared memory allows; 20 for eight dot products
-// per group, whose accumulators need the larger register budget (96 instead of 80 per thread)
-constexpr int fused_warps(int kV) { return kV >= 8 ? 20 : 22; }
+// warps per CTA of the scalar fused kernels (one or two dot products per group): as many as shared memory allows
+constexpr int fused_warps(int) { return 22; }
 // per-warp GEMV: every warp also carries its own slice of x, which leaves room for 22 / 20 warps
 constexpr int gemv_warp_warps(int kV) { return kV >= 2 ? 20 : 22; }
 
-// GEMV launch plan: one persistent CTA per SM (fewer if there are fewer work units), workspace of
-// (CTAs + row tiles) partial slots and one ticket per row tile.
 struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
-
-GemvPlan gemv_plan(int n_out, int kblocks, int vpad, int ctas_max)
-{
-    GemvPlan p;
-    const int kFusedRows = fused_warps(vpad) * 32;
-    p.row_tiles = (n_out + kFusedRows - 1) / kFusedRows;
-    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
-    p.grid = static_cast<int>(balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(ctas_max)));   // same units per CTA
-    p.partial_bytes = static_cast<size_t>(p.grid + p.row_tiles) * vpad * kFusedRows * sizeof(float);
-    p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
-    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
-    return p;
-}
 
 // plan of the per-warp GEMV (one or two rows of x)
 GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
@@ -1209,6 +1336,21 @@ GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
     p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
     p.partial_bytes = static_cast<size_t>(p.grid * gemv_warp_warps(vpad) + p.row_tiles) * vpad * 32 * sizeof(float);
     p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return p;
+}
+
+constexpr int kMmaWarps = 20;
+
+// plan of the tensor-core GEMV (3..8 rows of x): units and slots as in the per-warp kernel, eight columns
+GemvPlan gemv_mma_plan(int n_out, int kblocks, int ctas_max)
+{
+    GemvPlan p;
+    p.row_tiles = (n_out + 31) / 32;
+    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
+    const int64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
+    p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
+    p.partial_bytes = (static_cast<size_t>(p.grid * kMmaWarps + p.row_tiles) * 8 * 32 * sizeof(float) + 255) & ~static_cast<size_t>(255);
     p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
     return p;
 }
@@ -1350,34 +1492,32 @@ extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t ba
 {
     if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return 0;
     // sized for the largest plan any supported device can ask for (at most 256 persistent CTAs)
-    const GemvPlan p = pad_v(batch) <= 2 ? gemv_warp_plan(n_out, k / kGroup, pad_v(batch), 256)
-                                         : gemv_plan(n_out, k / kGroup, pad_v(batch), 256);
+    const GemvPlan p = pad_v(batch) <= 2 ? gemv_warp_plan(n_out, k / kGroup, pad_v(batch), 256) : gemv_mma_plan(n_out, k / kGroup, 256);
     return p.partial_bytes + p.ticket_bytes;
 }
 
-template <int kV>
-static int launch_gemv(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
-                       const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+// three to eight rows of x: the tensor-core kernel
+static int launch_gemv_mma(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
+                           const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
-    constexpr int kFusedWarps = fused_warps(kV);
-    auto kernel = ecco_gemv_kernel<kV, kFusedWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + 2 * kGroup * kV * 4;
+    auto kernel = ecco_gemv_mma_kernel<kMmaWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kMmaWarps) * kMmaWarpBytes;
     static thread_local bool configured[64] = {};
     if (!configured[di.device]) {
         int rc = set_smem(kernel, smem);
         if (rc) return rc;
         configured[di.device] = true;
     }
-    const GemvPlan p = gemv_plan(n_out, kblocks, kV, di.sms < 256 ? di.sms : 256);
+    const GemvPlan p = gemv_mma_plan(n_out, kblocks, di.sms < 256 ? di.sms : 256);
     if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-    // the workspace's previous contents are irrelevant: tickets start from zero on every call
     cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
     if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
-    kernel<<<p.grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
-                                                       static_cast<const __half*>(d_x), batch, d_y, partial, tickets);
+    const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kMmaWarps));
+    kernel<<<p.grid, kMmaWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
+                                                     static_cast<const __half*>(d_x), batch, d_y, partial, tickets, active);
     return check_launch();
 }
 
@@ -1422,8 +1562,7 @@ extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_
     switch (pad_v(batch)) {
         case 1: return launch_gemv_warp<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
         case 2: return launch_gemv_warp<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
-        case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
-        default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+        default: return launch_gemv_mma(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
     }
 }
 
@@ -1447,7 +1586,7 @@ extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, 
     const int kblocks = k / kGroup, vpad = pad_v(batch);
     // refuse, before any launch, a shape whose plan does not fit the fixed array
     const int ctas = di.sms < 256 ? di.sms : 256;
-    const GemvPlan p = vpad <= 2 ? gemv_warp_plan(n_out, kblocks, vpad, ctas) : gemv_plan(n_out, kblocks, vpad, ctas);
+    const GemvPlan p = vpad <= 2 ? gemv_warp_plan(n_out, kblocks, vpad, ctas) : gemv_mma_plan(n_out, kblocks, ctas);
     if (p.partial_bytes + p.ticket_bytes > ECCO_STATIC_WORKSPACE_BYTES) return ECCO_ERR_WORKSPACE;
     // one-time set-up per device (the current device is di.device): resolve the array's address
     static std::mutex mu;
@@ -1467,8 +1606,7 @@ extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, 
     switch (vpad) {
         case 1: return launch_gemv_warp<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
         case 2: return launch_gemv_warp<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
-        case 4: return launch_gemv<4>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
-        default: return launch_gemv<8>(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
+        default: return launch_gemv_mma(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, ws, ECCO_STATIC_WORKSPACE_BYTES, s);
     }
 }
 
@@ -1508,8 +1646,23 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
     switch (pad_v(q_per_kv)) {
         case 1: return launch_attn<1>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
         case 2: return launch_attn<2>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
-        case 4: return launch_attn<4>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
-        default: return launch_attn<8>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
+        default: {
+            auto kernel = ecco_attn_scores_mma_kernel<kMmaWarps>;
+            const size_t smem = kSmemWarpBase + static_cast<size_t>(kMmaWarps) * kMmaWarpBytes;
+            static thread_local bool configured[64] = {};
+            if (!configured[di.device]) {
+                rc = set_smem(kernel, smem);
+                if (rc) return rc;
+                configured[di.device] = true;
+            }
+            const uint64_t units = static_cast<uint64_t>(batch) * n_kv_heads * ((seq + 31) / 32);
+            const uint64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
+            const unsigned grid = static_cast<unsigned>(ctas < static_cast<uint64_t>(di.sms) ? ctas : di.sms);
+            const int active = static_cast<int>(balanced_warps(units, grid * kMmaWarps));
+            kernel<<<grid, kMmaWarps * 32, smem, s>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, batch * n_kv_heads, seq, q_per_kv,
+                                                      static_cast<const __half*>(d_q), scale, d_scores, active);
+            return check_launch();
+        }
     }
 }
 
