@@ -22,7 +22,7 @@ constexpr int kExpMin = -32, kExpMax = 16;
 // Device image of the per-tensor metadata.  The tables follow the 64-byte header back to back
 // so that one bulk copy brings them into shared memory.
 constexpr uint32_t kDevMagic = 0x4F434345u;  // "ECCO"
-constexpr uint32_t kDevVersion = 2;
+constexpr uint32_t kDevVersion = 3;
 struct DevHeader {
     uint32_t magic, version;
     int32_t S, H, e;
@@ -44,8 +44,27 @@ constexpr uint32_t kOffEncCb = kOffSymLut + kSymLutBytes;             // [256][1
 constexpr uint32_t kEncCbBytes = kMaxPatterns * kCodebooks * kSymbols * 2;
 constexpr uint32_t kOffEncKp = kOffEncCb + kEncCbBytes;               // [64] u16: stream-order ID_KP codeword | length << 12
 constexpr uint32_t kEncKpBytes = kMaxPatterns * 2;
-constexpr uint32_t kDevBytes = kOffEncKp + kEncKpBytes;               // 84160
 constexpr uint32_t kEncBytes = kEncCbBytes + kEncKpBytes;             // 8320, a multiple of 16
+// Tables of the decompress kernel's mixed decoder (table lookups and arithmetic decoding of the canonical
+// code take turns, so that neither the load/store pipe nor the integer pipe carries every symbol).
+// Both work on the symbol's RANK, a relabelling of the 16 symbols per codebook:
+//   rank(s) = (position of s in (length, id) order + rho) mod 16, rho such that an 8-bit codeword's rank is
+//   its own low four bits (rho = 0 without 8-bit codewords).
+// Then rank = (codeword + delta[L]) mod 16 for a codeword of length L, with delta[8] = 0.
+constexpr uint32_t kOffRankLut = kOffEncKp + kEncKpBytes;             // 84160: [256][256] u8: len << 4 | rank, rotated like the symbol tables
+constexpr uint32_t kRankLutBytes = kSymLutBytes;
+constexpr uint32_t kOffArith = kOffRankLut + kRankLutBytes;           // [5][256] u32, one row per word, column = codebook:
+constexpr int kArithWords = 5;                                        //   0, 1: addends of the length compare (see below)
+constexpr uint32_t kArithBytes = kArithWords * kMaxPatterns * kCodebooks * 4;   //   2: delta[2..7], 4 bits each, delta[L] in bits 4(L-2)
+constexpr uint32_t kDevBytes = kOffArith + kArithBytes;               //   3, 4: rank of symbol s in bits 4s of the 64-bit pair
+// Length compare: with b = the next 8 stream bits, first bit on top, and thr[L] = the smallest b whose codeword
+// is longer than L (256 if none), field i of word 0 (bits 10 i ..) holds 256 - thr[2 + i] and field i of word 1
+// (bits 10 i + 1 .., one bit higher so that the two words' result bits do not meet) holds 256 - thr[5 + i],
+// i = 0..2; word 0 also has bits 30 and 31 set.  b * kArithSpread + word 0 and b * 2 kArithSpread + word 1 put
+// b + 256 - thr in every field, whose bit 8 says b >= thr; the codeword length is the number of set bits under
+// kArithGuard | bits 30, 31 of the first and 2 kArithGuard of the second, i.e. 2 + the number of thresholds passed.
+constexpr uint32_t kArithSpread = 1u | (1u << 10) | (1u << 20);
+constexpr uint32_t kArithGuard = (0x100u) | (0x100u << 10) | (0x100u << 20);
 // Both lookup tables are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.
 //

@@ -909,6 +909,53 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
             uint8_t* t = sl + (static_cast<size_t>(k) * kCodebooks + c) * 256;
             for (uint32_t i = 0; i < 256; ++i) t[i] = static_cast<uint8_t>((4 << 4) | bit_reverse(i & 15u, 4));
         }
+    // rank tables and arithmetic-decode constants of the decompress kernel (layout: ecco_format.h)
+    uint8_t* rl = base + kOffRankLut;
+    uint32_t* ar = reinterpret_cast<uint32_t*>(base + kOffArith);
+    const uint32_t n_cb = kMaxPatterns * kCodebooks;
+    for (int k = 0; k < kMaxPatterns; ++k)
+        for (int c = 0; c < kCodebooks; ++c) {
+            const uint32_t cb = static_cast<uint32_t>(k) * kCodebooks + c, rot = lut_rotation(cb);
+            int len[kSymbols];
+            uint32_t code[kSymbols];                       // codeword value, first code bit on top
+            for (int s = 0; s < kSymbols; ++s) {
+                len[s] = k < tmp.S ? tmp.cb_len[k][c][s] : 4;
+                code[s] = k < tmp.S ? bit_reverse(tmp.cb_rev[k][c][s], len[s]) : static_cast<uint32_t>(s);
+            }
+            // first[L]: smallest codeword of length L; ahead[L]: number of symbols with shorter codewords
+            uint32_t first[kMaxLen + 2] = {0}, count[kMaxLen + 2] = {0}, ahead[kMaxLen + 2] = {0}, thr[kMaxLen + 2] = {0};
+            for (int s = 0; s < kSymbols; ++s) ++count[len[s]];
+            uint32_t next = 0, seen = 0;
+            for (int L = 1; L <= kMaxLen; ++L) {
+                first[L] = next; ahead[L] = seen;
+                thr[L] = (next + count[L]) << (kMaxLen - L);   // <= 256: first window byte past the codewords of length <= L
+                next = (next + count[L]) << 1; seen += count[L];
+            }
+            const uint32_t rho = count[kMaxLen] ? (first[kMaxLen] - ahead[kMaxLen]) & 15u : 0u;
+            uint32_t delta[kMaxLen + 1];
+            for (int L = kMinLen; L <= kMaxLen; ++L) delta[L] = (ahead[L] + rho - first[L]) & 15u;
+            uint64_t rank_of = 0;
+            uint8_t* t = rl + static_cast<size_t>(cb) * 256;
+            for (int s = 0; s < kSymbols; ++s) {
+                const int L = len[s];
+                const uint32_t rank = (code[s] + delta[L]) & 15u;
+                rank_of |= static_cast<uint64_t>(rank) << (4 * s);
+                const uint32_t rev = bit_reverse(code[s], L);
+                for (uint32_t hi = 0; hi < (1u << (kMaxLen - L)); ++hi)
+                    t[(rev | (hi << L)) ^ rot] = static_cast<uint8_t>((L << 4) | rank);
+            }
+            uint32_t w0 = 0xC0000000u, w1 = 0, w2 = 0;
+            for (int i = 0; i < 3; ++i) {
+                w0 |= (256u - thr[2 + i]) << (10 * i);
+                w1 |= (256u - thr[5 + i]) << (10 * i + 1);
+            }
+            for (int L = kMinLen; L < kMaxLen; ++L) w2 |= delta[L] << (4 * (L - kMinLen));
+            ar[0 * n_cb + cb] = w0;
+            ar[1 * n_cb + cb] = w1;
+            ar[2 * n_cb + cb] = w2;
+            ar[3 * n_cb + cb] = static_cast<uint32_t>(rank_of);
+            ar[4 * n_cb + cb] = static_cast<uint32_t>(rank_of >> 32);
+        }
     return ECCO_OK;
 }
 

@@ -16,6 +16,7 @@
 //            syms[16][32] u32   (fused kernels) decoded indices, 8 nibbles per word, for the
 //                               outlier fix-up
 #include <cuda.h>
+#include <cuda/std/type_traits>
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include <cuda_runtime.h>
@@ -40,10 +41,13 @@ constexpr uint32_t kSmemPattern = 0;
 constexpr uint32_t kSmemKpLut = kPatternBytes;
 constexpr uint32_t kSmemSymLut = kPatternBytes + kKpLutBytes;        // 10240: 256-aligned
 constexpr uint32_t kSmemWarpBase = kTableBytes;                      // 75776: 1024-aligned
+constexpr uint32_t kSmemArith = kTableBytes;                         // mixed decoder: constants after the rank tables,
+constexpr uint32_t kSmemRankWarpBase = kTableBytes + kArithBytes;    // per-warp arrays after them (80896: 1024-aligned)
 constexpr uint32_t kBitsRows = 18;
 constexpr uint32_t kBitsBytes = kBitsRows * 32 * 4;                  // 2304
 constexpr uint32_t kTabBytes = 16 * 32 * 4;                          // 2048
 constexpr uint32_t kSymsBytes = 16 * 32 * 4;                         // 2048
+constexpr int kFusedFree = 12;                                       // fused kernels: leading decode steps without the clip test
 constexpr int kWaitLimit = 1 << 22;                                  // bounded mbarrier polling
 
 // ---------------------------------------------------------------------------------------------
@@ -158,6 +162,27 @@ __device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_met
     return all;
 }
 
+// Same for the mixed decoder: patterns and ID_KP table, then rank tables and arithmetic constants
+// (adjacent in the image and in shared memory), two bulk copies on one barrier.
+__device__ __forceinline__ bool stage_rank_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+{
+    const uint32_t bar = smem_u32(bar_storage);
+    if (threadIdx.x == 0) mbar_init(bar, 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        mbar_expect_tx(bar, kPatternBytes + kKpLutBytes + kRankLutBytes + kArithBytes);
+        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kPatternBytes + kKpLutBytes, bar);
+        bulk_g2s(smem_u32(smem) + kSmemSymLut, d_meta + kOffRankLut, kRankLutBytes + kArithBytes, bar);
+    }
+    bool done = false;
+    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+    if (!done)
+        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+    const bool all = __syncthreads_and(done);
+    if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
+    return all;
+}
+
 // ---------------------------------------------------------------------------------------------
 // the per-group decoder
 // ---------------------------------------------------------------------------------------------
@@ -170,13 +195,22 @@ struct WarpSmem {
 struct GroupHeader {
     uint32_t pos;       // first bit of the coded indices
     uint32_t lut;       // shared address of the symbol table of (ID_KP, ID_HF), OR-ed with its index rotation
+    // mixed decoder only: addends of the length compare, and delta[L] in byte L of {dhi:dlo} (byte 0 = 0)
+    uint32_t c1, c2, dlo, dhi;
 };
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
 
 // Pattern retriever (Sec. 4.2): scale byte, ID_HF, Huffman-coded ID_KP from the group's first 22
 // stream bits (hdr, first bit in bit 0); writes the lane's 16 dequantised values (fp16 bits, or
 // fp32 bits when kFloatTab).  first_bit = position of the group's first bit in the lane's staged
 // bit stream.
-template <bool kFloatTab>
+// kRank: the kernel staged the rank tables (stage_rank_tables); tab is then indexed by rank.
+template <bool kFloatTab, bool kRank = false>
 __device__ __forceinline__ GroupHeader open_header(uint32_t hdr, uint32_t first_bit, uint32_t smem_base, const WarpSmem& ws, float T)
 {
     const uint32_t qs = hdr & 0xffu, hf = (hdr >> 8) & 3u;
@@ -194,23 +228,36 @@ __device__ __forceinline__ GroupHeader open_header(uint32_t hdr, uint32_t first_
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(p0.x), "=r"(p0.y), "=r"(p0.z), "=r"(p0.w) : "r"(smem_base + kSmemPattern + kp * 32));
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(p1.x), "=r"(p1.y), "=r"(p1.z), "=r"(p1.w) : "r"(smem_base + kSmemPattern + kp * 32 + 16));
     const uint32_t pr[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+    uint32_t rank_lo = 0, rank_hi = 0;
+    if (kRank) {
+        const uint32_t a = smem_base + kSmemArith + cb * 4;
+        h.c1 = lds_u32(a);
+        h.c2 = lds_u32(a + 1024);
+        const uint32_t d = lds_u32(a + 2048);
+        rank_lo = lds_u32(a + 3072);
+        rank_hi = lds_u32(a + 4096);
+        const uint32_t even = d & 0x0f0f0fu, odd = (d >> 4) & 0x0f0f0fu;     // delta[2], [4], [6] and delta[3], [5], [7]
+        h.dlo = prmt(even, odd, 0x4033u);
+        h.dhi = prmt(even, odd, 0x6251u);
+    }
 #pragma unroll
     for (int j = 0; j < 16; ++j) {
         const __half c = __ushort_as_half(static_cast<unsigned short>((pr[j >> 1] >> ((j & 1) * 16)) & 0xffffu));
         // mapper (Sec. 4.2): one fp32 product, one rounding to fp16
         const __half v = __float2half_rn(j < 15 ? __half2float(c) * s : top);
-        sts_u32(ws.tab + j * 128, kFloatTab ? __float_as_uint(__half2float(v)) : static_cast<uint32_t>(__half_as_ushort(v)));
+        const uint32_t row = kRank ? ((j < 8 ? rank_lo : rank_hi) >> ((j & 7) * 4)) & 15u : static_cast<uint32_t>(j);
+        sts_u32(ws.tab + row * 128, kFloatTab ? __float_as_uint(__half2float(v)) : static_cast<uint32_t>(__half_as_ushort(v)));
     }
     return h;
 }
 
 // 64-byte block: stage the 16 words in the lane's column of the transposed bit-stream array, then the header
-template <bool kFloatTab>
+template <bool kFloatTab, bool kRank = false>
 __device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T)
 {
 #pragma unroll
     for (int i = 0; i < 16; ++i) sts_u32(ws.bits + i * 128, blk.w[i]);
-    return open_header<kFloatTab>(blk.w[0], 0u, smem_base, ws, T);
+    return open_header<kFloatTab, kRank>(blk.w[0], 0u, smem_base, ws, T);
 }
 
 // Decodes the 128 indices of the lane's group (Sec. 4.2, Huffman decode) and hands each value to
@@ -220,24 +267,40 @@ __device__ __forceinline__ GroupHeader open_group(const Block& blk, uint32_t sme
 // per-symbol clip test runs only in steps where some lane of the warp reaches bit 512.
 // kLastRow / kEndBit: last data row of the lane's staged stream (two zero rows follow) and the bit
 // at which the stream ends (16 and 512 for the 64-byte block).
-template <bool kLookup = true, uint32_t kLastRow = 16, uint32_t kEndBit = kBlockBits, class Sink>
+// kArith (rank tables only): bit j set = symbol j of every four is decoded arithmetically from the canonical
+// code's length thresholds instead of through the byte table; the sink's symbol is then the rank, and only its
+// low four bits are meaningful.
+// kFreeSteps (a multiple of 4): that many leading steps run without the clip test; the caller guarantees that
+// the stream cannot end within them (a block's indices start at bit 22 at the latest, so 12 steps of at most
+// 32 bits end by bit 406).
+template <bool kLookup = true, uint32_t kLastRow = 16, uint32_t kEndBit = kBlockBits, uint32_t kArith = 0, int kFreeSteps = 0, class Sink>
 __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const WarpSmem& ws, Sink&& sink)
 {
+    static_assert(kFreeSteps % 4 == 0 && kFreeSteps < 32, "whole unrolled iterations");
     uint32_t pos = h.pos;
     bool alive = true;
-#pragma unroll 4
-    for (int step = 0; step < 32; ++step) {
-        const uint32_t wi = min(pos >> 5, kLastRow);
+    auto four = [&](int step, auto tested) {
+        constexpr bool kTest = decltype(tested)::value;
+        const uint32_t wi = kTest ? min(pos >> 5, kLastRow) : pos >> 5;
         const uint32_t lo = lds_u32(ws.bits + wi * 128), hi = lds_u32(ws.bits + wi * 128 + 128);
         const uint32_t win = __funnelshift_r(lo, hi, pos);           // 32 stream bits from pos
+        const uint32_t wrev = kArith ? __brev(win) : 0u;             // the same bits, first one on top
         uint32_t e[4], end[4], acc = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            e[j] = lds_u8(h.lut ^ ((win >> acc) & 0xffu));           // rotated index, see lut_rotation()
-            acc += e[j] >> 4;
+            if ((kArith >> j) & 1u) {
+                const uint32_t t = wrev << acc, b = t >> 24;
+                const uint32_t m = ((b * kArithSpread + h.c1) & (kArithGuard | 0xC0000000u)) | ((b * (2u * kArithSpread) + h.c2) & (2u * kArithGuard));
+                const uint32_t len = __popc(m);                      // 2 + thresholds passed
+                e[j] = __funnelshift_l(t, 0u, len) + prmt(h.dlo, h.dhi, len);   // codeword + delta[len]
+                acc += len;
+            } else {
+                e[j] = lds_u8(h.lut ^ ((win >> acc) & 0xffu));       // rotated index, see lut_rotation()
+                acc += e[j] >> 4;
+            }
             end[j] = acc;
         }
-        if (__any_sync(0xffffffffu, pos + acc > kEndBit)) {
+        if (kTest && __any_sync(0xffffffffu, pos + acc > kEndBit)) {
             const uint32_t limit = kEndBit - min(pos, kEndBit);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -251,7 +314,13 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
                 sink(step * 4 + j, kLookup ? lds_u32(ws.tab + (e[j] & 15u) * 128) : 0u, e[j] & 15u, true);
         }
         pos += acc;
+    };
+    if (kFreeSteps > 0) {
+#pragma unroll 4
+        for (int step = 0; step < kFreeSteps; ++step) four(step, cuda::std::false_type{});
     }
+#pragma unroll 4
+    for (int step = kFreeSteps; step < 32; ++step) four(step, cuda::std::true_type{});
     return alive ? pos : 0u;
 }
 
@@ -331,23 +400,24 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
 // tensor and drops rows past its end.  Outliers: those in the last tile (positions >= 112) are
 // patched in shared memory before that tile leaves; the others are 2-byte global stores issued
 // after the group's earlier tiles have been written (bulk wait + warp barrier), so they land last.
-template <int kWarps>
+template <int kWarps, uint32_t kArith, int kDecFree = 12>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
                            uint16_t* __restrict__ d_out, uint32_t active_warps, const __grid_constant__ CUtensorMap out_map)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const uint32_t smem_base = smem_u32(smem);
-    constexpr uint32_t kStageBase = (kSmemWarpBase + kWarps * (kBitsBytes + kTabBytes) + 1023u) & ~1023u;
+    constexpr uint32_t kStageBase = (kSmemRankWarpBase + kWarps * (kBitsBytes + kTabBytes) + 1023u) & ~1023u;
     WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * (kBitsBytes + kTabBytes) + lane * 4;
+    ws.bits = smem_base + kSmemRankWarpBase + warp * (kBitsBytes + kTabBytes) + lane * 4;
     ws.tab = ws.bits + kBitsBytes;
     ws.syms = 0;
     sts_u32(ws.bits + 16 * 128, 0u);
     sts_u32(ws.bits + 17 * 128, 0u);
     const uint32_t stage = smem_base + kStageBase + warp * 1024;                 // this warp's staging tile
+    const uint32_t fp8tab = smem_base + kStageBase + kWarps * 1024;              // [256] fp16: outlier byte -> value
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem + kStageBase + kWarps * 1024 + 512);   // in the dynamic part: no room for a static one
     const uint32_t swz = ((lane >> 2) & 1u) << 4;                               // 32-byte swizzle: bit 4 ^= bit 7
     const uint32_t my_row = stage + lane * 32;
 
@@ -357,13 +427,16 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
     if (tile >= tile_stride) tile = n_tiles;
     Block blk;
     if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
-    if (!stage_tables(smem, d_meta, &bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (threadIdx.x < 256)                                 // visible after the barrier inside stage_rank_tables
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(fp8tab + threadIdx.x * 2),
+                     "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(threadIdx.x) * T))) : "memory");
+    if (!stage_rank_tables(smem, d_meta, bar)) return;
 
     for (; tile < n_tiles; tile += tile_stride) {
         const uint64_t g = tile * 32 + lane;
         const bool store = g < n_groups;
-        const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
+        const GroupHeader h = open_group<false, true>(blk, smem_base, ws, T);
         const uint64_t tn = tile + tile_stride;
         if (tn < n_tiles) ldg_block(blk, d_blocks + min(tn * 32 + lane, n_groups - 1) * kBlockBytes);
         const int row0 = static_cast<int>(tile * 32);
@@ -379,7 +452,7 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
             __syncwarp();
             if (lane == 0) { tma_store_2d(&out_map, stage, chunk * 16, row0); bulk_commit(); }
         };
-        const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
+        const uint32_t end = decode_symbols<true, 16, kBlockBits, kArith, kDecFree>(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
             const int slot = (n & 15) >> 1;
             if (n & 1) r[slot] |= v << 16; else r[slot] = v;
             if ((n & 15) == 15 && n != 127) { stage_rows(); send_tile(n >> 4); }
@@ -390,15 +463,21 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
             if (lane == 0) bulk_wait_all();                // tiles 0..6 of this group are in memory
             __syncwarp();
             uint16_t* out = d_out + min(g, n_groups - 1) * kGroup;
-            for (int j = 0; j < n_pad; ++j) {              // ascending: a later pad overrides an earlier one
-                const uint32_t f = read_pad(ws, j);
-                const uint32_t loc = f & 127u;
-                const uint16_t val = static_cast<uint16_t>(f2h_bits(fp8_to_float(f >> 7) * T));
-                if (loc >= 112u) {
-                    const uint32_t byte = (loc - 112u) * 2;
-                    asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)), "h"(val) : "memory");
-                } else if (store) {
-                    out[loc] = val;
+            const int n_max = __reduce_max_sync(0xffffffffu, n_pad);
+#pragma unroll
+            for (int j = 0; j < kMaxPads; ++j) {           // ascending: a later pad overrides an earlier one
+                if (j >= n_max) break;
+                if (j < n_pad) {
+                    const uint32_t f = read_pad(ws, j);
+                    const uint32_t loc = f & 127u;
+                    unsigned short val;
+                    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(val) : "r"(fp8tab + (f >> 7) * 2));
+                    if (loc >= 112u) {
+                        const uint32_t byte = (loc - 112u) * 2;
+                        asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)), "h"(val) : "memory");
+                    } else if (store) {
+                        out[loc] = val;
+                    }
                 }
             }
         }
@@ -559,7 +638,7 @@ __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base
 {
     const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
     uint32_t packed = 0;
-    const uint32_t end = decode_symbols(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
         acc.fma(n, __uint_as_float(v), xs);
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
@@ -963,7 +1042,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
         uint32_t packed = 0;
         int n_fit = kGroup;
-        const uint32_t end = decode_symbols<false>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+        const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
             if (!alive) n_fit = min(n_fit, n);             // only the clip path can see alive == false
             packed |= sym << ((n & 7) * 4);
             if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
@@ -1058,7 +1137,7 @@ __device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base
     const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
     uint32_t packed = 0;
     int n_fit = kGroup;
-    const uint32_t end = decode_symbols<false>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+    const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
         if (!alive) n_fit = min(n_fit, n);
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
@@ -1408,6 +1487,9 @@ static bool make_out_map(CUtensorMap* map, void* d_out, uint64_t n_groups)
 }
 
 constexpr int kDecompressTmaWarps = 28;
+// symbols 1 and 3 of every four are decoded arithmetically, 0 and 2 through the byte table: measured best of
+// {none, one, two, three, all} on the 11008x4096 matrix and on a 256 MiB cache (all-table 441 us, this 394 us, all-arithmetic 459 us)
+constexpr uint32_t kDecompressArith = 0b1010;
 
 extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out, void* stream)
 {
@@ -1423,10 +1505,11 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     // bulk-store variant for everything but tiny tensors (its box is 32 rows tall)
     CUtensorMap map;
     if (n_groups >= 32 && make_out_map(&map, d_out, n_groups)) {
-        auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps>;
+        auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps, kDecompressArith>;
         constexpr size_t smem =
-            ((kSmemWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
-            static_cast<size_t>(kDecompressTmaWarps) * 1024;
+            ((kSmemRankWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
+            static_cast<size_t>(kDecompressTmaWarps) * 1024 + 512 + 16;       // + outlier value table + barrier
+        static_assert(smem <= 232448, "227 KB per CTA");
         if (!configured_tma[di.device]) {
             rc = set_smem(kernel, smem);
             if (rc) return rc;

@@ -160,7 +160,7 @@ def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
     ometa = cfg1_small["meta"]
     lm = lib_meta_from_oracle(binding, ometa)
     img = binding.ecco_meta_serialize_device(lm)
-    assert img.size == binding.ecco_meta_device_bytes(lm) == 84160
+    assert img.size == binding.ecco_meta_device_bytes(lm) == 84160 + 65536 + 5120
     hdr = img[:64].view(np.uint32)
     assert hdr[0] == 0x4F434345 and hdr[2] == 64 and hdr[3] == 4 and hdr[4:5].view(np.int32)[0] == ometa.e
     assert img[20:24].view(np.float32)[0] == 2.0 ** ometa.e
@@ -191,6 +191,44 @@ def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
             pos += t >> 4
             n += 1
         assert n == info.n_fit and pos == info.end_bit
+
+
+def test_device_image_rank_tables_and_arithmetic_constants(binding, eo, cfg1_small):
+    """The mixed decoder's tables against the oracle's canonical codes: for every codebook and every 8-bit
+    window, the rank table has the oracle's codeword length and a rank that is a bijection of the symbol,
+    and the arithmetic route (threshold compare, codeword + delta) lands on the same length and rank."""
+    ometa = cfg1_small["meta"]
+    lm = lib_meta_from_oracle(binding, ometa)
+    img = binding.ecco_meta_serialize_device(lm)
+    syml = img[64 + 2048 + 8192:64 + 2048 + 8192 + 65536].reshape(256, 256)
+    rankl = img[84160:84160 + 65536].reshape(256, 256)
+    ar = img[84160 + 65536:].view(np.uint32).reshape(5, 256)
+    lengths = ometa.cb_lengths()                                   # [pattern][codebook][symbol]
+    spread = 1 | 1 << 10 | 1 << 20
+    guard = 0x100 | 0x100 << 10 | 0x100 << 20
+    for cb in range(ometa.S * 4):
+        lens = [int(x) for x in lengths[cb // 4, cb % 4]]
+        codes, kraft = eo.canonical_codes(lens, 8)
+        assert kraft == 256
+        rot = ((cb * 11 + (cb >> 3)) & 31) << 2
+        c1, c2, d, rlo, rhi = (int(ar[i, cb]) for i in range(5))
+        rank_of = rlo | rhi << 32
+        assert sorted((rank_of >> 4 * s) & 15 for s in range(16)) == list(range(16))
+        delta = {L: (d >> 4 * (L - 2)) & 15 for L in range(2, 8)}
+        delta[8] = 0
+        for s in range(16):                                        # every window that starts with the codeword of s
+            L, code = lens[s], int(codes[s])
+            for rest in range(1 << (8 - L)):
+                b = code << (8 - L) | rest                         # first stream bit on top
+                i = int(f"{b:08b}"[::-1], 2)                       # the same window, first stream bit in bit 0
+                assert int(syml[cb, i ^ rot]) == (L << 4 | s)
+                assert int(rankl[cb, i ^ rot]) == (L << 4 | ((rank_of >> 4 * s) & 15))
+                m = ((b * spread + c1) & 0xFFFFFFFF & (guard | 0xC0000000)) | ((b * 2 * spread + c2) & 0xFFFFFFFF & (2 * guard))
+                assert bin(m).count("1") == L
+                assert ((b >> (8 - L)) + delta[L]) & 15 == (rank_of >> 4 * s) & 15
+    # rows of unused patterns decode as sixteen 4-bit codewords in every table
+    for cb in range(ometa.S * 4, 256):
+        assert np.all(rankl[cb] >> 4 == 4) and np.all(syml[cb] >> 4 == 4)
 
 
 def test_variable_length_host_encoder_matches_oracle(binding, eo, cfg1_small, kv_small):
