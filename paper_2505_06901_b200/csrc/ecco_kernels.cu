@@ -162,27 +162,52 @@ __device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_met
     return all;
 }
 
-// Same for the mixed decoder: patterns and ID_KP table, then rank tables and arithmetic constants
-// (adjacent in the image and in shared memory), two bulk copies on one barrier.
-__device__ __forceinline__ bool stage_rank_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+// The same in two halves, so that the caller can put work between the issue and the wait.
+__device__ __forceinline__ void issue_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
 {
     const uint32_t bar = smem_u32(bar_storage);
-    if (threadIdx.x == 0) mbar_init(bar, 1);
-    __syncthreads();
     if (threadIdx.x == 0) {
-        mbar_expect_tx(bar, kPatternBytes + kKpLutBytes + kRankLutBytes + kArithBytes);
-        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kPatternBytes + kKpLutBytes, bar);
-        bulk_g2s(smem_u32(smem) + kSmemSymLut, d_meta + kOffRankLut, kRankLutBytes + kArithBytes, bar);
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar, kTableBytes);
+        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kTableBytes, bar);
     }
+}
+__device__ __forceinline__ bool wait_tables(uint64_t* bar_storage)
+{
+    const uint32_t bar = smem_u32(bar_storage);
+    __syncthreads();                             // the barrier word is initialised
     bool done = false;
     for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
-    if (!done)
+    if (!done)                                   // second, bounded chance for the copy in flight
         for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
     const bool all = __syncthreads_and(done);
     if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
     return all;
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
+// while the previous kernel in the stream is still draining; dependency_wait() returns once that kernel
+// has completed and its writes are visible (at once if there is no such overlap), release_dependents()
+// lets the next kernel of the stream do the same with respect to this one.  The metadata image is an
+// input that no kernel of this library writes: its tables are fetched before the wait; every other
+// buffer is touched only after it.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+// Same for the mixed decoder: patterns and ID_KP table, then rank tables and arithmetic constants
+// (adjacent in the image and in shared memory), two bulk copies on one barrier.  In two halves so
+// that the caller can put work between the issue and the wait.
+__device__ __forceinline__ void issue_rank_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+{
+    const uint32_t bar = smem_u32(bar_storage);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_expect_tx(bar, kPatternBytes + kKpLutBytes + kRankLutBytes + kArithBytes);
+        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kPatternBytes + kKpLutBytes, bar);
+        bulk_g2s(smem_u32(smem) + kSmemSymLut, d_meta + kOffRankLut, kRankLutBytes + kArithBytes, bar);
+    }
+}
 // ---------------------------------------------------------------------------------------------
 // the per-group decoder
 // ---------------------------------------------------------------------------------------------
@@ -425,13 +450,18 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
     const uint64_t tile_stride = active_warps;             // see ecco_decompress_kernel
     uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
     if (tile >= tile_stride) tile = n_tiles;
-    Block blk;
-    if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
+    // The metadata image is an input that no kernel of this library writes: its tables are fetched before
+    // the wait on the previous kernel of the stream; blocks and output are touched only after it.
+    issue_rank_tables(smem, d_meta, bar);
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
-    if (threadIdx.x < 256)                                 // visible after the barrier inside stage_rank_tables
+    if (threadIdx.x < 256)                                 // visible after the barriers inside wait_rank_tables
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(fp8tab + threadIdx.x * 2),
                      "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(threadIdx.x) * T))) : "memory");
-    if (!stage_rank_tables(smem, d_meta, bar)) return;
+    dependency_wait();
+    release_dependents();
+    Block blk;
+    if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
+    if (!wait_tables(bar)) return;
 
     for (; tile < n_tiles; tile += tile_stride) {
         const uint64_t g = tile * 32 + lane;
@@ -722,9 +752,12 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!stage_tables(smem, d_meta, &bar)) return;
+    if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     Accum<kV> acc;
@@ -836,9 +869,12 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!stage_tables(smem, d_meta, &bar)) return;
+    if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     int cur_bh = -1;
@@ -884,6 +920,8 @@ __global__ void __launch_bounds__(256)
 ecco_softmax_stats_kernel(const float* __restrict__ d_scores, int rows, int seq, float2* __restrict__ d_stats)
 {
     const int row = static_cast<int>(blockIdx.x) * 8 + static_cast<int>(threadIdx.x >> 5), lane = static_cast<int>(threadIdx.x & 31u);
+    dependency_wait();                                     // the scores may come from the previous kernel of the stream
+    release_dependents();
     if (row >= rows) return;
     const float* s = d_scores + static_cast<size_t>(row) * seq;
     float mx = -INFINITY;
@@ -945,9 +983,12 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!stage_tables(smem, d_meta, &bar)) return;
+    if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     float acc[8][4];                                       // [16-dim chunk][mma accumulator]
@@ -1229,10 +1270,13 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     Block blk;
     uint32_t vnext[16];
     if (u0 < u1) { ldg_block(blk, block_ptr(u0)); load_vfrag(vnext, d_x + static_cast<int>(u0 % kblocks) * kGroup, k, batch); }
-    if (!stage_tables(smem, d_meta, &bar)) return;
+    if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
@@ -1321,9 +1365,12 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!stage_tables(smem, d_meta, &bar)) return;
+    if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
     uint32_t vfrag[16];
@@ -1377,6 +1424,44 @@ int device_info(DeviceInfo* out)
     }
     *out = c;
     return c.cc_major == 10 ? ECCO_OK : ECCO_ERR_UNSUPPORTED_ARCH;
+}
+
+int check_launch();
+// Launch with the programmatic stream-serialisation attribute (see dependency_wait in the kernels):
+// the kernel must call dependency_wait() before it touches anything but the metadata image.
+template <class... Params, class... Args>
+int launch_overlapped(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    return check_launch();
+}
+
+// Zeroes the ticket words of a workspace.  A kernel rather than a memset so that it can sit in a chain of
+// overlapped launches: it lets its successor start at once and clears only after its predecessor (which may
+// still be using the same workspace) has completed.
+__global__ void ecco_zero_words_kernel(unsigned int* __restrict__ p, size_t n)
+{
+    release_dependents();
+    dependency_wait();
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<size_t>(gridDim.x) * blockDim.x) p[i] = 0u;
+}
+inline int zero_tickets(unsigned int* tickets, size_t bytes, cudaStream_t stream)
+{
+    const size_t n = bytes / sizeof(unsigned int);
+    if (n == 0) return ECCO_OK;
+    const unsigned grid = static_cast<unsigned>(n < 8192 ? (n + 255) / 256 : 32);
+    return launch_overlapped(ecco_zero_words_kernel, grid, 256u, 0, stream, tickets, n);
 }
 
 template <class K>
@@ -1518,9 +1603,8 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
         const uint64_t cta_tiles = (n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
         const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
         const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kDecompressTmaWarps);
-        kernel<<<grid, kDecompressTmaWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-            static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), active, map);
-        return check_launch();
+        return launch_overlapped(kernel, grid, static_cast<unsigned>(kDecompressTmaWarps * 32), smem, static_cast<cudaStream_t>(stream),
+                                 static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), active, map);
     }
     auto kernel = ecco_decompress_kernel<kDecompressWarps>;
     const size_t smem = kSmemWarpBase + static_cast<size_t>(kDecompressWarps) * (kBitsBytes + kTabBytes);
@@ -1596,12 +1680,12 @@ static int launch_gemv_mma(const DeviceInfo& di, const void* d_meta, const uint8
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-    cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
-    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    int rc = zero_tickets(tickets, p.ticket_bytes, stream);
+    if (rc) return rc;
     const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kMmaWarps));
-    kernel<<<p.grid, kMmaWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
-                                                     static_cast<const __half*>(d_x), batch, d_y, partial, tickets, active);
-    return check_launch();
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kMmaWarps * 32), smem, stream,
+                             static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), batch, d_y,
+                             partial, tickets, active);
 }
 
 // one or two rows of x (batch == kV): the per-warp kernel
@@ -1623,12 +1707,12 @@ static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-    cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, stream);
-    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    int rc = zero_tickets(tickets, p.ticket_bytes, stream);
+    if (rc) return rc;
     const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kFusedWarps));
-    kernel<<<p.grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks,
-                                                       static_cast<const __half*>(d_x), d_y, partial, tickets, active);
-    return check_launch();
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kFusedWarps * 32), smem, stream,
+                             static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), d_y, partial,
+                             tickets, active);
 }
 
 extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x,
@@ -1709,9 +1793,8 @@ static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* 
     const int heads = batch * n_kv_heads;
     const int64_t units = static_cast<int64_t>(heads) * ((seq + kFusedRows - 1) / kFusedRows);
     const unsigned grid = balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(di.sms));   // persistent CTAs, same units each
-    kernel<<<grid, kFusedWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, heads, seq, q_per_kv,
-                                                     static_cast<const __half*>(d_q), scale, d_scores);
-    return check_launch();
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kFusedWarps * 32), smem, stream, static_cast<const uint8_t*>(d_meta),
+                             d_kblocks, heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores);
 }
 
 extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch, int32_t n_kv_heads, int32_t seq,
@@ -1742,9 +1825,8 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
             const uint64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
             const unsigned grid = static_cast<unsigned>(ctas < static_cast<uint64_t>(di.sms) ? ctas : di.sms);
             const int active = static_cast<int>(balanced_warps(units, grid * kMmaWarps));
-            kernel<<<grid, kMmaWarps * 32, smem, s>>>(static_cast<const uint8_t*>(d_meta), d_kblocks, batch * n_kv_heads, seq, q_per_kv,
-                                                      static_cast<const __half*>(d_q), scale, d_scores, active);
-            return check_launch();
+            return launch_overlapped(kernel, grid, static_cast<unsigned>(kMmaWarps * 32), smem, s, static_cast<const uint8_t*>(d_meta),
+                                     d_kblocks, batch * n_kv_heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores, active);
         }
     }
 }
@@ -1805,15 +1887,13 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     float2* stats = reinterpret_cast<float2*>(wsb);
     float* partial = reinterpret_cast<float*>(wsb + p.stats_bytes);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(wsb + p.stats_bytes + p.partial_bytes);
-    cudaError_t e = cudaMemsetAsync(tickets, 0, p.ticket_bytes, s);
-    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
-    const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
-    ecco_softmax_stats_kernel<<<(rows + 7) / 8, 256, 0, s>>>(d_scores, rows, seq, stats);
-    rc = check_launch();
+    rc = zero_tickets(tickets, p.ticket_bytes, s);
     if (rc) return rc;
-    kernel<<<p.grid, kAvWarps * 32, smem, s>>>(static_cast<const uint8_t*>(d_meta), d_vblocks, heads, seq, q_per_kv, d_scores,
-                                                stats, d_out, partial, tickets);
-    return check_launch();
+    const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
+    rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>((rows + 7) / 8), 256u, 0, s, d_scores, rows, seq, stats);
+    if (rc) return rc;
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kAvWarps * 32), smem, s,
+                             static_cast<const uint8_t*>(d_meta), d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets);
 }
 
 // ---------------------------------------------------------------------------------------------
