@@ -561,3 +561,85 @@ def test_var_decompress_config2_gate_full_size(B, eo, W, synth):
         assert_bit_exact(d_out[g0:g0 + 512].cpu().numpy(), want)
     assert bool(torch.isfinite(d_out).all())
     assert total / n < 512                                                  # on average the stream is shorter than the blocks
+
+
+# ------------------------------------------------------------------ stream order of back-to-back calls
+def test_back_to_back_calls_keep_stream_order(B, eo, kv_small, cfg1_small, synth):
+    """The kernels are launched so that one may start while its predecessor in the stream drains.  Calls that
+    depend on each other through a buffer (write-after-write on an output, read-after-write on blocks, scores and
+    a shared workspace), issued with no synchronisation in between, must give what they give one at a time."""
+    meta, lm = kv_small["meta"], lib_meta_from_oracle(B, kv_small["meta"])
+    d_meta = B.meta_to_device(lm)
+    reps = 96                                              # 196 608 groups: every SM busy, tails overlap heads
+    x = np.tile(kv_small["k"].reshape(-1, 128), (reps, 1))
+    n = x.shape[0]
+    want_blocks = np.tile(kv_small["blocks"], (reps, 1))
+    want_a = np.tile(eo.decode(meta, kv_small["blocks"]), (reps, 1))
+    other = np.ascontiguousarray(want_blocks[::-1])        # a second, different tensor of the same size
+    want_b = np.ascontiguousarray(want_a[::-1])
+    d_x, d_other = dev(x.reshape(-1)), dev(other)
+    d_blocks = torch.full((n, 64), 0xEE, dtype=torch.uint8, device="cuda")
+    d_out = torch.zeros(n * 128, dtype=torch.float16, device="cuda")
+    d_out2 = torch.zeros(n * 128, dtype=torch.float16, device="cuda")
+    for _ in range(6):
+        B.ecco_kv_compress(d_meta, d_x, n, d_blocks)       # blocks written ...
+        B.ecco_decompress(d_meta, d_blocks, n, d_out2)     # ... and read by the next kernel
+        B.ecco_decompress(d_meta, d_other, n, d_out)       # the same output twice: the later call wins
+        B.ecco_decompress(d_meta, d_blocks, n, d_out)
+        B.ecco_decompress(d_meta, d_other, n, d_out)
+        d_blocks_snapshot = d_blocks.clone()
+        d_blocks.fill_(0xEE)                               # a non-library kernel in between
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    assert_blocks_equal(d_blocks_snapshot.cpu().numpy(), want_blocks)
+    assert_bit_exact(d_out2.cpu().numpy().reshape(n, 128), want_a)
+    assert_bit_exact(d_out.cpu().numpy().reshape(n, 128), want_b)
+
+    # two products through ONE workspace, then scores -> softmax . V, all back to back
+    wmeta, wlm = cfg1_small["meta"], lib_meta_from_oracle(B, cfg1_small["meta"])
+    d_wmeta = B.meta_to_device(wlm)
+    n_out, k = 4096, 2048
+    blocks_a = np.tile(cfg1_small["blocks"], (32, 1))[: n_out * k // 128]
+    blocks_b = np.ascontiguousarray(blocks_a[::-1])
+    d_a, d_b = dev(blocks_a), dev(blocks_b)
+    for batch in (1, 8):
+        xs = synth.activations(batch, k, 400 + batch)
+        d_xs = dev(xs)
+        wsb = B.ecco_gemv_workspace_bytes(n_out, k, batch)
+        ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+        ws.fill_(0xA5)
+        one = []
+        for blk in (d_a, d_b):                             # one at a time
+            y = torch.empty((batch, n_out), dtype=torch.float32, device="cuda")
+            B.ecco_gemv(d_wmeta, blk, n_out, k, d_xs, batch, y, ws, wsb)
+            torch.cuda.synchronize()
+            one.append(y.cpu().numpy())
+        ys = [torch.empty((batch, n_out), dtype=torch.float32, device="cuda") for _ in range(8)]
+        for i, y in enumerate(ys):                         # back to back through the same workspace
+            B.ecco_gemv(d_wmeta, d_b if i & 1 else d_a, n_out, k, d_xs, batch, y, ws, wsb)
+        torch.cuda.synchronize()
+        assert B.ecco_device_status() == 0
+        for i, y in enumerate(ys):
+            assert np.array_equal(y.cpu().numpy(), one[i & 1]), (batch, i)
+
+    batch, heads, seq, qpk = 2, 4, 256, 4
+    kb, vb = kv_small["blocks"], np.ascontiguousarray(kv_small["blocks"][::-1])
+    q = synth.queries(batch, heads * qpk, 77)
+    d_k, d_v, d_q = dev(kb), dev(vb), dev(q)
+    wsb = B.ecco_attn_values_workspace_bytes(batch, heads, seq, qpk)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    sc = torch.empty((batch, heads * qpk, seq), dtype=torch.float32, device="cuda")
+    out = torch.empty((batch, heads * qpk, 128), dtype=torch.float32, device="cuda")
+    B.ecco_attn_scores(d_meta, d_k, batch, heads, seq, qpk, d_q, 0.0884, sc)
+    torch.cuda.synchronize()
+    B.ecco_attn_values(d_meta, d_v, batch, heads, seq, qpk, sc, out, ws, wsb)
+    torch.cuda.synchronize()
+    want = out.cpu().numpy().copy()
+    for _ in range(4):
+        sc.zero_()
+        out.zero_()
+        B.ecco_attn_scores(d_meta, d_k, batch, heads, seq, qpk, d_q, 0.0884, sc)
+        B.ecco_attn_values(d_meta, d_v, batch, heads, seq, qpk, sc, out, ws, wsb)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    assert np.array_equal(out.cpu().numpy(), want)
