@@ -451,6 +451,12 @@ def run_ours(args):
                      "note": "kernel of the headline metric; limited by the SM load/store pipe, see kernels[] and profiles/"},
         "kernels": kernels,
     }
+    if "decompress" not in segs:
+        # a diagnostic run without the headline segment has no headline number
+        line["value"] = None
+        line["roofline"] = None
+        line["e2e"] = None
+        line["note"] = "--only without decompress: the segment of the headline metric was not timed; see segments_us_per_step"
     if sweep is not None:
         line["stream_sweep"] = sweep
     if world == 1 and not args.no_cpu_baseline and dec:
