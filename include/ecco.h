@@ -24,6 +24,14 @@
  * never allocate.  fp16 values travel as raw uint16_t / void*.  d_blocks, d_out, d_x, d_q and
  * d_meta must be 16-byte aligned.  The library refuses to run on a device that is not
  * compute capability 10.x (ECCO_ERR_UNSUPPORTED_ARCH); there is no CPU fallback.
+ *
+ * Stream order: a call's results are those of running the calls of a stream one after the
+ * other.  Internally the decode kernels are launched so that one may become resident and fetch
+ * its tables from d_meta while the previous kernel of the stream is still draining; they touch
+ * blocks, vectors, workspaces and outputs only after that kernel has completed.  The one thing
+ * this asks of the caller: the metadata image at d_meta must be in place by ordinary stream order
+ * (ecco_meta_serialize_device + a copy), not be produced by a kernel that itself signals early
+ * completion to its successors (a programmatic launch trigger).
  */
 #ifndef ECCO_H_
 #define ECCO_H_

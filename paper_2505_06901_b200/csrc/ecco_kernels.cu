@@ -143,26 +143,8 @@ __device__ __forceinline__ uint32_t f2h_bits(float f) { return static_cast<uint3
 // ---------------------------------------------------------------------------------------------
 // table staging (Sec. 4.2: metadata "loaded once" before the compressed loads)
 // ---------------------------------------------------------------------------------------------
-// Returns false (CTA-uniform) if the bounded wait expired; the caller must then return.
-__device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
-{
-    const uint32_t bar = smem_u32(bar_storage);
-    if (threadIdx.x == 0) mbar_init(bar, 1);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        mbar_expect_tx(bar, kTableBytes);
-        bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kTableBytes, bar);
-    }
-    bool done = false;
-    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
-    if (!done)                                   // second, bounded chance for the copy in flight
-        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
-    const bool all = __syncthreads_and(done);
-    if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
-    return all;
-}
-
-// The same in two halves, so that the caller can put work between the issue and the wait.
+// In two halves, so that the caller can put work between the issue and the wait.  wait_tables returns false
+// (CTA-uniform) if the bounded wait expired; the caller must then return.
 __device__ __forceinline__ void issue_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
 {
     const uint32_t bar = smem_u32(bar_storage);
@@ -184,6 +166,11 @@ __device__ __forceinline__ bool wait_tables(uint64_t* bar_storage)
     const bool all = __syncthreads_and(done);
     if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
     return all;
+}
+__device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+{
+    issue_tables(smem, d_meta, bar_storage);
+    return wait_tables(bar_storage);
 }
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
 // while the previous kernel in the stream is still draining; dependency_wait() returns once that kernel
