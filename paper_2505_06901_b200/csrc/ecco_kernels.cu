@@ -48,6 +48,16 @@ constexpr uint32_t kBitsBytes = kBitsRows * 32 * 4;                  // 2304
 constexpr uint32_t kTabBytes = 16 * 32 * 4;                          // 2048
 constexpr uint32_t kSymsBytes = 16 * 32 * 4;                         // 2048
 constexpr int kFusedFree = 12;                                       // fused kernels: leading decode steps without the clip test
+// Scalar fused kernels (one or two dot products per group): decode mix as in the decompress kernel, 0 = all-table.
+// They issue more instructions per symbol than the decompress kernel and gain nothing from the mix (11008x4096,
+// batch 1: 44.2 us all-table, 44.3 us with one symbol in four decoded arithmetically, 46.1 us with two; scores over
+// the cfg-3 K cache 128.0 / 128.3 / 134.6 us), so it stays off; -DECCO_FUSED_ARITH=<mask> builds the other variants.
+#ifndef ECCO_FUSED_ARITH
+#define ECCO_FUSED_ARITH 0
+#endif
+constexpr uint32_t kFusedArith = ECCO_FUSED_ARITH;
+constexpr bool kFusedRank = kFusedArith != 0;
+constexpr uint32_t kFusedBase = kFusedRank ? kSmemRankWarpBase : kSmemWarpBase;
 constexpr int kWaitLimit = 1 << 22;                                  // bounded mbarrier polling
 
 // ---------------------------------------------------------------------------------------------
@@ -653,9 +663,9 @@ template <int kV>
 __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T,
                                             uint32_t xs, Accum<kV>& acc)
 {
-    const GroupHeader h = open_group<true>(blk, smem_base, ws, T);
+    const GroupHeader h = open_group<true, kFusedRank>(blk, smem_base, ws, T);
     uint32_t packed = 0;
-    const uint32_t end = decode_symbols<true, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedArith, kFusedFree>(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
         acc.fma(n, __uint_as_float(v), xs);
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
@@ -696,7 +706,7 @@ __device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
     WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * kWarpBytes + lane * 4;
+    ws.bits = smem_base + kFusedBase + warp * kWarpBytes + lane * 4;
     ws.tab = ws.bits + kBitsBytes;
     ws.syms = ws.tab + kTabBytes;
     sts_u32(ws.bits + 16 * 128, 0u);
@@ -725,7 +735,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
     const uint32_t smem_base = smem_u32(smem);
     const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    const uint32_t xs = smem_base + kSmemWarpBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
+    const uint32_t xs = smem_base + kFusedBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
 
     // W working warps (chosen by the host so that they all get the same number of units, and never
     // more than there are units); warp ids interleave over the CTAs; the other warps idle
@@ -739,7 +749,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
-    issue_tables(smem, d_meta, &bar);
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
     dependency_wait();
     release_dependents();
     Block blk;
@@ -844,7 +854,7 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
     const uint32_t smem_base = smem_u32(smem);
     const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
-    float* xs = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kWarpBytes);
+    float* xs = reinterpret_cast<float*>(smem + kFusedBase + kWarps * kWarpBytes);
     const uint32_t xs_addr = smem_u32(xs);
 
     const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
@@ -856,7 +866,7 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    issue_tables(smem, d_meta, &bar);
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
     dependency_wait();
     release_dependents();
     Block blk;
@@ -1473,7 +1483,7 @@ constexpr int kDecompressWarps = 32;
 // warps per CTA of the scalar fused kernels (one or two dot products per group): as many as shared memory allows
 constexpr int fused_warps(int) { return 22; }
 // per-warp GEMV: every warp also carries its own slice of x, which leaves room for 22 / 20 warps
-constexpr int gemv_warp_warps(int kV) { return kV >= 2 ? 20 : 22; }
+constexpr int gemv_warp_warps(int kV) { return kFusedRank ? (kV >= 2 ? 20 : 21) : (kV >= 2 ? 20 : 22); }
 
 struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
 
@@ -1682,7 +1692,7 @@ static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint
 {
     constexpr int kFusedWarps = gemv_warp_warps(kV);
     auto kernel = ecco_gemv_warp_kernel<kV, kFusedWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes + kGroup * kV * 4);
+    const size_t smem = kFusedBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes + kGroup * kV * 4);
     static thread_local bool configured[64] = {};
     if (!configured[di.device]) {
         int rc = set_smem(kernel, smem);
@@ -1770,7 +1780,7 @@ static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* 
 {
     constexpr int kFusedWarps = fused_warps(kV), kFusedRows = kFusedWarps * 32;
     auto kernel = ecco_attn_scores_kernel<kV, kFusedWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + kGroup * kV * 4;
+    const size_t smem = kFusedBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + kGroup * kV * 4;
     static thread_local bool configured[64] = {};
     if (!configured[di.device]) {
         int rc = set_smem(kernel, smem);
