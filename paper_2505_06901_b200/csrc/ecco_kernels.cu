@@ -2090,9 +2090,7 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
             key[j] = ((h16[j] & 0x7fffu) << 7) | static_cast<uint32_t>(127 - (lane * 4 + j));
         }
         // sorter: abs-max, first index on ties
-        uint32_t best = max(max(key[0], key[1]), max(key[2], key[3]));
-#pragma unroll
-        for (int o = 16; o; o >>= 1) best = max(best, __shfl_xor_sync(full, best, o));
+        const uint32_t best = __reduce_max_sync(full, max(max(key[0], key[1]), max(key[2], key[3])));
         const int pstar = 127 - static_cast<int>(best & 127u);
         const float xsel = (pstar & 3) == 0 ? x[0] : (pstar & 3) == 1 ? x[1] : (pstar & 3) == 2 ? x[2] : x[3];
         const float xp = __shfl_sync(full, xsel, pstar >> 2);
@@ -2105,8 +2103,12 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
             u[j] = (is_max || scale == 0.0f) ? 0.0f : __fdiv_rn(x[j], scale);
             if (!is_max) { lo = fminf(lo, u[j]); hi = fmaxf(hi, u[j]); }
         }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) { lo = fminf(lo, __shfl_xor_sync(full, lo, o)); hi = fmaxf(hi, __shfl_xor_sync(full, hi, o)); }
+        // warp min / max through the order-preserving integer image of a float (the sign of a zero result is
+        // irrelevant below: it only enters differences)
+        auto ordered = [](float f) { const uint32_t b = __float_as_uint(f); return b ^ (static_cast<uint32_t>(static_cast<int32_t>(b) >> 31) | 0x80000000u); };
+        auto unordered = [](uint32_t o) { return __uint_as_float(o ^ ((o >> 31) ? 0x80000000u : 0xffffffffu)); };
+        lo = unordered(__reduce_min_sync(full, ordered(lo)));
+        hi = unordered(__reduce_max_sync(full, ordered(hi)));
         // pattern selector: min/max fitness, two patterns per lane
         double score = INFINITY;
         int kp = lane;
@@ -2120,25 +2122,34 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
                 if (sc < score) { score = sc; kp = k; }
             }
         }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            const double os = __shfl_xor_sync(full, score, o);
-            const int ok = __shfl_xor_sync(full, kp, o);
-            if (os < score || (os == score && ok < kp)) { score = os; kp = ok; }
+        {   // arg-min over the lanes, ties to the lower id: a non-negative double orders like its bit pattern
+            const uint64_t sb = static_cast<uint64_t>(__double_as_longlong(score));
+            const uint32_t s_hi = static_cast<uint32_t>(sb >> 32), s_lo = static_cast<uint32_t>(sb);
+            const uint32_t m_hi = __reduce_min_sync(full, s_hi);
+            const uint32_t m_lo = __reduce_min_sync(full, s_hi == m_hi ? s_lo : 0xffffffffu);
+            kp = static_cast<int>(__reduce_min_sync(full, (s_hi == m_hi && s_lo == m_lo) ? static_cast<uint32_t>(kp) : 0xffffffffu));
         }
         // value mappers: nearest centroid, ties to the lower index
         // The pattern is ascending, so the nearest centroid is one of the two that bracket the value
         // (exact fp32 comparisons find them); the fp64 squared distances of those two decide, as in the
         // definition, and equal centroids resolve to the lowest index.
-        float cen[kCentroids];
-#pragma unroll
-        for (int m = 0; m < kCentroids; ++m) cen[m] = __half2float(__ushort_as_half(pat_s[kp * 16 + m]));
+        // A centroid is an fp16 number, so c <= u exactly when c <= u rounded down to fp16: the fifteen
+        // comparisons are eight packed fp16 ones (entry 15 of the row is replaced by +inf).
+        uint4 c_lo = reinterpret_cast<const uint4*>(pat_s)[kp * 2], c_hi = reinterpret_cast<const uint4*>(pat_s)[kp * 2 + 1];
+        c_hi.w = (c_hi.w & 0xffffu) | 0x7c000000u;
+        const uint32_t crow[8] = {c_lo.x, c_lo.y, c_lo.z, c_lo.w, c_hi.x, c_hi.y, c_hi.z, c_hi.w};
         uint32_t sym[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            int below = 0;                                 // centroids <= u
+            const __half2 uu = __half2half2(__float2half_rd(u[j]));
+            __half2 cnt = __floats2half2_rn(0.0f, 0.0f);
 #pragma unroll
-            for (int m = 0; m < kCentroids; ++m) below += cen[m] <= u[j] ? 1 : 0;
+            for (int m = 0; m < 8; ++m) {
+                __half2 c2;
+                asm("mov.b32 %0, %1;" : "=r"(*reinterpret_cast<uint32_t*>(&c2)) : "r"(crow[m]));
+                cnt = __hadd2(cnt, __hle2(c2, uu));
+            }
+            const int below = __half2int_rn(__hadd(__low2half(cnt), __high2half(cnt)));     // centroids <= u
             const int a = max(below - 1, 0), b = min(below, kCentroids - 1);
             const float ca = __half2float(__ushort_as_half(pat_s[kp * 16 + a])), cb = __half2float(__ushort_as_half(pat_s[kp * 16 + b]));
             const double da = static_cast<double>(u[j]) - static_cast<double>(ca), db = static_cast<double>(u[j]) - static_cast<double>(cb);
@@ -2154,13 +2165,14 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
             t01 += (e[0] >> 8) | (static_cast<uint32_t>(e[kSymbols] >> 8) << 16);
             t23 += (e[2 * kSymbols] >> 8) | (static_cast<uint32_t>(e[3 * kSymbols] >> 8) << 16);
         }
-#pragma unroll
-        for (int o = 16; o; o >>= 1) { t01 += __shfl_xor_sync(full, t01, o); t23 += __shfl_xor_sync(full, t23, o); }
+        t01 = __reduce_add_sync(full, t01);
+        t23 = __reduce_add_sync(full, t23);
         const uint32_t tot[4] = {t01 & 0xffffu, t01 >> 16, t23 & 0xffffu, t23 >> 16};
         int hf = 0;
+        uint32_t shortest = tot[0];
 #pragma unroll
         for (int hh = 1; hh < 4; ++hh)
-            if (tot[hh] < tot[hf]) hf = hh;
+            if (tot[hh] < shortest) { shortest = tot[hh]; hf = hh; }
         // bit positions: header, ID_KP codeword, then a prefix sum over the 128 code lengths
         const uint32_t kpe = kp_s[kp];
         const uint32_t kp_len = kpe >> 12;
@@ -2198,20 +2210,32 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
         if (end_bit <= static_cast<uint32_t>(kBlockBits)) {
             // outliers: the next-largest |x| (ties: lower index), as many 15-bit slots as fit, at most 16
             const int n_pad = min(kMaxPads, static_cast<int>((kBlockBits - end_bit) / kPadBits));
-            uint32_t taken = 0;
-            if ((pstar >> 2) == lane) taken = 1u << (pstar & 3);
+            // Every lane sorts its four keys (the abs-max itself left out); n_pad times the warp takes the largest
+            // head and its owner advances.  A lane then knows which of its values are outliers and with which
+            // slot numbers, and all lanes write their fields at once.
+            uint32_t k0 = key[0] + 1u, k1 = key[1] + 1u, k2 = key[2] + 1u, k3 = key[3] + 1u;      // +1: zero means "nothing left"
+            if ((pstar >> 2) == lane) {
+                if ((pstar & 3) == 0) k0 = 0; else if ((pstar & 3) == 1) k1 = 0; else if ((pstar & 3) == 2) k2 = 0; else k3 = 0;
+            }
+            auto order = [](uint32_t& a, uint32_t& b) { const uint32_t hi_ = max(a, b), lo_ = min(a, b); a = hi_; b = lo_; };
+            order(k0, k1); order(k2, k3); order(k0, k2); order(k1, k3); order(k1, k2);            // descending
+            const uint32_t s0 = k0, s1 = k1, s2 = k2, s3 = k3;
+            uint32_t slots = 0;                            // slot numbers of this lane's outliers, the latest in the low byte
+            int mine = 0;
             for (int p = 0; p < n_pad; ++p) {
-                uint32_t cand = 0;
+                const uint32_t top = __reduce_max_sync(full, k0);
+                if (k0 == top) {                           // keys are distinct: exactly one lane
+                    k0 = k1; k1 = k2; k2 = k3; k3 = 0;
+                    slots = (slots << 8) | static_cast<uint32_t>(p);
+                    ++mine;
+                }
+            }
 #pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (!(taken & (1u << j))) cand = max(cand, key[j] + 1u);      // +1: zero means "nothing left"
-                uint32_t top = cand;
-#pragma unroll
-                for (int o = 16; o; o >>= 1) top = max(top, __shfl_xor_sync(full, top, o));
-                const int idx = 127 - static_cast<int>((top - 1u) & 127u);
-                if ((idx >> 2) == lane) {
+            for (int i = 0; i < 4; ++i) {
+                if (i < mine) {
+                    const int idx = 127 - static_cast<int>(((i == 0 ? s0 : i == 1 ? s1 : i == 2 ? s2 : s3) - 1u) & 127u);
+                    const int p = static_cast<int>((slots >> (8 * (mine - 1 - i))) & 0xffu);
                     const int j = idx & 3;
-                    taken |= 1u << j;
                     const float xv = j == 0 ? x[0] : j == 1 ? x[1] : j == 2 ? x[2] : x[3];
                     const uint32_t field = static_cast<uint32_t>(idx) | (fp8(xv) << 7);
                     const uint32_t bp = kBlockBits - kPadBits * (p + 1), w = bp >> 5, off = bp & 31u;
