@@ -543,6 +543,9 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
 
+    issue_tables(smem, d_meta, &bar);
+    dependency_wait();
+    release_dependents();
     const uint64_t total_bits = d_index[0];
     const uint64_t stream_chunks = (total_bits + 127) >> 7;
     const uint64_t* chunk_base = d_index + 1;
@@ -553,19 +556,44 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     const uint64_t tile_stride = active_warps;
     uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
     if (tile >= tile_stride) tile = n_tiles;
-    if (!stage_tables(smem, d_meta, &bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
     uint32_t dirty_rows = 0;                               // rows of this lane's column that hold a previous group
 
+    // The span of a group comes from the index and its chunks from the stream: two dependent trips to memory.
+    // Both are fetched one tile ahead, the first kVarAhead chunks into registers (an average group covers five),
+    // the rare rest when the tile is staged.
+    constexpr uint32_t kVarAhead = 6;
+    struct Span { uint64_t start, end, c0; uint32_t nc; };
+    auto span_of = [&](uint64_t t) {
+        Span sp;
+        const uint64_t g = min(t * 32 + lane, n_groups - 1);
+        sp.start = min(start_of(g), total_bits);
+        sp.end = max(min(start_of(g + 1), total_bits), sp.start);          // the group sees [start, end), zeros after
+        sp.c0 = sp.start >> 7;
+        sp.nc = static_cast<uint32_t>(min(static_cast<uint64_t>(kVarRows / 4), ((sp.end + 127) >> 7) - sp.c0));
+        return sp;
+    };
+    auto load_chunk = [&](uint64_t c) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (c < stream_chunks) asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d_stream + c));
+        return v;
+    };
+    Span cur = {0, 0, 0, 0};
+    uint4 ahead[kVarAhead];
+    if (tile < n_tiles) {
+        cur = span_of(tile);
+#pragma unroll
+        for (uint32_t c = 0; c < kVarAhead; ++c) ahead[c] = c < cur.nc ? load_chunk(cur.c0 + c) : make_uint4(0, 0, 0, 0);
+    }
+
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
     for (; tile < n_tiles; tile += tile_stride) {
-        const uint64_t g = min(tile * 32 + lane, n_groups - 1);
-        const uint64_t start = min(start_of(g), total_bits);
-        const uint64_t end = max(min(start_of(g + 1), total_bits), start);   // the group sees [start, end), zeros after
-        const uint64_t c0 = start >> 7;
-        const uint32_t nc = static_cast<uint32_t>(min(static_cast<uint64_t>(kVarRows / 4), ((end + 127) >> 7) - c0));
-        for (uint32_t c = 0; c < nc; ++c) {
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (c0 + c < stream_chunks) asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d_stream + c0 + c));
+        const uint64_t end = cur.end;
+        const uint64_t c0 = cur.c0;
+        const uint32_t nc = cur.nc;
+        const uint32_t first_bit = static_cast<uint32_t>(cur.start & 127u);
+        auto stage_chunk = [&](uint32_t c, const uint4& v) {
             uint32_t w[4] = {v.x, v.y, v.z, v.w};
             const uint64_t first = (c0 + c) << 7;          // stream bit of w[0] bit 0
             if (first + 128 > end) {                       // bits of the next group read as zero
@@ -577,16 +605,25 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
             }
 #pragma unroll
             for (int k = 0; k < 4; ++k) sts_u32(ws.bits + (4 * c + k) * 128, w[k]);
+        };
+#pragma unroll
+        for (uint32_t c = 0; c < kVarAhead; ++c)
+            if (c < nc) stage_chunk(c, ahead[c]);
+        for (uint32_t c = kVarAhead; c < nc; ++c) stage_chunk(c, load_chunk(c0 + c));
+        const uint64_t tn = tile + tile_stride;
+        if (tn < n_tiles) {                                // the next tile's span and first chunks, in flight during this decode
+            cur = span_of(tn);
+#pragma unroll
+            for (uint32_t c = 0; c < kVarAhead; ++c) ahead[c] = c < cur.nc ? load_chunk(cur.c0 + c) : make_uint4(0, 0, 0, 0);
         }
         for (uint32_t r = 4 * nc; r < dirty_rows; ++r) sts_u32(ws.bits + r * 128, 0u);
         dirty_rows = 4 * nc;
-        const uint32_t first_bit = static_cast<uint32_t>(start & 127u);
         const uint32_t hw = first_bit >> 5;
         const uint32_t hdr = __funnelshift_r(lds_u32(ws.bits + hw * 128), lds_u32(ws.bits + hw * 128 + 128), first_bit);
         const GroupHeader h = open_header<false>(hdr, first_bit, smem_base, ws, T);
         const int row0 = static_cast<int>(tile * 32);
         uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-        decode_symbols<true, kVarRows - 2, kVarRows * 32>(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
+        decode_symbols<true, kVarRows - 2, kVarRows * 32, 0, 28>(h, ws, [&](int n, uint32_t v, uint32_t, bool) {
             const int slot = (n & 15) >> 1;
             if (n & 1) r[slot] |= v << 16; else r[slot] = v;
             if ((n & 15) == 15) {
@@ -1646,10 +1683,9 @@ extern "C" int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, 
     const uint64_t cta_tiles = (n_groups + kVarWarps * 32 - 1) / (kVarWarps * 32);
     const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
     const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kVarWarps);
-    kernel<<<grid, kVarWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t*>(d_meta), reinterpret_cast<const uint4*>(d_stream), static_cast<const uint64_t*>(d_index),
-        n_groups, static_cast<uint16_t*>(d_out), active, map);
-    return check_launch();
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kVarWarps * 32), smem, static_cast<cudaStream_t>(stream),
+                             static_cast<const uint8_t*>(d_meta), reinterpret_cast<const uint4*>(d_stream),
+                             static_cast<const uint64_t*>(d_index), n_groups, static_cast<uint16_t*>(d_out), active, map);
 }
 
 extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch)
@@ -2072,6 +2108,8 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
         for (int i = tid; i < static_cast<int>(kEncKpBytes / 16); i += kKvWarps * 32) reinterpret_cast<uint4*>(kp_s)[i] = src_k[i];
     }
     __syncthreads();
+    dependency_wait();                                     // the values may come from the previous kernel of the stream
+    release_dependents();
     const DevHeader* hdr = reinterpret_cast<const DevHeader*>(d_meta);
     const int S = hdr->S;
     const float T = hdr->T, invT = 1.0f / T;             // both exact powers of two
@@ -2263,7 +2301,7 @@ extern "C" int ecco_kv_compress(const void* d_meta, const void* d_x_fp16, uint64
     if (rc) return rc;
     const uint64_t ctas = (n_groups + kKvWarps - 1) / kKvWarps;
     const uint64_t cap = static_cast<uint64_t>(di.sms) * 8;
-    ecco_kv_compress_kernel<<<static_cast<unsigned>(ctas < cap ? ctas : cap), kKvWarps * 32, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t*>(d_meta), static_cast<const __half*>(d_x_fp16), n_groups, d_blocks);
-    return check_launch();
+    return launch_overlapped(ecco_kv_compress_kernel, static_cast<unsigned>(ctas < cap ? ctas : cap), static_cast<unsigned>(kKvWarps * 32), 0,
+                             static_cast<cudaStream_t>(stream), static_cast<const uint8_t*>(d_meta), static_cast<const __half*>(d_x_fp16),
+                             n_groups, d_blocks);
 }
