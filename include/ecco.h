@@ -25,13 +25,9 @@
  * d_meta must be 16-byte aligned.  The library refuses to run on a device that is not
  * compute capability 10.x (ECCO_ERR_UNSUPPORTED_ARCH); there is no CPU fallback.
  *
- * Stream order: a call's results are those of running the calls of a stream one after the
- * other.  Internally the decode kernels are launched so that one may become resident and fetch
- * its tables from d_meta while the previous kernel of the stream is still draining; they touch
- * blocks, vectors, workspaces and outputs only after that kernel has completed.  The one thing
- * this asks of the caller: the metadata image at d_meta must be in place by ordinary stream order
- * (ecco_meta_serialize_device + a copy), not be produced by a kernel that itself signals early
- * completion to its successors (a programmatic launch trigger).
+ * Stream order: the usual one.  Internally the kernels are launched so that one may become
+ * resident while the previous kernel of the stream is still draining, but each waits for that
+ * kernel to complete before its first access to memory, so only launch latency overlaps.
  */
 #ifndef ECCO_H_
 #define ECCO_H_

@@ -182,12 +182,11 @@ __device__ __forceinline__ bool stage_tables(uint8_t* smem, const uint8_t* d_met
     issue_tables(smem, d_meta, bar_storage);
     return wait_tables(bar_storage);
 }
-// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may start
-// while the previous kernel in the stream is still draining; dependency_wait() returns once that kernel
-// has completed and its writes are visible (at once if there is no such overlap), release_dependents()
-// lets the next kernel of the stream do the same with respect to this one.  The metadata image is an
-// input that no kernel of this library writes: its tables are fetched before the wait; every other
-// buffer is touched only after it.
+// Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may become resident
+// while the previous kernel in the stream is still draining.  dependency_wait() returns once that kernel has
+// completed and its writes are visible (at once if there is no such overlap); every kernel executes it before
+// its first access to global memory, so stream order is what it is without the attribute and only launch and
+// prologue overlap.  release_dependents() lets the next kernel of the stream do the same with respect to this one.
 __device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -447,15 +446,13 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
     const uint64_t tile_stride = active_warps;             // see ecco_decompress_kernel
     uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
     if (tile >= tile_stride) tile = n_tiles;
-    // The metadata image is an input that no kernel of this library writes: its tables are fetched before
-    // the wait on the previous kernel of the stream; blocks and output are touched only after it.
+    dependency_wait();
+    release_dependents();
     issue_rank_tables(smem, d_meta, bar);
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
     if (threadIdx.x < 256)                                 // visible after the barriers inside wait_rank_tables
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(fp8tab + threadIdx.x * 2),
                      "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(threadIdx.x) * T))) : "memory");
-    dependency_wait();
-    release_dependents();
     Block blk;
     if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
     if (!wait_tables(bar)) return;
@@ -543,9 +540,9 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
 
-    issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    issue_tables(smem, d_meta, &bar);
     const uint64_t total_bits = d_index[0];
     const uint64_t stream_chunks = (total_bits + 127) >> 7;
     const uint64_t* chunk_base = d_index + 1;
@@ -786,9 +783,9 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
-    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!wait_tables(&bar)) return;
@@ -903,9 +900,9 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!wait_tables(&bar)) return;
@@ -1017,9 +1014,9 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    issue_tables(smem, d_meta, &bar);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!wait_tables(&bar)) return;
@@ -1304,9 +1301,9 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
-    issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    issue_tables(smem, d_meta, &bar);
     Block blk;
     uint32_t vnext[16];
     if (u0 < u1) { ldg_block(blk, block_ptr(u0)); load_vfrag(vnext, d_x + static_cast<int>(u0 % kblocks) * kGroup, k, batch); }
@@ -1399,9 +1396,9 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    issue_tables(smem, d_meta, &bar);
-    dependency_wait();
+    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
+    issue_tables(smem, d_meta, &bar);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!wait_tables(&bar)) return;
@@ -1462,7 +1459,7 @@ int device_info(DeviceInfo* out)
 
 int check_launch();
 // Launch with the programmatic stream-serialisation attribute (see dependency_wait in the kernels):
-// the kernel must call dependency_wait() before it touches anything but the metadata image.
+// the kernel must call dependency_wait() before its first access to global memory.
 template <class... Params, class... Args>
 int launch_overlapped(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args)
 {
@@ -2099,6 +2096,8 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
     __shared__ __align__(16) uint16_t kp_s[kMaxPatterns];
     __shared__ uint32_t blk_s[kKvWarps][16];
     const int tid = static_cast<int>(threadIdx.x), lane = tid & 31, warp = tid >> 5;
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
     {
         const uint4* src_p = reinterpret_cast<const uint4*>(d_meta + kOffPattern);
         for (int i = tid; i < static_cast<int>(kPatternBytes / 16); i += kKvWarps * 32) reinterpret_cast<uint4*>(pat_s)[i] = src_p[i];
@@ -2108,8 +2107,6 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
         for (int i = tid; i < static_cast<int>(kEncKpBytes / 16); i += kKvWarps * 32) reinterpret_cast<uint4*>(kp_s)[i] = src_k[i];
     }
     __syncthreads();
-    dependency_wait();                                     // the values may come from the previous kernel of the stream
-    release_dependents();
     const DevHeader* hdr = reinterpret_cast<const DevHeader*>(d_meta);
     const int S = hdr->S;
     const float T = hdr->T, invT = 1.0f / T;             // both exact powers of two
