@@ -438,6 +438,28 @@ def run_ours(args):
     if os.path.exists(tp):
         with open(tp) as f:
             traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
+    # What really limits the decoder are the SM's issue slots and its load/store pipe.  Their ceilings come from the
+    # unit counts and the clock (4 warp instructions and 1 wavefront per clock per SM); the per-symbol costs are ncu
+    # counters of this kernel (profiles/), the symbol rate is this run's.
+    sm_limits = None
+    cp = os.path.join(ROOT, "profiles", "decompress_sm_counters.json")
+    if os.path.exists(cp) and dec_ms > 0:
+        with open(cp) as f:
+            c = json.load(f)
+        props = torch.cuda.get_device_properties(local)
+        sms, ghz = props.multi_processor_count, (clocks or {}).get("sm_mhz", 0) / 1e3
+        if ghz > 0:
+            warp_symbols_per_s = groups * (G / 32) * args.steps / (dec_ms / 1e3)
+            sm_limits = {
+                "issue": {"bound": "alu", "unit": "G warp-instr/s", "peak": sms * 4 * ghz,
+                          "achieved": warp_symbols_per_s * c["warp_instructions_per_warp_symbol"] / 1e9},
+                "lsu": {"bound": "lsu", "unit": "G wavefronts/s", "peak": sms * 1 * ghz,
+                        "achieved": warp_symbols_per_s * c["lsu_wavefronts_per_warp_symbol"] / 1e9},
+                "per_warp_symbol": {"instructions": c["warp_instructions_per_warp_symbol"], "wavefronts": c["lsu_wavefronts_per_warp_symbol"]},
+                "source": "profiles/decompress_sm_counters.json; peaks = SMs x units x sampled SM clock",
+            }
+            for k in ("issue", "lsu"):
+                sm_limits[k]["frac"] = sm_limits[k]["achieved"] / sm_limits[k]["peak"]
     # the fused kernels against the same HBM peak (algorithmic bytes: blocks + vectors + results); what bounds them
     # is the SM load/store pipe, so the symbol rate is reported next to the HBM fraction
     seg_total = dec_ms + g1_ms + g8_ms + at_ms + av_ms + kc_ms
@@ -478,6 +500,8 @@ def run_ours(args):
                      "note": "kernel of the headline metric; limited by the SM load/store pipe, see kernels[] and profiles/"},
         "kernels": kernels,
     }
+    if sm_limits is not None:
+        line["sm_limits"] = sm_limits
     if "decompress" not in segs:
         # a diagnostic run without the headline segment has no headline number
         line["value"] = None
