@@ -47,6 +47,8 @@ def parse_args():
                          "sweep; cfg5: long-context GQA K cache [16][8][32768][128] (decompress + attention scores with 8 "
                          "query heads per KV head); act2x: the 2x activation codec on a [32768][8192] fp16 tensor; var: the "
                          "variable-length container on the cfg2 gate/up/down matrices")
+    ap.add_argument("--decompress-calls", choices=["batch", "single"], default="batch",
+                    help="decompress segment: one ecco_decompress_batch call over the step's tensors (default) or one ecco_decompress per tensor")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -196,7 +198,7 @@ def cpu_baseline(layer, c: int):
 WORKLOADS = {
     "cfg2": dict(label="cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
                        "+ cfg3 K and V caches [8][32][4096][128]",
-                 step="decompress x7, gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache); --only kvcomp times ecco_kv_compress over the whole K cache",
+                 step="decompress of the 7 matrices (one ecco_decompress_batch call), gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache); --only kvcomp times ecco_kv_compress over the whole K cache",
                  l2="inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
     "cfg4": dict(label="cfg4 llama-70b-shaped MLP weights (gate, up 28672x8192; down 8192x28672; 5,505,024 groups)",
                  step="decompress x3, gemv batch 1 x3; plus a decompress sweep over 64 MiB .. 4 GiB streams (stream_sweep)",
@@ -279,9 +281,18 @@ def run_ours(args):
             kv["out"] = torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")
             dec.append(kv)
 
-    def seg_decompress():
+    dec_items = [(d["meta"], d["blocks"], d["n"], d["out"]) for d in dec]
+
+    def seg_decompress_single():
         for d in dec:
             B.ecco_decompress(d["meta"], d["blocks"], d["n"], d["out"], stream)
+
+    def seg_decompress():
+        # the tensors of a layer are decompressed together: one ecco_decompress_batch call (one launch per 8 tensors)
+        if args.decompress_calls == "batch":
+            B.ecco_decompress_batch(dec_items, stream)
+        else:
+            seg_decompress_single()
 
     def seg_gemv(b):
         for d in mats:
@@ -428,8 +439,24 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
+    # the same tensors through one ecco_decompress call each, for the record
+    single_us = None
+    if "decompress" in segs and dec and args.decompress_calls == "batch":
+        for _ in range(3):
+            seg_decompress_single()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(3, min(args.steps, 20))
+        barrier()
+        s0.record(stream)
+        for _ in range(reps):
+            seg_decompress_single()
+        s1.record(stream)
+        barrier()
+        (sms_,) = distutil.max_over_ranks([s0.elapsed_time(s1)], dist, "cuda")
+        single_us = sms_ * 1e3 / reps
+
     peak, peak_kind = measured_peaks()
-    n_launch = max(1, len(dec))
+    n_launch = max(1, -(-len(dec) // 8) if args.decompress_calls == "batch" else len(dec))
     avg_launch_s = dec_ms / 1e3 / (args.steps * n_launch) if dec_ms > 0 else float("nan")
     alg_bytes_per_launch = groups * (BLOCK + G * 2) / n_launch
     achieved = alg_bytes_per_launch / avg_launch_s / 1e9 if dec_ms > 0 else 0.0
@@ -492,6 +519,7 @@ def run_ours(args):
         "segments_us_per_step": {"decompress": dec_ms / args.steps * 1e3, "gemv_batch1": g1_ms / args.steps * 1e3,
                                  "gemv_batch8": g8_ms / args.steps * 1e3, "attn_scores": at_ms / args.steps * 1e3,
                                  "attn_values": av_ms / args.steps * 1e3, "kv_compress": kc_ms / args.steps * 1e3},
+        "decompress_one_call_per_tensor_us": single_us,
         "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3 if wname == "cfg2" else None,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",

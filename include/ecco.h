@@ -125,6 +125,20 @@ int ecco_meta_serialize_device(const ecco_meta* meta, void* host_staging, size_t
  * clipped positions read +0.  n_groups == 0 is a no-op. */
 int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out_fp16, void* stream);
 
+/* The same for several tensors in one call (the seven matrices of a decoder layer, the K and V caches of a
+ * layer): the effect is that of ecco_decompress on every item in order, but tensors of 32 groups or more share
+ * one kernel launch per 8 items, in which every SM moves on to the next tensor as soon as it is done with its
+ * share of the current one, so launch latency and tail are paid once.  `items` is a HOST array read before the
+ * call returns; every item has its own metadata image; items with n_groups == 0 are skipped.  Errors are those
+ * of ecco_decompress and are found before anything is launched. */
+typedef struct ecco_decompress_item {
+    const void* d_meta;        /* device: metadata image of this tensor */
+    const uint8_t* d_blocks;   /* device: 64 * n_groups bytes */
+    uint64_t n_groups;
+    void* d_out_fp16;          /* device: 128 * n_groups fp16 values */
+} ecco_decompress_item;
+int ecco_decompress_batch(const ecco_decompress_item* items, int32_t n_items, void* stream);
+
 /* Decode-phase GEMV on compressed weights (Sec. 2.1: M = 1 matrix-vector products; Sec. 4.2
  * decode): y[b][n] = sum_k W~[n][k] * x[b][k], fp32 accumulation.  W is row-major [n_out][k],
  * groups along k, block of (n, kblock) at byte 64*(n*(k/128) + kblock).  x is fp16 [batch][k],

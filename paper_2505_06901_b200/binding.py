@@ -32,12 +32,17 @@ ERR_DEVICE_TIMEOUT = -8
 
 EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
-    "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_gemv_workspace_bytes",
+    "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_decompress_batch", "ecco_gemv_workspace_bytes",
     "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
     "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress",
     "ecco_var_stream_bytes_bound", "ecco_var_index_bytes", "ecco_var_encode_host", "ecco_var_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count",
 ]
+
+
+class DecompressItem(C.Structure):
+    """ecco_decompress_item of include/ecco.h."""
+    _fields_ = [("d_meta", C.c_void_p), ("d_blocks", C.c_void_p), ("n_groups", C.c_uint64), ("d_out_fp16", C.c_void_p)]
 
 
 class EccoError(RuntimeError):
@@ -86,6 +91,7 @@ def lib():
         L.ecco_meta_device_bytes.restype = sz
         L.ecco_meta_serialize_device.argtypes = [vp, vp, sz]
         L.ecco_decompress.argtypes = [vp, vp, u64, vp, vp]
+        L.ecco_decompress_batch.argtypes = [C.POINTER(DecompressItem), i32, vp]
         L.ecco_gemv_workspace_bytes.argtypes = [i32, i32, i32]
         L.ecco_gemv_workspace_bytes.restype = sz
         L.ecco_gemv.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, vp]
@@ -251,6 +257,14 @@ def meta_to_device(meta: Meta, device="cuda"):
 def ecco_decompress(d_meta, d_blocks, n_groups: int, d_out_fp16, stream=None) -> None:
     _check(lib().ecco_decompress(_ptr(d_meta), _ptr(d_blocks), n_groups, _ptr(d_out_fp16), _stream(stream)),
            "ecco_decompress")
+
+
+def ecco_decompress_batch(items, stream=None) -> None:
+    """items: sequence of (d_meta, d_blocks, n_groups, d_out_fp16); one call for all of them (see include/ecco.h)."""
+    arr = (DecompressItem * max(len(items), 1))()
+    for i, (d_meta, d_blocks, n_groups, d_out) in enumerate(items):
+        arr[i].d_meta, arr[i].d_blocks, arr[i].n_groups, arr[i].d_out_fp16 = _ptr(d_meta), _ptr(d_blocks), n_groups, _ptr(d_out)
+    _check(lib().ecco_decompress_batch(arr, len(items), _stream(stream)), "ecco_decompress_batch")
 
 
 def ecco_gemv_workspace_bytes(n_out: int, k: int, batch: int) -> int:

@@ -24,6 +24,7 @@
 #include <atomic>
 #include <cstdint>
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 
 #include "../../include/ecco.h"
@@ -165,14 +166,14 @@ __device__ __forceinline__ void issue_tables(uint8_t* smem, const uint8_t* d_met
         bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kTableBytes, bar);
     }
 }
-__device__ __forceinline__ bool wait_tables(uint64_t* bar_storage)
+__device__ __forceinline__ bool wait_tables(uint64_t* bar_storage, uint32_t parity = 0)
 {
     const uint32_t bar = smem_u32(bar_storage);
     __syncthreads();                             // the barrier word is initialised
     bool done = false;
-    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, parity);
     if (!done)                                   // second, bounded chance for the copy in flight
-        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, 0);
+        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, parity);
     const bool all = __syncthreads_and(done);
     if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
     return all;
@@ -193,12 +194,14 @@ __device__ __forceinline__ void release_dependents() { asm volatile("griddepcont
 // Same for the mixed decoder: patterns and ID_KP table, then rank tables and arithmetic constants
 // (adjacent in the image and in shared memory), two bulk copies on one barrier.  In two halves so
 // that the caller can put work between the issue and the wait.
-__device__ __forceinline__ void issue_rank_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage)
+__device__ __forceinline__ void issue_rank_tables(uint8_t* smem, const uint8_t* d_meta, uint64_t* bar_storage, bool first = true)
 {
     const uint32_t bar = smem_u32(bar_storage);
     if (threadIdx.x == 0) {
-        mbar_init(bar, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (first) {                             // later phases of the same barrier only re-arm it
+            mbar_init(bar, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
         mbar_expect_tx(bar, kPatternBytes + kKpLutBytes + kRankLutBytes + kArithBytes);
         bulk_g2s(smem_u32(smem), d_meta + kOffPattern, kPatternBytes + kKpLutBytes, bar);
         bulk_g2s(smem_u32(smem) + kSmemSymLut, d_meta + kOffRankLut, kRankLutBytes + kArithBytes, bar);
@@ -421,10 +424,28 @@ ecco_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __rest
 // tensor and drops rows past its end.  Outliers: those in the last tile (positions >= 112) are
 // patched in shared memory before that tile leaves; the others are 2-byte global stores issued
 // after the group's earlier tiles have been written (bulk wait + warp barrier), so they land last.
+// The kernel takes up to kMaxJobs tensors and works through them one after the other without leaving the SM:
+// between two tensors only the CTA's own warps meet (the tables are the CTA's), so an SM that is done with
+// one tensor starts the next while others still finish, and launch latency and tail are paid once per call.
+constexpr int kMaxJobs = 8;
+struct alignas(64) DecompressJob {
+    const uint8_t* meta;
+    const uint8_t* blocks;
+    uint64_t n_groups;
+    uint16_t* out;
+    uint32_t active_warps;     // working warps for this tensor: all get the same number of tiles
+    uint32_t reserved[7];
+    CUtensorMap map;           // [n_groups][128] fp16, box 32 x 16, 32-byte swizzle
+};
+struct DecompressBatch {
+    int32_t n;
+    int32_t reserved[15];
+    DecompressJob job[kMaxJobs];
+};
+
 template <int kWarps, uint32_t kArith, int kDecFree = 12>
 __global__ void __launch_bounds__(kWarps * 32, 1)
-ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, uint64_t n_groups,
-                           uint16_t* __restrict__ d_out, uint32_t active_warps, const __grid_constant__ CUtensorMap out_map)
+ecco_decompress_tma_kernel(const __grid_constant__ DecompressBatch batch)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
@@ -442,20 +463,28 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
     const uint32_t swz = ((lane >> 2) & 1u) << 4;                               // 32-byte swizzle: bit 4 ^= bit 7
     const uint32_t my_row = stage + lane * 32;
 
-    const uint64_t n_tiles = (n_groups + 31) / 32;
-    const uint64_t tile_stride = active_warps;             // see ecco_decompress_kernel
-    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
-    if (tile >= tile_stride) tile = n_tiles;
     dependency_wait();
     release_dependents();
-    issue_rank_tables(smem, d_meta, bar);
+  for (int t = 0; t < batch.n; ++t) {
+    const DecompressJob& job = batch.job[t];
+    const uint8_t* __restrict__ d_meta = job.meta;
+    const uint8_t* __restrict__ d_blocks = job.blocks;
+    const uint64_t n_groups = job.n_groups;
+    uint16_t* __restrict__ d_out = job.out;
+    const CUtensorMap& out_map = job.map;
+    const uint64_t n_tiles = (n_groups + 31) / 32;
+    const uint64_t tile_stride = job.active_warps;         // see ecco_decompress_kernel
+    uint64_t tile = static_cast<uint64_t>(warp) * gridDim.x + blockIdx.x;
+    if (tile >= tile_stride) tile = n_tiles;
+    if (t > 0) __syncthreads();                            // every warp is done with the previous tensor's tables
+    issue_rank_tables(smem, d_meta, bar, t == 0);
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
-    if (threadIdx.x < 256)                                 // visible after the barriers inside wait_rank_tables
+    if (threadIdx.x < 256)                                 // visible after the barriers inside wait_tables
         asm volatile("st.shared.u16 [%0], %1;" ::"r"(fp8tab + threadIdx.x * 2),
                      "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(threadIdx.x) * T))) : "memory");
     Block blk;
     if (tile < n_tiles) ldg_block(blk, d_blocks + min(tile * 32 + lane, n_groups - 1) * kBlockBytes);
-    if (!wait_tables(bar)) return;
+    if (!wait_tables(bar, static_cast<uint32_t>(t & 1))) return;
 
     for (; tile < n_tiles; tile += tile_stride) {
         const uint64_t g = tile * 32 + lane;
@@ -507,6 +536,7 @@ ecco_decompress_tma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __
         }
         send_tile(7);
     }
+  }
     if (lane == 0) bulk_wait_all();                        // shared memory must outlive the engine's reads
 }
 
@@ -1607,49 +1637,105 @@ constexpr int kDecompressTmaWarps = 28;
 // {none, one, two, three, all} on the 11008x4096 matrix and on a 256 MiB cache (all-table 441 us, this 394 us, all-arithmetic 459 us)
 constexpr uint32_t kDecompressArith = 0b1010;
 
-extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out, void* stream)
+// tensors of fewer than 32 groups (the tile store's box is 32 rows tall), or when no tensor map can be made
+static int launch_decompress_small(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out,
+                                   cudaStream_t stream)
 {
-    if (n_groups == 0) return ECCO_OK;
-    if (!d_meta || !d_blocks || !d_out) return ECCO_ERR_INVALID_ARG;
-    if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_out)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
-    DeviceInfo di;
-    int rc = device_info(&di);
-    if (rc) return rc;
     static thread_local bool configured[64] = {};
-    static thread_local bool configured_tma[64] = {};
-    // bulk-store variant for everything but tiny tensors (its box is 32 rows tall)
-    CUtensorMap map;
-    if (n_groups >= 32 && make_out_map(&map, d_out, n_groups)) {
-        auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps, kDecompressArith>;
-        constexpr size_t smem =
-            ((kSmemRankWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
-            static_cast<size_t>(kDecompressTmaWarps) * 1024 + 512 + 16;       // + outlier value table + barrier
-        static_assert(smem <= 232448, "227 KB per CTA");
-        if (!configured_tma[di.device]) {
-            rc = set_smem(kernel, smem);
-            if (rc) return rc;
-            configured_tma[di.device] = true;
-        }
-        const uint64_t cta_tiles = (n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
-        const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
-        const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kDecompressTmaWarps);
-        return launch_overlapped(kernel, grid, static_cast<unsigned>(kDecompressTmaWarps * 32), smem, static_cast<cudaStream_t>(stream),
-                                 static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out), active, map);
-    }
     auto kernel = ecco_decompress_kernel<kDecompressWarps>;
     const size_t smem = kSmemWarpBase + static_cast<size_t>(kDecompressWarps) * (kBitsBytes + kTabBytes);
     if (!configured[di.device]) {
-        rc = set_smem(kernel, smem);
+        int rc = set_smem(kernel, smem);
         if (rc) return rc;
         configured[di.device] = true;
     }
     const uint64_t cta_tiles = (n_groups + kDecompressWarps * 32 - 1) / (kDecompressWarps * 32);   // one tile per warp
     const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
-    kernel<<<grid, kDecompressWarps * 32, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const uint8_t*>(d_meta), d_blocks, n_groups, static_cast<uint16_t*>(d_out),
-        balanced_warps((n_groups + 31) / 32, grid * kDecompressWarps));
+    kernel<<<grid, kDecompressWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_groups,
+                                                          static_cast<uint16_t*>(d_out),
+                                                          balanced_warps((n_groups + 31) / 32, grid * kDecompressWarps));
     return check_launch();
+}
+
+// one launch of the tile-store kernel over batch.n tensors (maps already made)
+static int launch_decompress_batch(const DeviceInfo& di, DecompressBatch& batch, cudaStream_t stream)
+{
+    static thread_local bool configured[64] = {};
+    auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps, kDecompressArith>;
+    constexpr size_t smem =
+        ((kSmemRankWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
+        static_cast<size_t>(kDecompressTmaWarps) * 1024 + 512 + 16;           // + outlier value table + barrier
+    static_assert(smem <= 232448, "227 KB per CTA");
+    if (!configured[di.device]) {
+        int rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    uint64_t cta_tiles = 0;
+    for (int t = 0; t < batch.n; ++t) {
+        const uint64_t c = (batch.job[t].n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
+        cta_tiles = c > cta_tiles ? c : cta_tiles;
+    }
+    const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
+    for (int t = 0; t < batch.n; ++t)
+        batch.job[t].active_warps = balanced_warps((batch.job[t].n_groups + 31) / 32, grid * kDecompressTmaWarps);
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kDecompressTmaWarps * 32), smem, stream, batch);
+}
+
+static int check_decompress_args(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, const void* d_out)
+{
+    if (!d_meta || !d_blocks || !d_out) return ECCO_ERR_INVALID_ARG;
+    if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_out)) return ECCO_ERR_ALIGNMENT;
+    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    return ECCO_OK;
+}
+
+extern "C" int ecco_decompress_batch(const ecco_decompress_item* items, int32_t n_items, void* stream)
+{
+    if (n_items < 0 || (n_items > 0 && !items)) return ECCO_ERR_INVALID_ARG;
+    for (int i = 0; i < n_items; ++i) {                    // nothing is launched unless every item is acceptable
+        if (items[i].n_groups == 0) continue;
+        const int rc = check_decompress_args(items[i].d_meta, items[i].d_blocks, items[i].n_groups, items[i].d_out_fp16);
+        if (rc) return rc;
+    }
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    DecompressBatch batch;
+    std::memset(&batch, 0, sizeof batch);
+    for (int i = 0; i < n_items; ++i) {
+        const ecco_decompress_item& it = items[i];
+        if (it.n_groups == 0) continue;
+        DecompressJob& job = batch.job[batch.n];
+        if (it.n_groups >= 32 && make_out_map(&job.map, it.d_out_fp16, it.n_groups)) {
+            job.meta = static_cast<const uint8_t*>(it.d_meta);
+            job.blocks = it.d_blocks;
+            job.n_groups = it.n_groups;
+            job.out = static_cast<uint16_t*>(it.d_out_fp16);
+            if (++batch.n == kMaxJobs) {
+                rc = launch_decompress_batch(di, batch, s);
+                if (rc) return rc;
+                batch.n = 0;
+            }
+        } else {                                           // items keep their order in the stream
+            if (batch.n) {
+                rc = launch_decompress_batch(di, batch, s);
+                if (rc) return rc;
+                batch.n = 0;
+            }
+            rc = launch_decompress_small(di, it.d_meta, it.d_blocks, it.n_groups, it.d_out_fp16, s);
+            if (rc) return rc;
+        }
+    }
+    return batch.n ? launch_decompress_batch(di, batch, s) : ECCO_OK;
+}
+
+extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out, void* stream)
+{
+    if (n_groups == 0) return ECCO_OK;
+    const ecco_decompress_item item = {d_meta, d_blocks, n_groups, d_out};
+    return ecco_decompress_batch(&item, 1, stream);
 }
 
 constexpr int kVarWarps = 18;

@@ -182,6 +182,45 @@ def test_decompress_adversarial_codebooks(B, eo):
     assert_bit_exact(gpu_decompress(B, lib_meta_from_oracle(B, m3), rb), eo.decode(m3, rb))
 
 
+def test_decompress_batch_matches_oracle_per_item(B, eo, cfg1_small, kv_small, synth):
+    """One call over tensors with different metadata and sizes: every item as ecco_decompress alone would give it.
+    Covers more than eight items (two launches), an empty item, tiny items (the small-tensor kernel in the middle
+    of the batch), a ragged tail and the same output written by two items (the later one wins)."""
+    wm, km = cfg1_small["meta"], kv_small["meta"]
+    d_wm, d_km = B.meta_to_device(lib_meta_from_oracle(B, wm)), B.meta_to_device(lib_meta_from_oracle(B, km))
+    wb, kb = cfg1_small["blocks"], kv_small["blocks"]
+    rb = synth.random_blocks(700, 5)
+    plan = [(wm, d_wm, np.tile(wb, (3, 1))), (km, d_km, kb), (wm, d_wm, wb[:0]), (wm, d_wm, wb[:7]), (km, d_km, kb[:33]),
+            (wm, d_wm, rb), (km, d_km, np.tile(kb, (2, 1))[:4095]), (wm, d_wm, wb[:1]), (km, d_km, kb[100:1124]),
+            (wm, d_wm, wb[5:1030]), (km, d_km, kb[:31])]
+    items, outs = [], []
+    for meta, d_meta, blocks in plan:
+        n = blocks.shape[0]
+        d_b = dev(blocks) if n else torch.empty((1, 64), dtype=torch.uint8, device="cuda")
+        d_o = torch.full((max(n, 1) * 128,), float("nan"), dtype=torch.float16, device="cuda")
+        items.append((d_meta, d_b, n, d_o))
+        outs.append(d_o)
+    shared = torch.zeros(2048 * 128, dtype=torch.float16, device="cuda")          # written twice: kv item last
+    items.append((d_wm, dev(wb), 2048, shared))
+    items.append((d_km, dev(kb), 2048, shared))
+    B.ecco_decompress_batch(items)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    for (meta, _, blocks), d_o in zip(plan, outs):
+        n = blocks.shape[0]
+        if n:
+            assert_bit_exact(d_o[: n * 128].cpu().numpy().reshape(n, 128), eo.decode(meta, blocks))
+    assert_bit_exact(shared.cpu().numpy().reshape(2048, 128), eo.decode(km, kb))
+    B.ecco_decompress_batch([])                                                   # nothing to do is not an error
+    # one bad item stops the whole call before anything runs
+    canary = torch.full((2048 * 128,), 7.0, dtype=torch.float16, device="cuda")
+    with pytest.raises(B.EccoError) as ei:
+        B.ecco_decompress_batch([(d_wm, dev(wb), 2048, canary), (d_wm, dev(wb).data_ptr() + 8, 2048, canary)])
+    assert ei.value.code == B.ERR_ALIGNMENT
+    torch.cuda.synchronize()
+    assert bool((canary == 7.0).all())
+
+
 def test_decompress_rejects_bad_arguments_on_device(B, cfg1_small):
     lm = lib_meta_from_oracle(B, cfg1_small["meta"])
     d_meta, d_blocks = B.meta_to_device(lm), dev(cfg1_small["blocks"])
