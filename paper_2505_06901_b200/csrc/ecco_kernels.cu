@@ -2098,18 +2098,20 @@ ecco_act_compress_kernel(const uint4* __restrict__ d_x, uint64_t n_chunks, uint4
         uint32_t out[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            uint32_t wv = 0;
+            // clamping before the rounding gives what clamping after it gives (the bounds are integers, rounding is
+            // monotone); cvt.rni rounds to nearest even like rintf; two pack instructions make the four bytes
+            int q[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                const int e = i * 4 + j;
-                int q = 0;
-                if (usable) {
-                    const float rr = rintf(__fmul_rn(x[e] - zero, inv));
-                    q = static_cast<int>(fminf(fmaxf(rr, -64.0f), 63.0f));
-                }
-                wv |= ((static_cast<uint32_t>(q) & 0x7fu) | (((meta16 >> e) & 1u) << 7)) << (8 * j);
+                const float p = fminf(fmaxf(__fmul_rn(x[i * 4 + j] - zero, inv), -64.0f), 63.0f);
+                q[j] = usable ? __float2int_rn(p) : 0;
             }
-            out[i] = wv;
+            uint32_t hi16, wv;                             // d = sat(a) << 8 | sat(b) | c << 16
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi16) : "r"(q[3]), "r"(q[2]), "r"(0));
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(wv) : "r"(q[1]), "r"(q[0]), "r"(hi16));
+            // bits 4i .. 4i+3 of the metadata go to bit 7 of bytes 0..3
+            const uint32_t m4 = (meta16 >> (4 * i)) & 15u;
+            out[i] = (wv & 0x7f7f7f7fu) | (((m4 * 0x00204081u) & 0x01010101u) << 7);
         }
         if (ok) d_blocks[c] = make_uint4(out[0], out[1], out[2], out[3]);
     }
