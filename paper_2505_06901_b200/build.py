@@ -9,7 +9,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libecco_b200.so")
 SOURCES = [os.path.join(CSRC, "ecco_kernels.cu"), os.path.join(CSRC, "ecco_host.cpp")]
-HEADERS = [os.path.join(CSRC, "ecco_format.h"), os.path.join(os.path.dirname(HERE), "include", "ecco.h")]
+HEADERS = [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if f.endswith((".h", ".cuh"))] + \
+          [os.path.join(os.path.dirname(HERE), "include", "ecco.h")]
 
 
 def nvcc_path() -> str:

@@ -1,0 +1,250 @@
+// ecco_attn_values_kernels.cuh -- K5: attention output over a compressed V cache
+// Part of the one translation unit ecco_kernels.cu; included from there only.
+#pragma once
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// K5: attention output over a compressed V cache (Eq. 3: softmax(QK^T / sqrt(d_k)) V).
+// out[b][hq][d] = sum_t p[b][hq][t] * V~[b][hq / q_per_kv][t][d] with p = softmax_t(scores).
+// A thread owns one token (one group) as in K3, but here the sum runs over tokens, i.e. across
+// lanes.  Pass 1 runs the serial Huffman chain and keeps only the 4-bit indices (syms[16][32]);
+// by then the end bit, hence the outliers, are known.  Pass 2 walks the eight 16-dim chunks: map
+// the indices through the lane's table, stage them in a [32 tokens][16 dims] fp16 tile (same
+// swizzle as the decompress staging tile), overwrite the outliers of that chunk in the tile, and
+// contract the tile on the tensor cores: (V tile)^T [16 dims x 32 tokens] x P^T [32 tokens x 8
+// heads] with mma.m16n8k16, fp32 accumulators (4 registers per 16 dims, 32 for the 128 dims).  p is
+// split into an fp16 head and an fp16 remainder (two MMAs) so that its rounding does not show.
+// The result does not depend on scheduling.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+ecco_softmax_stats_kernel(const float* __restrict__ d_scores, int rows, int seq, float2* __restrict__ d_stats)
+{
+    const int row = static_cast<int>(blockIdx.x) * 8 + static_cast<int>(threadIdx.x >> 5), lane = static_cast<int>(threadIdx.x & 31u);
+    dependency_wait();                                     // the scores may come from the previous kernel of the stream
+    release_dependents();
+    if (row >= rows) return;
+    const float* s = d_scores + static_cast<size_t>(row) * seq;
+    float mx = -INFINITY;
+    for (int t = lane; t < seq; t += 32) mx = fmaxf(mx, s[t]);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float sum = 0.0f;
+    for (int t = lane; t < seq; t += 32) sum += expf(s[t] - mx);
+#pragma unroll
+    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    if (lane == 0) d_stats[row] = make_float2(mx, 1.0f / sum);
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3])
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+
+constexpr uint32_t kAvWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;   // + the [32][16] fp16 tile
+
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_vblocks, int heads, int seq,
+                        int q_per_kv, const float* __restrict__ d_scores, const float2* __restrict__ d_stats,
+                        float* __restrict__ d_out, float* __restrict__ d_partial, unsigned int* __restrict__ d_tickets)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    __shared__ unsigned int ticket;
+    __shared__ float2 stats_s[8];
+    constexpr int kTokens = kWarps * 32;
+    const uint32_t smem_base = smem_u32(smem);
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const int tid = static_cast<int>(threadIdx.x);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kAvWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kAvWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+    const uint32_t swz = ((lane >> 2) & 1u) << 4;
+    const uint32_t my_row = stage + lane * 32;
+    float* out_s = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kAvWarpBytes);    // [128 dims][8 heads]
+
+    const int G = gridDim.x, c = blockIdx.x;
+    const int chunks = (seq + kTokens - 1) / kTokens;
+    const int64_t U = static_cast<int64_t>(heads) * chunks;
+    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
+    auto block_ptr = [&](int64_t u) {
+        const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
+        return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    };
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    issue_tables(smem, d_meta, &bar);
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    float acc[8][4];                                       // [16-dim chunk][mma accumulator]
+    auto clear_acc = [&]() {
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+    };
+    clear_acc();
+
+    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in warp order, then
+    // either store (this CTA owns the whole head) or hand a partial to the slot-and-ticket reduction
+    auto flush = [&](int bh) {
+        for (int i = tid; i < kGroup * 8; i += kTokens) out_s[i] = 0.0f;
+        __syncthreads();
+        for (int w = 0; w < kWarps; ++w) {
+            if (static_cast<int>(warp) == w) {
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch)
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
+                        const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
+                        out_s[dim * 8 + head] += acc[ch][j];
+                    }
+            }
+            __syncthreads();
+        }
+        const int c_lo = unit_owner(U, G, static_cast<int64_t>(bh) * chunks);
+        const int c_hi = unit_owner(U, G, static_cast<int64_t>(bh + 1) * chunks - 1);
+        if (c_lo == c_hi) {
+            for (int i = tid; i < kGroup * 8; i += kTokens) {
+                const int dim = i >> 3, r = i & 7;
+                if (r < q_per_kv) d_out[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + dim] = out_s[i];
+            }
+        } else {
+            float* mine = d_partial + static_cast<size_t>(c + bh) * (kGroup * 8);
+            for (int i = tid; i < kGroup * 8; i += kTokens) mine[i] = out_s[i];
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) ticket = atomicAdd(&d_tickets[bh], 1u);
+            __syncthreads();
+            if (ticket == static_cast<unsigned int>(c_hi - c_lo)) {
+                __threadfence();
+                for (int i = tid; i < kGroup * 8; i += kTokens) {
+                    const int dim = i >> 3, r = i & 7;
+                    if (r >= q_per_kv) continue;
+                    float sum = 0.0f;
+                    for (int cc = c_lo; cc <= c_hi; ++cc) sum += __ldcg(d_partial + static_cast<size_t>(cc + bh) * (kGroup * 8) + i);
+                    d_out[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + dim] = sum;
+                }
+                if (tid == 0) d_tickets[bh] = 0;
+            }
+        }
+        __syncthreads();
+    };
+
+    int cur_bh = -1;
+    for (int64_t u = u0; u < u1; ++u) {
+        const int bh = static_cast<int>(u / chunks);
+        const int tile_base = static_cast<int>(u % chunks) * kTokens + static_cast<int>(warp) * 32;
+        const int t = tile_base + static_cast<int>(lane);
+        if (bh != cur_bh) {
+            if (cur_bh >= 0) { flush(cur_bh); clear_acc(); }
+            if (tid < 8) stats_s[tid] = tid < q_per_kv ? d_stats[static_cast<size_t>(bh) * q_per_kv + tid] : make_float2(0.0f, 0.0f);
+            __syncthreads();
+            cur_bh = bh;
+        }
+        // P^T fragments (B operand): head = lane / 4, tokens (lane % 4) * 2 + {0, 1} + 8 j
+        uint32_t p_hi[4], p_lo[4];
+        {
+            const int r = static_cast<int>(lane >> 2);
+            const float2 st = stats_s[r];
+            const float* srow = d_scores + (static_cast<size_t>(bh) * q_per_kv + min(r, q_per_kv - 1)) * seq;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int tk = tile_base + static_cast<int>(lane & 3u) * 2 + 8 * j;
+                float p0 = 0.0f, p1 = 0.0f;
+                if (r < q_per_kv && tk < seq) p0 = __expf(srow[tk] - st.x) * st.y;
+                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(srow[tk + 1] - st.x) * st.y;
+                const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
+                const __half l0 = __float2half_rn(p0 - __half2float(h0)), l1 = __float2half_rn(p1 - __half2float(h1));
+                p_hi[j] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);
+                p_lo[j] = static_cast<uint32_t>(__half_as_ushort(l0)) | (static_cast<uint32_t>(__half_as_ushort(l1)) << 16);
+            }
+        }
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        const bool valid = t < seq;                        // lanes past the end stage zeros (their p is zero too)
+        const GroupHeader h = open_group<false>(cur, smem_base, ws, T);
+        // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
+        uint32_t packed = 0;
+        int n_fit = kGroup;
+        const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+            if (!alive) n_fit = min(n_fit, n);             // only the clip path can see alive == false
+            packed |= sym << ((n & 7) * 4);
+            if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+        });
+        if (!valid) n_fit = 0;
+        // outliers of a complete group: which 16-dim chunks they fall into
+        const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
+        uint64_t pads_lo = 0, pads_hi = 0;                 // 16 bits per chunk: which pads fall into it
+        for (int j = 0; j < n_pad; ++j) {
+            const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
+            const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
+            if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+        }
+        // pass 2: per 16-dim chunk map the indices, patch the outliers in the tile, contract on the tensor cores
+        for (int ch = 0; ch < 8; ++ch) {
+            uint32_t r8[8];
+            const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
+            const bool whole = ch * 16 + 16 <= n_fit;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+                const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
+                uint32_t v = lds_u32(ws.tab + sym * 128);
+                if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;      // clipped positions (and lanes past the end) are +0
+                if (i & 1) r8[i >> 1] |= v << 16; else r8[i >> 1] = v;
+            }
+            __syncwarp();                                  // the previous tile has been read
+            sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
+            sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
+            uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
+            while (mine) {                                 // ascending: a later pad overrides an earlier one
+                const int j = __ffs(static_cast<int>(mine)) - 1;
+                mine &= mine - 1;
+                const uint32_t f = read_pad(ws, j);
+                const uint32_t byte = (f & 15u) * 2;
+                asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
+                             "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
+            }
+            __syncwarp();                                  // tile complete
+            uint32_t a[2][4];
+#pragma unroll
+            for (int ks = 0; ks < 2; ++ks) {
+                const uint32_t tok = (lane >> 4) * 8 + (lane & 7u) + 16 * ks, half = (lane >> 3) & 1u;
+                ldmatrix_x4_trans(a[ks], stage + tok * 32 + ((half ^ ((tok >> 2) & 1u)) << 4));
+            }
+            // ch is uniform but not a compile-time constant: pick the accumulator set by uniform branches so
+            // that it stays in registers
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (ch == k) {
+#pragma unroll
+                    for (int ks = 0; ks < 2; ++ks) {
+                        mma_16816(acc[k], a[ks], p_hi[2 * ks], p_hi[2 * ks + 1]);
+                        mma_16816(acc[k], a[ks], p_lo[2 * ks], p_lo[2 * ks + 1]);
+                    }
+                }
+            }
+        }
+    }
+    if (cur_bh >= 0) flush(cur_bh);
+}
+
+
+}  // namespace

@@ -1,0 +1,255 @@
+// ecco_fused_mma_kernels.cuh -- K2m / K3m: fused GEMV and attention scores for three to eight dot products per group (tensor cores)
+// Part of the one translation unit ecco_kernels.cu; included from there only.
+#pragma once
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// K2m / K3m: the fused consumers for 3 to 8 dot products per group (rows of x, query heads) on the
+// tensor cores.  With eight products per weight the scalar path spends four shared-memory
+// wavefronts and eight FMAs per symbol on the vector operand alone.  Here a group is decoded in
+// two passes as in K5 (indices first; then per 16 values: map, stage a [32 rows][16 k] fp16 tile,
+// patch its outliers) and each tile is contracted against the fp16 vector fragments, which stay
+// in registers for the whole group: C[32 rows][8] += tile[32 x 16] * V[16 x 8], two
+// mma.m16n8k16 per tile, fp32 accumulate (fp16 x fp16 products are exact in fp32).  A warp is
+// independent of the others: no vector slice in shared memory, no block barrier.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];" : "=r"(a[0]), "=r"(a[1]), "=r"(a[2]), "=r"(a[3]) : "r"(addr));
+}
+
+// Position i (0..15) of a 16-value chunk is staged in tile column 2q + (j & 1) + 8 (j >> 1) with i = 4q + j.  The
+// contraction index of an MMA may be permuted freely as long as both operands agree, and with this
+// order the four vector elements a lane needs per chunk (columns 2q, 2q+1, 2q+8, 2q+9) are the
+// contiguous k = 4q .. 4q+3: one 8-byte load instead of two 4-byte ones.
+__host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i & 1) + 8 * ((i >> 1) & 1); }
+
+// vfrag[2c], vfrag[2c+1]: B fragments of chunk c (tile columns (lane%4)*2 + {0,1}, and + 8), vector lane/4
+// acc[0] / acc[1]: C fragments of rows 0..15 / 16..31 of the warp's 32 groups
+__device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base, const WarpSmem& ws, uint32_t stage, float T,
+                                            bool valid, const uint32_t (&vfrag)[16], float (&acc)[2][4])
+{
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = stage + lane * 32;
+    const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
+    uint32_t packed = 0;
+    int n_fit = kGroup;
+    const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+        if (!alive) n_fit = min(n_fit, n);
+        packed |= sym << ((n & 7) * 4);
+        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+    });
+    if (!valid) n_fit = 0;                                 // rows past the end contribute zeros
+    const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
+    uint64_t pads_lo = 0, pads_hi = 0;                     // 16 bits per chunk: which pads fall into it
+    for (int j = 0; j < n_pad; ++j) {
+        const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
+        const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
+        if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+    }
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        uint32_t r8[8];
+        const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
+        const bool whole = ch * 16 + 16 <= n_fit;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
+            uint32_t v = lds_u32(ws.tab + sym * 128);
+            if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;
+            const int col = tile_column(i);                // see load_vfrag
+            if (col & 1) r8[col >> 1] |= v << 16; else r8[col >> 1] = v;
+        }
+        __syncwarp();                                      // the previous tile has been read
+        sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
+        sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
+        uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
+        while (mine) {                                     // ascending: a later pad overrides an earlier one
+            const int j = __ffs(static_cast<int>(mine)) - 1;
+            mine &= mine - 1;
+            const uint32_t f = read_pad(ws, j);
+            const uint32_t byte = static_cast<uint32_t>(tile_column(static_cast<int>(f & 15u))) * 2;
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
+                         "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
+        }
+        __syncwarp();                                      // tile complete
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt) {
+            const uint32_t row = ((lane >> 3) & 1u) * 8 + (lane & 7u) + 16 * mt, half = lane >> 4;
+            uint32_t a[4];
+            ldmatrix_x4(a, stage + row * 32 + ((half ^ ((row >> 2) & 1u)) << 4));
+            mma_16816(acc[mt], a, vfrag[2 * ch], vfrag[2 * ch + 1]);
+        }
+    }
+}
+
+// fragments of eight fp16 vectors v[col][k0 .. k0+127] (col = lane/4; columns >= n_cols are zero)
+__device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols)
+{
+    const int lane = static_cast<int>(threadIdx.x & 31u), col = lane >> 2;
+    const uint2* p = reinterpret_cast<const uint2*>(base + static_cast<size_t>(min(col, n_cols - 1)) * col_stride) + (lane & 3);
+#pragma unroll
+    for (int c = 0; c < 8; ++c) {
+        const uint2 v = col < n_cols ? __ldg(p + c * 4) : make_uint2(0u, 0u);     // k = 16c + 4 (lane%4) .. + 3
+        vfrag[2 * c] = v.x;                                // tile columns 2q, 2q+1
+        vfrag[2 * c + 1] = v.y;                            // tile columns 2q+8, 2q+9
+    }
+}
+
+// K2m: y[b][n] = sum_k W~[n][k] x[b][k] for 3..8 rows of x.  Units, ownership and the slot-and-ticket
+// reduction are those of the per-warp kernel (unit = 32 rows x one k-block).
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                     const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+                     unsigned int* __restrict__ d_tickets, int active_warps)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t smem_base = smem_u32(smem);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int tiles = (n_out + 31) / 32;
+    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    const int W = active_warps;
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    const int k = kblocks * kGroup;
+    auto block_ptr = [&](int64_t u) {
+        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
+        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
+    };
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    issue_tables(smem, d_meta, &bar);
+    Block blk;
+    uint32_t vnext[16];
+    if (u0 < u1) { ldg_block(blk, block_ptr(u0)); load_vfrag(vnext, d_x + static_cast<int>(u0 % kblocks) * kGroup, k, batch); }
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+    // C fragment element (mt, i): row = 16 mt + lane/4 + 8 (i >= 2), column b = (lane%4)*2 + (i & 1)
+    auto flush = [&](int tile) {
+        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
+        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
+        float* mine = d_partial + static_cast<size_t>(wg + tile) * 8 * 32;
+        if (w_lo != w_hi) {
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    mine[((lane & 3) * 2 + (i & 1)) * 32 + 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0)] = acc[mt][i];
+            __threadfence();
+            __syncwarp();
+            unsigned int t = 0;
+            if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+            t = __shfl_sync(0xffffffffu, t, 0);
+            if (t != static_cast<unsigned int>(w_hi - w_lo)) return;
+            __threadfence();
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int r = 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0), b = (lane & 3) * 2 + (i & 1);
+                const int row = tile * 32 + r;
+                float sum = acc[mt][i];
+                if (w_lo != w_hi) {                        // slots in warp order, whatever the arrival order
+                    sum = 0.0f;
+                    for (int ww = w_lo; ww <= w_hi; ++ww) sum += __ldcg(d_partial + (static_cast<size_t>(ww + tile) * 8 + b) * 32 + r);
+                }
+                if (row < n_out && b < batch) d_y[static_cast<size_t>(b) * n_out + row] = sum;
+            }
+        if (w_lo != w_hi && lane == 0) d_tickets[tile] = 0;
+    };
+
+    int cur_tile = static_cast<int>(u0 / kblocks);
+    for (int64_t u = u0; u < u1; ++u) {
+        const int tile = static_cast<int>(u / kblocks);
+        if (tile != cur_tile) {
+            flush(cur_tile);
+#pragma unroll
+            for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[mt][i] = 0.0f;
+            cur_tile = tile;
+        }
+        const Block cur = blk;
+        uint32_t vfrag[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) vfrag[i] = vnext[i];
+        if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_vfrag(vnext, d_x + static_cast<int>((u + 1) % kblocks) * kGroup, k, batch); }
+        row_dot_mma(cur, smem_base, ws, stage, T, tile * 32 + lane < n_out, vfrag, acc);
+    }
+    if (u0 < u1) flush(cur_tile);
+}
+
+// K3m: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for 3..8 query heads per KV head.
+// Unit = (one (batch, kv head), 32 tokens); every working warp owns a contiguous run of units.
+template <int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
+                            int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores,
+                            int active_warps)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    const uint32_t smem_base = smem_u32(smem);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    WarpSmem ws;
+    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int tiles = (seq + 31) / 32;
+    const int64_t U = static_cast<int64_t>(heads) * tiles;
+    const int W = active_warps;
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    auto block_ptr = [&](int64_t u) {
+        const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    };
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    issue_tables(smem, d_meta, &bar);
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    uint32_t vfrag[16];
+    int cur_bh = -1;
+    for (int64_t u = u0; u < u1; ++u) {
+        const int bh = static_cast<int>(u / tiles), t0 = static_cast<int>(u % tiles) * 32;
+        if (bh != cur_bh) { load_vfrag(vfrag, d_q + static_cast<size_t>(bh) * q_per_kv * kGroup, kGroup, q_per_kv); cur_bh = bh; }
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
+        row_dot_mma(cur, smem_base, ws, stage, T, t0 + lane < seq, vfrag, acc);
+#pragma unroll
+        for (int mt = 0; mt < 2; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int t = t0 + 16 * mt + (lane >> 2) + (i >= 2 ? 8 : 0), r = (lane & 3) * 2 + (i & 1);
+                if (t < seq && r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = scale * acc[mt][i];
+            }
+    }
+}
+
+
+}  // namespace

@@ -1,0 +1,305 @@
+// ecco_fused_scalar_kernels.cuh -- K2 / K3: fused GEMV and attention scores for one or two dot products per group
+// Part of the one translation unit ecco_kernels.cu; included from there only.
+#pragma once
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// K2/K3: fused consumers.  kV = number of dot products per group (batch rows of x, or query
+// heads per KV head).  The vector slice xs[128][kV] fp32 lives in shared memory; every lane reads
+// the same element at the same time (one broadcast wavefront), 16 bytes per load, so a slice
+// element costs 1/4 (kV = 1) to 2 (kV = 8) loads per symbol.
+// ---------------------------------------------------------------------------------------------
+template <int kV>
+struct Accum {
+    float a[kV];
+    float4 cache;                       // the current 16 bytes of the slice (kV <= 2)
+    __device__ __forceinline__ void clear()
+    {
+#pragma unroll
+        for (int v = 0; v < kV; ++v) a[v] = 0.0f;
+    }
+    static __device__ __forceinline__ float4 lds_f4(uint32_t addr)
+    {
+        float4 x;
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(x.x), "=f"(x.y), "=f"(x.z), "=f"(x.w) : "r"(addr));
+        return x;
+    }
+    // value w of position n (n is a compile-time constant after unrolling); xs = shared address of xs[0][0]
+    __device__ __forceinline__ void fma(int n, float w, uint32_t xs)
+    {
+        if constexpr (kV == 1) {
+            if ((n & 3) == 0) cache = lds_f4(xs + n * 4);
+            const float x = (n & 3) == 0 ? cache.x : (n & 3) == 1 ? cache.y : (n & 3) == 2 ? cache.z : cache.w;
+            a[0] = fmaf(w, x, a[0]);
+        } else if constexpr (kV == 2) {
+            if ((n & 1) == 0) cache = lds_f4(xs + n * 8);
+            a[0] = fmaf(w, (n & 1) ? cache.z : cache.x, a[0]);
+            a[1] = fmaf(w, (n & 1) ? cache.w : cache.y, a[1]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < kV / 4; ++q) {
+                const float4 x = lds_f4(xs + n * (kV * 4) + q * 16);
+                a[q * 4 + 0] = fmaf(w, x.x, a[q * 4 + 0]);
+                a[q * 4 + 1] = fmaf(w, x.y, a[q * 4 + 1]);
+                a[q * 4 + 2] = fmaf(w, x.z, a[q * 4 + 2]);
+                a[q * 4 + 3] = fmaf(w, x.w, a[q * 4 + 3]);
+            }
+        }
+    }
+    // out-of-order correction at a run-time position (outlier fix-up)
+    __device__ __forceinline__ void fma_at(uint32_t loc, float w, uint32_t xs)
+    {
+#pragma unroll
+        for (int v = 0; v < kV; ++v) {
+            float x;
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(x) : "r"(xs + (loc * kV + v) * 4));
+            a[v] = fmaf(w, x, a[v]);
+        }
+    }
+};
+
+// decode one group and accumulate its kV dot products against xs (shared address of xs[0][0])
+template <int kV>
+__device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T,
+                                            uint32_t xs, Accum<kV>& acc)
+{
+    const GroupHeader h = open_group<true, kFusedRank>(blk, smem_base, ws, T);
+    uint32_t packed = 0;
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedArith, kFusedFree>(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
+        acc.fma(n, __uint_as_float(v), xs);
+        packed |= sym << ((n & 7) * 4);
+        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+    });
+    if (end) {
+        // outliers replace the mapped value at their location: add (outlier - mapped) * x
+        const int n_pad = min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits));
+        uint64_t seen_lo = 0, seen_hi = 0;                  // 128-bit "already replaced" mask
+        for (int j = n_pad - 1; j >= 0; --j) {             // the last pad wins on a duplicate location
+            const uint32_t f = read_pad(ws, j);
+            const uint32_t loc = f & 127u;
+            const uint64_t bit = 1ull << (loc & 63u);
+            const bool upper = loc >= 64u;
+            if ((upper ? seen_hi : seen_lo) & bit) continue;
+            if (upper) seen_hi |= bit; else seen_lo |= bit;
+            const uint32_t word = lds_u32(ws.syms + (loc >> 3) * 128);
+            const uint32_t sym = (word >> ((loc & 7u) * 4)) & 15u;
+            const float mapped = __uint_as_float(lds_u32(ws.tab + sym * 128));
+            const float outlier = __half2float(__float2half_rn(fp8_to_float(f >> 7) * T));
+            acc.fma_at(loc, outlier - mapped, xs);
+        }
+    }
+}
+
+// Contiguous split of U work units over G CTAs: CTA c owns [unit_begin(c), unit_begin(c + 1)).
+__host__ __device__ __forceinline__ int64_t unit_begin(int64_t U, int G, int c) { return U * c / G; }
+__host__ __device__ __forceinline__ int unit_owner(int64_t U, int G, int64_t u)
+{
+    int c = static_cast<int>(u * G / U);
+    while (c + 1 < G && unit_begin(U, G, c + 1) <= u) ++c;
+    while (c > 0 && unit_begin(U, G, c) > u) --c;
+    return c;
+}
+
+template <int kWarps>
+__device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    WarpSmem ws;
+    ws.bits = smem_base + kFusedBase + warp * kWarpBytes + lane * 4;
+    ws.tab = ws.bits + kBitsBytes;
+    ws.syms = ws.tab + kTabBytes;
+    sts_u32(ws.bits + 16 * 128, 0u);
+    sts_u32(ws.bits + 17 * 128, 0u);
+    return ws;
+}
+
+// K2 for one or two rows of x: the slice is small enough (512 B or 1 KB) for every warp to keep
+// its own, so warps never meet at a barrier.  A work unit is (32 consecutive rows, one k-block),
+// numbered row-tile major; every working warp owns a contiguous run of units and keeps its rows'
+// partial sums in registers along k.  When a row tile is shared by several warps each writes its
+// partial sums to its own workspace slot (slot = global warp id + row tile: unique along the
+// staircase of (warp, tile) pairs) and the last to arrive (ticket counter) adds the slots in warp
+// order: the result does not depend on scheduling.  Workspace: partial[slot][kV][32] floats, then
+// one ticket per 32-row tile.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
+                      const __half* __restrict__ d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
+                      unsigned int* __restrict__ d_tickets, int active_warps)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    constexpr uint32_t kXsBytes = kGroup * kV * 4;
+    const uint32_t smem_base = smem_u32(smem);
+    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    const uint32_t xs = smem_base + kFusedBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
+
+    // W working warps (chosen by the host so that they all get the same number of units, and never
+    // more than there are units); warp ids interleave over the CTAs; the other warps idle
+    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int tiles = (n_out + 31) / 32;
+    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    const int W = active_warps;
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
+    const int k = kblocks * kGroup;
+    auto block_ptr = [&](int64_t u) {
+        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
+        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
+    };
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    Accum<kV> acc;
+    acc.clear();
+    auto flush = [&](int tile) {
+        const int row = tile * 32 + lane;
+        const bool row_ok = row < n_out;
+        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
+        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
+        if (w_lo == w_hi) {
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b) d_y[static_cast<size_t>(b) * n_out + row] = acc.a[b];
+            }
+            return;
+        }
+        float* mine = d_partial + static_cast<size_t>(wg + tile) * kV * 32;
+#pragma unroll
+        for (int b = 0; b < kV; ++b) mine[b * 32 + lane] = acc.a[b];
+        __threadfence();
+        __syncwarp();
+        unsigned int t = 0;
+        if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+        t = __shfl_sync(0xffffffffu, t, 0);
+        if (t == static_cast<unsigned int>(w_hi - w_lo)) {  // last of the warps that share this tile
+            __threadfence();
+            if (row_ok) {
+#pragma unroll
+                for (int b = 0; b < kV; ++b) {
+                    // slots are added in warp order whatever the arrival order; loads go out sixteen at a time
+                    const float* slot = d_partial + (static_cast<size_t>(w_lo + tile) * kV + b) * 32 + lane;
+                    float sum = 0.0f;
+                    int ww = w_lo;
+                    for (; ww + 16 <= w_hi + 1; ww += 16, slot += 16 * kV * 32) {
+                        float v[16];
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = __ldcg(slot + i * kV * 32);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) sum += v[i];
+                    }
+                    for (; ww <= w_hi; ++ww, slot += kV * 32) sum += __ldcg(slot);
+                    d_y[static_cast<size_t>(b) * n_out + row] = sum;
+                }
+            }
+            if (lane == 0) d_tickets[tile] = 0;
+        }
+    };
+
+    // x for a unit is fetched one unit ahead, like the block
+    uint2 xraw[kV];
+    auto load_x = [&](int64_t u) {
+        const int kb = static_cast<int>(u % kblocks);
+#pragma unroll
+        for (int b = 0; b < kV; ++b)
+            xraw[b] = __ldg(reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4));
+    };
+    if (u0 < u1) load_x(u0);
+    int cur_tile = static_cast<int>(u0 / kblocks);
+    for (int64_t u = u0; u < u1; ++u) {
+        const int tile = static_cast<int>(u / kblocks);
+        if (tile != cur_tile) { flush(cur_tile); acc.clear(); cur_tile = tile; }
+        // this warp's slice: lane l converts x[b][kb*128 + 4l .. 4l+3] to fp32, layout xs[i][b]
+        __syncwarp();
+        {
+            float v[kV][4];
+#pragma unroll
+            for (int b = 0; b < kV; ++b) {
+                const __half2 h0 = *reinterpret_cast<const __half2*>(&xraw[b].x), h1 = *reinterpret_cast<const __half2*>(&xraw[b].y);
+                v[b][0] = __low2float(h0); v[b][1] = __high2float(h0); v[b][2] = __low2float(h1); v[b][3] = __high2float(h1);
+            }
+            if constexpr (kV == 1) {
+                sts_v4(xs + lane * 16, __float_as_uint(v[0][0]), __float_as_uint(v[0][1]), __float_as_uint(v[0][2]), __float_as_uint(v[0][3]));
+            } else {
+                sts_v4(xs + lane * 32, __float_as_uint(v[0][0]), __float_as_uint(v[1][0]), __float_as_uint(v[0][1]), __float_as_uint(v[1][1]));
+                sts_v4(xs + lane * 32 + 16, __float_as_uint(v[0][2]), __float_as_uint(v[1][2]), __float_as_uint(v[0][3]), __float_as_uint(v[1][3]));
+            }
+        }
+        __syncwarp();
+        const Block cur = blk;
+        if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_x(u + 1); }
+        fused_group<kV>(cur, smem_base, ws, T, xs, acc);
+    }
+    if (u0 < u1) flush(cur_tile);
+}
+
+// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t].  A work unit is (one (batch, kv
+// head) pair, a chunk of kWarps*32 tokens); units are dealt to persistent CTAs in contiguous runs,
+// the query slice is restaged when the head changes, a thread owns one token.
+template <int kV, int kWarps>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
+                        int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
+{
+    extern __shared__ __align__(1024) uint8_t smem[];
+    __shared__ uint64_t bar;
+    constexpr int kTokens = kWarps * 32;
+    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+    const uint32_t smem_base = smem_u32(smem);
+    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
+    float* xs = reinterpret_cast<float*>(smem + kFusedBase + kWarps * kWarpBytes);
+    const uint32_t xs_addr = smem_u32(xs);
+
+    const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
+    const int chunks = (seq + kTokens - 1) / kTokens;
+    const int64_t U = static_cast<int64_t>(heads) * chunks;
+    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
+    // lanes past the end of the sequence decode its last token again and store nothing
+    auto block_ptr = [&](int64_t u) {
+        const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    };
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
+    Block blk;
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(&bar)) return;
+    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+
+    int cur_bh = -1;
+    for (int64_t u = u0; u < u1; ++u) {
+        const int bh = static_cast<int>(u / chunks), t = static_cast<int>(u % chunks) * kTokens + tid;
+        if (bh != cur_bh) {
+            __syncthreads();                               // everyone is done with the previous head's slice
+            // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
+            for (int i = tid; i < kGroup * kV; i += kTokens) {
+                const int r = i % kV, d = i / kV;
+                xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
+            }
+            __syncthreads();
+            cur_bh = bh;
+        }
+        const Block cur = blk;
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        Accum<kV> acc;
+        acc.clear();
+        fused_group<kV>(cur, smem_base, ws, T, xs_addr, acc);
+        if (t < seq) {
+#pragma unroll
+            for (int r = 0; r < kV; ++r)
+                if (r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = acc.a[r];
+        }
+    }
+}
+
+
+}  // namespace

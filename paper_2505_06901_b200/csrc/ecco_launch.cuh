@@ -1,0 +1,137 @@
+// ecco_launch.cuh -- host-side launch helpers: device query, overlapped launches, work plans
+// Part of the one translation unit ecco_kernels.cu; included from there only.
+#pragma once
+
+namespace {
+
+// ---------------------------------------------------------------------------------------------
+// host-side launch helpers
+// ---------------------------------------------------------------------------------------------
+// number of working warps <= w_max such that `units` split evenly: all get ceil(units / w_max) or one less
+inline uint32_t balanced_warps(uint64_t units, uint32_t w_max)
+{
+    if (units <= w_max) return static_cast<uint32_t>(units);
+    const uint64_t per_warp = (units + w_max - 1) / w_max;
+    return static_cast<uint32_t>((units + per_warp - 1) / per_warp);
+}
+
+struct DeviceInfo {
+    int device = -1, sms = 0, cc_major = 0;
+    bool ok = false;
+};
+
+int device_info(DeviceInfo* out)
+{
+    static thread_local DeviceInfo cache[64];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    if (dev < 0 || dev >= 64) return ECCO_ERR_INVALID_ARG;
+    DeviceInfo& c = cache[dev];
+    if (!c.ok) {
+        cudaDeviceProp prop;
+        e = cudaGetDeviceProperties(&prop, dev);
+        if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+        c.device = dev; c.sms = prop.multiProcessorCount; c.cc_major = prop.major; c.ok = true;
+    }
+    *out = c;
+    return c.cc_major == 10 ? ECCO_OK : ECCO_ERR_UNSUPPORTED_ARCH;
+}
+
+int check_launch();
+// Launch with the programmatic stream-serialisation attribute (see dependency_wait in the kernels):
+// the kernel must call dependency_wait() before its first access to global memory.
+template <class... Params, class... Args>
+int launch_overlapped(void (*kernel)(Params...), unsigned grid, unsigned block, size_t smem, cudaStream_t stream, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    return check_launch();
+}
+
+// Zeroes the ticket words of a workspace.  A kernel rather than a memset so that it can sit in a chain of
+// overlapped launches: it lets its successor start at once and clears only after its predecessor (which may
+// still be using the same workspace) has completed.
+__global__ void ecco_zero_words_kernel(unsigned int* __restrict__ p, size_t n)
+{
+    release_dependents();
+    dependency_wait();
+    for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n; i += static_cast<size_t>(gridDim.x) * blockDim.x) p[i] = 0u;
+}
+inline int zero_tickets(unsigned int* tickets, size_t bytes, cudaStream_t stream)
+{
+    const size_t n = bytes / sizeof(unsigned int);
+    if (n == 0) return ECCO_OK;
+    const unsigned grid = static_cast<unsigned>(n < 8192 ? (n + 255) / 256 : 32);
+    return launch_overlapped(ecco_zero_words_kernel, grid, 256u, 0, stream, tickets, n);
+}
+
+template <class K>
+int set_smem(K kernel, size_t bytes)
+{
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes));
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    return ECCO_OK;
+}
+
+int check_launch()
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { t_last_cuda_error = static_cast<int>(e); return ECCO_ERR_CUDA; }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ECCO_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+constexpr int kDecompressWarps = 32;
+// warps per CTA of the scalar fused kernels (one or two dot products per group): as many as shared memory allows
+constexpr int fused_warps(int) { return 22; }
+// per-warp GEMV: every warp also carries its own slice of x, which leaves room for 22 / 20 warps
+constexpr int gemv_warp_warps(int kV) { return kFusedRank ? (kV >= 2 ? 20 : 21) : (kV >= 2 ? 20 : 22); }
+
+struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
+
+// plan of the per-warp GEMV (one or two rows of x)
+GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
+{
+    GemvPlan p;
+    p.row_tiles = (n_out + 31) / 32;
+    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
+    const int64_t ctas = (units + gemv_warp_warps(vpad) - 1) / gemv_warp_warps(vpad);
+    p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
+    p.partial_bytes = static_cast<size_t>(p.grid * gemv_warp_warps(vpad) + p.row_tiles) * vpad * 32 * sizeof(float);
+    p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return p;
+}
+
+constexpr int kMmaWarps = 20;
+
+// plan of the tensor-core GEMV (3..8 rows of x): units and slots as in the per-warp kernel, eight columns
+GemvPlan gemv_mma_plan(int n_out, int kblocks, int ctas_max)
+{
+    GemvPlan p;
+    p.row_tiles = (n_out + 31) / 32;
+    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
+    const int64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
+    p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
+    p.partial_bytes = (static_cast<size_t>(p.grid * kMmaWarps + p.row_tiles) * 8 * 32 * sizeof(float) + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    return p;
+}
+
+inline int pad_v(int v) { return v <= 1 ? 1 : v <= 2 ? 2 : v <= 4 ? 4 : 8; }
+
+
+}  // namespace
