@@ -126,11 +126,13 @@ int ecco_meta_serialize_device(const ecco_meta* meta, void* host_staging, size_t
 int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out_fp16, void* stream);
 
 /* The same for several tensors in one call (the seven matrices of a decoder layer, the K and V caches of a
- * layer): the effect is that of ecco_decompress on every item in order, but tensors of 32 groups or more share
- * one kernel launch per 8 items, in which every SM moves on to the next tensor as soon as it is done with its
- * share of the current one, so launch latency and tail are paid once.  `items` is a HOST array read before the
- * call returns; every item has its own metadata image; items with n_groups == 0 are skipped.  Errors are those
- * of ecco_decompress and are found before anything is launched. */
+ * layer).  The items must be independent of each other: no item's output may overlap another item's output or
+ * blocks.  Then the effect is that of ecco_decompress on every item, but tensors of 32 groups or more share one
+ * kernel launch per 8 items, in which every SM moves on to the next tensor as soon as it is done with its share
+ * of the current one, so launch latency and tail are paid once.  With respect to other work in the stream the
+ * call is ordered like a single kernel.  `items` is a HOST array read before the call returns; every item has
+ * its own metadata image; items with n_groups == 0 are skipped.  Errors are those of ecco_decompress and are
+ * found before anything is launched. */
 typedef struct ecco_decompress_item {
     const void* d_meta;        /* device: metadata image of this tensor */
     const uint8_t* d_blocks;   /* device: 64 * n_groups bytes */
