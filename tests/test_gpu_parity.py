@@ -339,10 +339,21 @@ def check_full_gemv(B, eo, synth, t, om, d_meta, d_blocks, batch):
 
 
 def test_config2_llama7b_layer_full_size(B, eo, W, synth):
+    items, metas = [], []
     for t in W.config2(names=("q", "gate", "down")):
         om, d_meta, d_blocks = check_full_decompress(B, eo, t)
         for batch in (1, 8):
             check_full_gemv(B, eo, synth, t, om, d_meta, d_blocks, batch)
+        items.append((d_meta, d_blocks, t.n_groups, torch.empty(t.n_groups * 128, dtype=torch.float16, device="cuda")))
+        metas.append((om, t))
+    # the three tensors in the launch configuration bench.py times: one batched call, sampled against the oracle
+    B.ecco_decompress_batch(items)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == 0
+    for (om, t), (_, _, n, d_out) in zip(metas, items):
+        idx = sample_groups(n, np.random.Generator(np.random.PCG64(n + 1)))
+        got = d_out.view(-1, 128)[torch.from_numpy(idx).cuda()].cpu().numpy()
+        assert_bit_exact(got, eo.decode_threads(om, t.blocks[idx], 8))
 
 
 def check_full_attn(B, eo, synth, t, qpk):
