@@ -41,7 +41,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--small", action="store_true", help="reduced workload (q and gate only, K cache batch 2) for profiler captures")
+    ap.add_argument("--small", action="store_true", help="reduced workload for profiler captures (q and gate only, K cache batch 2; with --workload cfg5: batch-2 long-context caches)")
     ap.add_argument("--workload", default="cfg2", choices=["cfg2", "cfg4", "cfg5", "act2x", "var"],
                     help="cfg2 (default): Llama-2-7B-shaped layer + cfg3 K cache; cfg4: 70B-shaped MLP weights + stream-size "
                          "sweep; cfg5: long-context GQA K cache [16][8][32768][128] (decompress + attention scores with 8 "
@@ -206,6 +206,8 @@ WORKLOADS = {
     "cfg5": dict(label="cfg5 long-context GQA K and V caches [16][8][32768][128] (4,194,304 groups each)",
                  step="decompress x1 (K), attn_scores x1 and attn_values x1 (8 query heads per KV head); --only kvcomp times ecco_kv_compress over the whole K cache",
                  l2="inputs larger than L2: each step streams 256 MiB of blocks and writes 1 GiB"),
+    "small5": dict(label="reduced (profiling): cfg5-shaped K and V caches [2][8][16384][128], 8 query heads per KV head",
+                   step="decompress x1 (K), attn_scores x1 and attn_values x1", l2="inputs larger than L2 for decompress only"),
     "small": dict(label="reduced (profiling): q + gate of cfg2, K cache [2][32][4096][128]",
                   step="decompress x2, gemv batch 1 x2, gemv batch 8 x2, attn_scores x1, attn_values x1",
                   l2="inputs larger than L2 except the q projection"),
@@ -220,6 +222,11 @@ def build_workload(name, workloads):
         return [], (kt, vt), 8, True, ["decompress", "attn", "attnv"]
     if name == "cfg4":
         return workloads.config4(), None, 1, False, ["decompress", "gemv1"]
+    if name == "small5":
+        base = workloads.calibrate_kv(5, 8)
+        kt = workloads.kv_tensor("K", 2, 8, 16384, 1005 * 16, 3005, base, keep_source=True)
+        vt = workloads.kv_tensor("V", 2, 8, 16384, 1005 * 16 + 1, 3005, base)
+        return [], (kt, vt), 8, True, ["decompress", "attn", "attnv"]
     if name == "small":
         base = workloads.calibrate_kv(3, 32)
         kt = workloads.kv_tensor("K", 2, 32, 4096, 1003 * 16, 3003, base, keep_source=True)
@@ -248,7 +255,7 @@ def run_ours(args):
     B.lib()
 
     # ---- workload (the same seeded tensors on every rank)
-    wname = "small" if args.small else args.workload
+    wname = ("small5" if args.workload == "cfg5" else "small") if args.small else args.workload
     weights, kvt, q_per_kv, decompress_kv, default_segs = build_workload(wname, workloads)
     kt, vt = kvt if kvt is not None else (None, None)
     segs = [s for s in args.only.split(",") if s] or default_segs
