@@ -468,18 +468,18 @@ def run_ours(args):
     alg_bytes_per_launch = groups * (BLOCK + G * 2) / n_launch
     achieved = alg_bytes_per_launch / avg_launch_s / 1e9 if dec_ms > 0 else 0.0
     traffic = None
-    tp = os.path.join(ROOT, "profiles", "decompress_dram_bytes_per_group.json")
+    ncu_consts = {}
+    tp = os.path.join(ROOT, "paper_2505_06901_b200", "ncu_constants.json")
     if os.path.exists(tp):
         with open(tp) as f:
-            traffic = json.load(f)["dram_bytes_per_group"] * groups / n_launch
+            ncu_consts = json.load(f)
+        traffic = ncu_consts["decompress_dram"]["dram_bytes_per_group"] * groups / n_launch
     # What really limits the decoder are the SM's issue slots and its load/store pipe.  Their ceilings come from the
     # unit counts and the clock (4 warp instructions and 1 wavefront per clock per SM); the per-symbol costs are ncu
     # counters of this kernel (profiles/), the symbol rate is this run's.
     sm_limits = None
-    cp = os.path.join(ROOT, "profiles", "decompress_sm_counters.json")
-    if os.path.exists(cp) and dec_ms > 0:
-        with open(cp) as f:
-            c = json.load(f)
+    if "decompress_sm" in ncu_consts and dec_ms > 0:
+        c = ncu_consts["decompress_sm"]
         props = torch.cuda.get_device_properties(local)
         sms, ghz = props.multi_processor_count, (clocks or {}).get("sm_mhz", 0) / 1e3
         if ghz > 0:
@@ -490,7 +490,7 @@ def run_ours(args):
                 "lsu": {"bound": "lsu", "unit": "G wavefronts/s", "peak": sms * 1 * ghz,
                         "achieved": warp_symbols_per_s * c["lsu_wavefronts_per_warp_symbol"] / 1e9},
                 "per_warp_symbol": {"instructions": c["warp_instructions_per_warp_symbol"], "wavefronts": c["lsu_wavefronts_per_warp_symbol"]},
-                "source": "profiles/decompress_sm_counters.json; peaks = SMs x units x sampled SM clock",
+                "source": "paper_2505_06901_b200/ncu_constants.json (from profiles/ecco_decompress_tma_kernel_cfg5_dram.md); peaks = SMs x units x sampled SM clock",
             }
             for k in ("issue", "lsu"):
                 sm_limits[k]["frac"] = sm_limits[k]["achieved"] / sm_limits[k]["peak"]
