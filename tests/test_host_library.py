@@ -231,6 +231,73 @@ def test_device_image_rank_tables_and_arithmetic_constants(binding, eo, cfg1_sma
         assert np.all(rankl[cb] >> 4 == 4) and np.all(syml[cb] >> 4 == 4)
 
 
+def _complete_length_multisets():
+    """Every way to give 16 symbols code lengths in 2..8 with Kraft sum exactly 1, as counts per length."""
+    out = []
+
+    def rec(L, left, kraft, counts):
+        if L == 9:
+            if left == 0 and kraft == 0:
+                out.append(tuple(counts))
+            return
+        worth = 1 << (8 - L)
+        for c in range(min(left, kraft // worth) + 1):
+            rec(L + 1, left - c, kraft - c * worth, counts + [c])
+
+    rec(2, 16, 256, [])
+    return out
+
+
+def test_rank_tables_and_arithmetic_constants_for_every_code_shape(binding, eo):
+    """The mixed decoder's tables over EVERY admissible shape of a 2..8-bit code on 16 symbols (all multisets of
+    lengths with Kraft sum 1, lengths dealt to the symbols at random): for all 256 window bytes the arithmetic
+    route gives the canonical code's length, and codeword + delta is a bijection onto the ranks that agrees with
+    the rank table.  The expected lengths and codewords come from the oracle's canonical-code routine."""
+    shapes = _complete_length_multisets()
+    assert len(shapes) > 200 and (0, 0, 16, 0, 0, 0, 0) in shapes and (3, 0, 3, 0, 2, 0, 8) in shapes
+    rng = np.random.Generator(np.random.PCG64(2024))
+    spread = 1 | 1 << 10 | 1 << 20
+    guard = 0x100 | 0x100 << 10 | 0x100 << 20
+    per_meta = 64 * 4
+    kp_len = eo.huffman_limited(np.ones(64), 12)
+    pat = np.sort(rng.uniform(-1, 1, (64, 15)), axis=1).astype(np.float16)
+    for base in range(0, len(shapes), per_meta):
+        chunk = shapes[base:base + per_meta]
+        cb = np.full((64, 4, 16), 4, dtype=np.uint8)
+        for i, counts in enumerate(chunk):
+            lens = np.repeat(np.arange(2, 9), counts)
+            cb[i // 4, i % 4] = rng.permutation(lens)
+        lm = binding.ecco_meta_create(64, -5, pat, cb, kp_len)
+        img = binding.ecco_meta_serialize_device(lm)
+        rankl = img[84160:84160 + 65536].reshape(256, 256)
+        ar = img[84160 + 65536:].view(np.uint32).reshape(5, 256)
+        for i in range(len(chunk)):
+            lens = [int(x) for x in cb[i // 4, i % 4]]
+            codes, kraft = eo.canonical_codes(lens, 8)
+            assert kraft == 256
+            rot = ((i * 11 + (i >> 3)) & 31) << 2
+            c1, c2, d, rlo, rhi = (int(ar[j, i]) for j in range(5))
+            rank_of = rlo | rhi << 32
+            assert sorted((rank_of >> 4 * s) & 15 for s in range(16)) == list(range(16))
+            delta = {L: (d >> 4 * (L - 2)) & 15 for L in range(2, 8)}
+            delta[8] = 0
+            expect_len = np.zeros(256, dtype=np.int64)
+            expect_rank = np.zeros(256, dtype=np.int64)
+            for s in range(16):
+                L, code = lens[s], int(codes[s])
+                lo = code << (8 - L)
+                expect_len[lo:lo + (1 << (8 - L))] = L
+                expect_rank[lo:lo + (1 << (8 - L))] = (rank_of >> 4 * s) & 15
+            assert expect_len.min() >= 2                       # the code is complete: every window byte decodes
+            for b in range(256):
+                m = ((b * spread + c1) & 0xFFFFFFFF & (guard | 0xC0000000)) | ((b * 2 * spread + c2) & 0xFFFFFFFF & (2 * guard))
+                L = bin(m).count("1")
+                assert L == expect_len[b], (chunk[i], b)
+                assert ((b >> (8 - L)) + delta[L]) & 15 == expect_rank[b], (chunk[i], b)
+                rev = int(f"{b:08b}"[::-1], 2)
+                assert int(rankl[i, rev ^ rot]) == (L << 4 | expect_rank[b])
+
+
 def test_variable_length_host_encoder_matches_oracle(binding, eo, cfg1_small, kv_small):
     for fx, key, flags in ((cfg1_small, "w", binding.SELECT_MSE), (kv_small, "k", binding.SELECT_MINMAX | binding.KEEP_EXPONENT)):
         ometa, x = fx["meta"], fx[key]
