@@ -217,6 +217,49 @@ def test_decompress_batch_matches_oracle_per_item(B, eo, cfg1_small, kv_small, s
     assert bool((canary == 7.0).all())
 
 
+def test_decompress_every_code_shape_on_random_streams(B, eo, synth):
+    """All 255 admissible shapes of a 2..8-bit code on 16 symbols (every multiset of lengths with Kraft sum 1,
+    dealt to the symbols at random), one per codebook, decoded from random bit streams: whatever a block's header
+    bits select, table lookups and arithmetic decoding must give the oracle's values, clips and outliers."""
+    shapes = []
+
+    def rec(L, left, kraft, counts):
+        if L == 9:
+            if left == 0 and kraft == 0:
+                shapes.append(tuple(counts))
+            return
+        worth = 1 << (8 - L)
+        for c in range(min(left, kraft // worth) + 1):
+            rec(L + 1, left - c, kraft - c * worth, counts + [c])
+
+    rec(2, 16, 256, [])
+    assert len(shapes) == 255
+    rng = np.random.Generator(np.random.PCG64(99))
+    m = eo.Meta()
+    m.S, m.H, m.e = 64, 4, -3
+    kl = eo.huffman_limited(np.ones(64), 12)
+    for k in range(64):
+        m.kp_len[k] = int(kl[k])
+        pat = np.sort(rng.uniform(-1, 1, 15))
+        for j in range(15):
+            m.pattern[k][j] = int(np.float16(pat[j]).view(np.uint16))
+        for h in range(4):
+            lens = rng.permutation(np.repeat(np.arange(2, 9), shapes[(k * 4 + h) % len(shapes)]))
+            for s in range(16):
+                m.cb_len[k][h][s] = int(lens[s])
+    assert eo.meta_check(m) == 0
+    rb = synth.random_blocks(32 * 1024, 31)
+    lm = lib_meta_from_oracle(B, m)
+    assert_bit_exact(gpu_decompress(B, lm, rb), eo.decode_threads(m, rb, 8))
+    # the fused consumers over the same streams (their decoder is all-table; one and eight rows of x take the
+    # scalar and the tensor-core kernel)
+    for batch in (1, 8):
+        x = synth.activations(batch, 2048, 40 + batch)
+        got, _ = gpu_gemv(B, lm, rb, 2048, 2048, x, batch)
+        ref, refabs = eo.gemv(m, rb, 2048, 2048, x, batch)
+        check_fused(got, ref, refabs)
+
+
 def test_decompress_rejects_bad_arguments_on_device(B, cfg1_small):
     lm = lib_meta_from_oracle(B, cfg1_small["meta"])
     d_meta, d_blocks = B.meta_to_device(lm), dev(cfg1_small["blocks"])
