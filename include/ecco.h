@@ -185,6 +185,7 @@ int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, int32_t batch
  * [batch][n_kv_heads][seq], one group = one token's 128-wide head vector; out is fp32
  * [batch][n_kv_heads*q_per_kv][128]; q_per_kv in 1..8; seq >= 1.  The sum over tokens runs on the
  * tensor cores with fp32 accumulation, in an order fixed by the shapes (results are reproducible).
+ * Probabilities are carried with 22 bits down to 2e-12; smaller ones count as zero.
  * d_workspace: at least ecco_attn_values_workspace_bytes(...)
  * bytes, 16-byte aligned, contents irrelevant before and undefined after; calls sharing a workspace
  * must not overlap. */

@@ -51,6 +51,8 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 
 constexpr uint32_t kAvWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;   // + the [32][16] fp16 tile
 
+constexpr float kProbScale = 32768.0f, kProbUnscale = 1.0f / 32768.0f;      // powers of two: exact
+
 template <int kWarps>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_vblocks, int heads, int seq,
@@ -114,7 +116,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                     for (int j = 0; j < 4; ++j) {
                         const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
                         const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
-                        out_s[dim * 8 + head] += acc[ch][j];
+                        out_s[dim * 8 + head] += acc[ch][j] * kProbUnscale;
                     }
             }
             __syncthreads();
@@ -164,13 +166,18 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         {
             const int r = static_cast<int>(lane >> 2);
             const float2 st = stats_s[r];
+            // Probabilities enter the tensor cores as fp16 pairs (value + remainder).  Taken as they are, everything
+            // below 6e-5 would sit in fp16's subnormal range (one part in a thousand at p = 3e-5, the typical weight of
+            // a token in a 32768-token row); scaled by 2^15 they keep 22 bits down to 2e-12, and p <= 1 cannot
+            // overflow.  The sums are scaled back when they leave the accumulators (kProbUnscale in flush).
+            const float to_p = st.y * kProbScale;
             const float* srow = d_scores + (static_cast<size_t>(bh) * q_per_kv + min(r, q_per_kv - 1)) * seq;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int tk = tile_base + static_cast<int>(lane & 3u) * 2 + 8 * j;
                 float p0 = 0.0f, p1 = 0.0f;
-                if (r < q_per_kv && tk < seq) p0 = __expf(srow[tk] - st.x) * st.y;
-                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(srow[tk + 1] - st.x) * st.y;
+                if (r < q_per_kv && tk < seq) p0 = __expf(srow[tk] - st.x) * to_p;
+                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(srow[tk + 1] - st.x) * to_p;
                 const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
                 const __half l0 = __float2half_rn(p0 - __half2float(h0)), l1 = __float2half_rn(p1 - __half2float(h1));
                 p_hi[j] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);

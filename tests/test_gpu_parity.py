@@ -526,6 +526,34 @@ def test_attn_values_on_garbage_blocks_and_peaked_softmax(B, eo, kv_small, synth
     check_fused(got, ref, refabs)
 
 
+@pytest.mark.parametrize("qpk", [1, 8])
+def test_attn_values_keeps_small_probabilities(B, eo, kv_small, synth, qpk):
+    """One token takes almost all the weight and its vector is all zeros, so every output is the sum of the other
+    tokens' contributions at p ~ 1e-9: probabilities must survive the trip through the fp16 operands of the tensor
+    cores.  A second row spreads its weight evenly over 5000 tokens (p = 2e-4 each, below fp16's normal range).
+    Bound: 1e-3 sum p|V| plus 2^-38 sum |V|, the floor of the scaled fp16 pair."""
+    meta = kv_small["meta"]
+    seq = 5000
+    rng = np.random.Generator(np.random.PCG64(17))
+    x = synth.kv_cache(1, 1, seq, 1003, 3003).reshape(seq, 128).copy()
+    x[1234] = 0
+    blocks, _ = eo.encode(meta, x.astype(np.float16), eo.SELECT_MINMAX)
+    dec = eo.decode(meta, blocks).astype(np.float64)
+    assert not dec[1234].any()
+    scores = (rng.standard_normal((1, qpk, seq))).astype(np.float32)
+    scores[0, 0, 1234] += 22.0                             # p of the others ~ e^-22 / 1: 3e-10
+    if qpk > 1:
+        scores[0, 1, :] = 0.25                             # uniform: p = 2e-4 for every token
+    got = gpu_attn_values(B, lib_meta_from_oracle(B, meta), blocks, 1, 1, seq, qpk, scores)
+    ref, refabs = eo.attn_values(meta, blocks, 1, 1, seq, qpk, scores)
+    floor = np.abs(dec).sum(axis=0) * 2.0 ** -38
+    err = np.abs(got - ref)
+    assert np.all(err <= TOL * refabs + floor), float((err / (TOL * refabs + floor)).max())
+    assert np.abs(ref[0, 0]).max() < 1e-6 and np.abs(got[0, 0]).max() > 0      # the small sums are really there
+    if qpk > 1:
+        assert np.all(err[0, 1] <= 2e-5 * refabs[0, 1])    # evenly spread weights: far inside the bound
+
+
 # ------------------------------------------------------------------ online KV compressor
 def gpu_kv_compress(B, lmeta, x):
     n = x.size // 128
