@@ -8,7 +8,9 @@
 //
 // Shared memory per CTA:
 //   tables   pattern[64][16] fp16 | ID_KP table [4096] u16 | symbol tables [256][256] u8,
-//            brought in by one bulk copy (cp.async.bulk + mbarrier)
+//            brought in by one bulk copy (cp.async.bulk + mbarrier); the tile-store decompress
+//            kernel takes the rank-valued tables and the arithmetic-decode constants instead
+//            (two copies, 80 KB)
 //   per warp bits[18][32] u32   the warp's 32 blocks, word-transposed: lane L's word w at
 //                               [w][L] -> bank L whatever w is (conflict-free refills);
 //                               rows 16 and 17 stay zero (stream bits past 512 read as 0)
