@@ -405,19 +405,46 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
 // ecco_attn_values
 // ---------------------------------------------------------------------------------------------
 namespace {
-constexpr int kAvWarps = 16;    // 512 tokens per unit: divides the usual sequence lengths
-struct AvPlan { int grid; size_t stats_bytes, partial_bytes, ticket_bytes; };
+// Warps per CTA = tokens per unit / 32.  Twenty warps keep more decode chains in flight (96 registers per thread
+// instead of 120), sixteen make a unit of 512 tokens, which divides the usual sequence lengths: the choice goes by
+// how much of the last unit of a row is padding (cfg-5 cache, 32768 tokens: 889 us with 16, 821 us with 20; cfg-3
+// cache, 4096 tokens: 210 us with 16, 223 us with 20).
+constexpr int kAvWarpsNarrow = 16, kAvWarpsWide = 20;
+inline int av_warps(int seq)
+{
+    auto fill = [&](int w) { const int t = 32 * w; return static_cast<double>(seq) / (static_cast<double>((seq + t - 1) / t) * t); };
+    return fill(kAvWarpsWide) * 1.08 > fill(kAvWarpsNarrow) ? kAvWarpsWide : kAvWarpsNarrow;
+}
+struct AvPlan { int grid, warps; size_t stats_bytes, partial_bytes, ticket_bytes; };
 AvPlan av_plan(int batch, int n_kv_heads, int seq, int q_per_kv, int ctas_max)
 {
     AvPlan p;
+    p.warps = av_warps(seq);
     const int heads = batch * n_kv_heads;
-    const int64_t units = static_cast<int64_t>(heads) * ((seq + kAvWarps * 32 - 1) / (kAvWarps * 32));
+    const int64_t units = static_cast<int64_t>(heads) * ((seq + p.warps * 32 - 1) / (p.warps * 32));
     p.grid = static_cast<int>(balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(ctas_max)));
     auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
     p.stats_bytes = up(static_cast<size_t>(heads) * q_per_kv * sizeof(float2));
     p.partial_bytes = up(static_cast<size_t>(p.grid + heads) * kGroup * 8 * sizeof(float));
     p.ticket_bytes = up(static_cast<size_t>(heads) * sizeof(unsigned int));
     return p;
+}
+
+template <int kWarps>
+int launch_attn_values(const DeviceInfo& di, const AvPlan& p, const void* d_meta, const uint8_t* d_vblocks, int heads, int seq,
+                       int q_per_kv, const float* d_scores, float2* stats, float* d_out, float* partial, unsigned int* tickets,
+                       cudaStream_t s)
+{
+    auto kernel = ecco_attn_values_kernel<kWarps>;
+    const size_t smem = kSmemWarpBase + static_cast<size_t>(kWarps) * kAvWarpBytes + kGroup * 8 * sizeof(float);
+    static thread_local bool configured[64] = {};
+    if (!configured[di.device]) {
+        const int rc = set_smem(kernel, smem);
+        if (rc) return rc;
+        configured[di.device] = true;
+    }
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kWarps * 32), smem, s,
+                             static_cast<const uint8_t*>(d_meta), d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets);
 }
 }  // namespace
 
@@ -444,14 +471,6 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     const AvPlan p = av_plan(batch, n_kv_heads, seq, q_per_kv, di.sms < 256 ? di.sms : 256);
     if (!d_workspace || !aligned16(d_workspace)) return d_workspace ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (workspace_bytes < p.stats_bytes + p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
-    auto kernel = ecco_attn_values_kernel<kAvWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kAvWarps) * kAvWarpBytes + kGroup * 8 * sizeof(float);
-    static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     uint8_t* wsb = static_cast<uint8_t*>(d_workspace);
     float2* stats = reinterpret_cast<float2*>(wsb);
@@ -462,8 +481,9 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
     rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>((rows + 7) / 8), 256u, 0, s, d_scores, rows, seq, stats);
     if (rc) return rc;
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kAvWarps * 32), smem, s,
-                             static_cast<const uint8_t*>(d_meta), d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets);
+    return p.warps == kAvWarpsWide
+               ? launch_attn_values<kAvWarpsWide>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s)
+               : launch_attn_values<kAvWarpsNarrow>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s);
 }
 
 
