@@ -14,7 +14,9 @@ namespace {
 // mma.m16n8k16 per tile, fp32 accumulate (fp16 x fp16 products are exact in fp32).  A warp is
 // independent of the others: no vector slice in shared memory, no block barrier.
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;
+// The [32][16] fp16 staging tile of the second pass (1 KB) lives in rows 0..7 of the warp's bit-stream array: the
+// first pass has consumed them by then, the outlier fields sit in rows 8..15.
+constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr)
 {
@@ -29,8 +31,14 @@ __host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i 
 
 // vfrag[2c], vfrag[2c+1]: B fragments of chunk c (tile columns (lane%4)*2 + {0,1}, and + 8), vector lane/4
 // acc[0] / acc[1]: C fragments of rows 0..15 / 16..31 of the warp's 32 groups
+// fetch_vectors(vfrag) is called between the two passes: a caller whose vectors change with every group (the GEMV)
+// loads them there, so that they do not occupy sixteen registers during the first pass; one whose vectors stay
+// (the scores) copies them.
+__device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols);
+
+template <class FetchVectors>
 __device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base, const WarpSmem& ws, uint32_t stage, float T,
-                                            bool valid, const uint32_t (&vfrag)[16], float (&acc)[2][4])
+                                            bool valid, FetchVectors&& fetch_vectors, float (&acc)[2][4])
 {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = stage + lane * 32;
@@ -42,6 +50,8 @@ __device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base
         packed |= sym << ((n & 7) * 4);
         if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
     });
+    uint32_t vfrag[16];
+    fetch_vectors(vfrag);
     if (!valid) n_fit = 0;                                 // rows past the end contribute zeros
     const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
     uint64_t pads_lo = 0, pads_hi = 0;                     // 16 bits per chunk: which pads fall into it
@@ -117,7 +127,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
     ws.syms = ws.tab + kTabBytes;
     sts_u32(ws.bits + 16 * 128, 0u);
     sts_u32(ws.bits + 17 * 128, 0u);
-    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes;      // = rows 0..7 of bits, see kMmaWarpBytes
 
     const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
     const int tiles = (n_out + 31) / 32;
@@ -133,8 +143,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
     release_dependents();
     issue_tables(smem, d_meta, &bar);
     Block blk;
-    uint32_t vnext[16];
-    if (u0 < u1) { ldg_block(blk, block_ptr(u0)); load_vfrag(vnext, d_x + static_cast<int>(u0 % kblocks) * kGroup, k, batch); }
+    if (u0 < u1) ldg_block(blk, block_ptr(u0));
     if (!wait_tables(&bar)) return;
     const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
 
@@ -186,11 +195,10 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
             cur_tile = tile;
         }
         const Block cur = blk;
-        uint32_t vfrag[16];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) vfrag[i] = vnext[i];
-        if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_vfrag(vnext, d_x + static_cast<int>((u + 1) % kblocks) * kGroup, k, batch); }
-        row_dot_mma(cur, smem_base, ws, stage, T, tile * 32 + lane < n_out, vfrag, acc);
+        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        const __half* xk = d_x + static_cast<int>(u % kblocks) * kGroup;
+        row_dot_mma(cur, smem_base, ws, stage, T, tile * 32 + lane < n_out,
+                    [&](uint32_t (&v)[16]) { load_vfrag(v, xk, static_cast<size_t>(k), batch); }, acc);
     }
     if (u0 < u1) flush(cur_tile);
 }
@@ -213,7 +221,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
     ws.syms = ws.tab + kTabBytes;
     sts_u32(ws.bits + 16 * 128, 0u);
     sts_u32(ws.bits + 17 * 128, 0u);
-    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes;      // = rows 0..7 of bits, see kMmaWarpBytes
 
     const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
     const int tiles = (seq + 31) / 32;
@@ -240,7 +248,11 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         const Block cur = blk;
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        row_dot_mma(cur, smem_base, ws, stage, T, t0 + lane < seq, vfrag, acc);
+        row_dot_mma(cur, smem_base, ws, stage, T, t0 + lane < seq,
+                    [&](uint32_t (&v)[16]) {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) v[i] = vfrag[i];
+                    }, acc);
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt)
 #pragma unroll

@@ -116,7 +116,7 @@ GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
     return p;
 }
 
-constexpr int kMmaWarps = 20;
+constexpr int kMmaWarps = 24;
 
 // plan of the tensor-core GEMV (3..8 rows of x): units and slots as in the per-warp kernel, eight columns
 GemvPlan gemv_mma_plan(int n_out, int kblocks, int ctas_max)
