@@ -481,7 +481,7 @@ def run_ours(args):
     if "decompress_sm" in ncu_consts and dec_ms > 0:
         c = ncu_consts["decompress_sm"]
         props = torch.cuda.get_device_properties(local)
-        sms, ghz = props.multi_processor_count, (clocks or {}).get("sm_mhz", 0) / 1e3
+        sms, ghz = props.multi_processor_count, ((clocks or {}).get("sm_mhz") or 0) / 1e3
         if ghz > 0:
             warp_symbols_per_s = groups * (G / 32) * args.steps / (dec_ms / 1e3)
             sm_limits = {

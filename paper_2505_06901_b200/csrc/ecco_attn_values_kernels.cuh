@@ -53,46 +53,53 @@ constexpr uint32_t kAvWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;   
 
 constexpr float kProbScale = 32768.0f, kProbUnscale = 1.0f / 32768.0f;      // powers of two: exact
 
-template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+template <int kMaxWarps>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_vblocks, int heads, int seq,
                         int q_per_kv, const float* __restrict__ d_scores, const float2* __restrict__ d_stats,
                         float* __restrict__ d_out, float* __restrict__ d_partial, unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    __shared__ unsigned int ticket;
-    __shared__ float2 stats_s[8];
-    constexpr int kTokens = kWarps * 32;
-    const uint32_t smem_base = smem_u32(smem);
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    const int tid = static_cast<int>(threadIdx.x);
+    const int tid = static_cast<int>(threadIdx.x), n_threads = static_cast<int>(blockDim.x);
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kGroup * 8 * sizeof(float));
+    const int kTokens = static_cast<int>(nw) * 32;         // tokens per unit: one per thread of the working warps
+    const bool working = warp < nw;
+    // small CTA-wide words in the misc area at the start of shared memory (the barrier word is its first)
+    unsigned int& ticket = *reinterpret_cast<unsigned int*>(smem + 32);
+    float2* stats_s = reinterpret_cast<float2*>(smem + 64);
     WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * kAvWarpBytes + lane * 4;
-    ws.tab = ws.bits + kBitsBytes;
-    ws.syms = ws.tab + kTabBytes;
-    sts_u32(ws.bits + 16 * 128, 0u);
-    sts_u32(ws.bits + 17 * 128, 0u);
-    const uint32_t stage = smem_base + kSmemWarpBase + warp * kAvWarpBytes + kBitsBytes + kTabBytes + kSymsBytes;
+    ws.tab = tb.warp_base + warp * kTabBytes + lane * 4;
+    const uint32_t stage = tb.warp_base + nw * kTabBytes + warp * (1024 + kBitsBytes + kSymsBytes);
+    ws.bits = stage + 1024 + lane * 4;
+    ws.syms = ws.bits + kBitsBytes;
+    if (working) {
+        sts_u32(ws.bits + 16 * 128, 0u);
+        sts_u32(ws.bits + 17 * 128, 0u);
+    }
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
-    float* out_s = reinterpret_cast<float*>(smem + kSmemWarpBase + kWarps * kAvWarpBytes);    // [128 dims][8 heads]
+    float* out_s = reinterpret_cast<float*>(smem + (tb.warp_base - tb.base) + nw * kAvWarpBytes);    // [128 dims][8 heads]
 
-    const int G = gridDim.x, c = blockIdx.x;
     const int chunks = (seq + kTokens - 1) / kTokens;
     const int64_t U = static_cast<int64_t>(heads) * chunks;
+    // the CTAs that share a head count each other in (ticket), so every CTA of the split must own a unit: the
+    // launch may bring more CTAs than there are units (the host does not know how many warps find room)
+    const int G = static_cast<int>(min(static_cast<int64_t>(gridDim.x), U)), c = blockIdx.x;
+    if (c >= G) return;
     const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
     auto block_ptr = [&](int64_t u) {
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    dependency_wait();                                     // the previous kernel of the stream has completed
-    release_dependents();
-    issue_tables(smem, d_meta, &bar);
+    issue_tables(tb, d_meta);
     Block blk;
-    if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!wait_tables(&bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (u0 < u1 && working) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(tb)) return;
+    const float T = tb.T;
 
     float acc[8][4];                                       // [16-dim chunk][mma accumulator]
     auto clear_acc = [&]() {
@@ -106,9 +113,9 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     // all tokens of head bh seen by this CTA are in acc: reduce over the warps in warp order, then
     // either store (this CTA owns the whole head) or hand a partial to the slot-and-ticket reduction
     auto flush = [&](int bh) {
-        for (int i = tid; i < kGroup * 8; i += kTokens) out_s[i] = 0.0f;
+        for (int i = tid; i < kGroup * 8; i += n_threads) out_s[i] = 0.0f;
         __syncthreads();
-        for (int w = 0; w < kWarps; ++w) {
+        for (int w = 0; w < static_cast<int>(nw); ++w) {
             if (static_cast<int>(warp) == w) {
 #pragma unroll
                 for (int ch = 0; ch < 8; ++ch)
@@ -124,20 +131,20 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int c_lo = unit_owner(U, G, static_cast<int64_t>(bh) * chunks);
         const int c_hi = unit_owner(U, G, static_cast<int64_t>(bh + 1) * chunks - 1);
         if (c_lo == c_hi) {
-            for (int i = tid; i < kGroup * 8; i += kTokens) {
+            for (int i = tid; i < kGroup * 8; i += n_threads) {
                 const int dim = i >> 3, r = i & 7;
                 if (r < q_per_kv) d_out[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + dim] = out_s[i];
             }
         } else {
             float* mine = d_partial + static_cast<size_t>(c + bh) * (kGroup * 8);
-            for (int i = tid; i < kGroup * 8; i += kTokens) mine[i] = out_s[i];
+            for (int i = tid; i < kGroup * 8; i += n_threads) mine[i] = out_s[i];
             __threadfence();
             __syncthreads();
             if (tid == 0) ticket = atomicAdd(&d_tickets[bh], 1u);
             __syncthreads();
             if (ticket == static_cast<unsigned int>(c_hi - c_lo)) {
                 __threadfence();
-                for (int i = tid; i < kGroup * 8; i += kTokens) {
+                for (int i = tid; i < kGroup * 8; i += n_threads) {
                     const int dim = i >> 3, r = i & 7;
                     if (r >= q_per_kv) continue;
                     float sum = 0.0f;
@@ -161,6 +168,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             __syncthreads();
             cur_bh = bh;
         }
+        if (!working) continue;                            // warps without room for their arrays only help with the reductions
         // P^T fragments (B operand): head = lane / 4, tokens (lane % 4) * 2 + {0, 1} + 8 j
         uint32_t p_hi[4], p_lo[4];
         {
@@ -187,14 +195,13 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const Block cur = blk;
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         const bool valid = t < seq;                        // lanes past the end stage zeros (their p is zero too)
-        const GroupHeader h = open_group<false>(cur, smem_base, ws, T);
+        const GroupHeader h = open_group<kTabHalfBits>(cur, tb, ws, T);
         // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
-        uint32_t packed = 0;
+        RankPacker rk;
         int n_fit = kGroup;
-        const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+        const uint32_t end = decode_symbols<false, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t, uint32_t, bool alive, uint32_t pair) {
             if (!alive) n_fit = min(n_fit, n);             // only the clip path can see alive == false
-            packed |= sym << ((n & 7) * 4);
-            if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+            rk.put(n, pair, ws.syms);
         });
         if (!valid) n_fit = 0;
         // outliers of a complete group: which 16-dim chunks they fall into

@@ -19,16 +19,42 @@ constexpr int kMaxPads = 16;       // the sorter's top 16 (Sec. 4.3)
 constexpr int kHeaderBits = 10;    // scale byte + ID_HF
 constexpr int kExpMin = -32, kExpMax = 16;
 
-// Device image of the per-tensor metadata.  The tables follow the 64-byte header back to back
-// so that one bulk copy brings them into shared memory.
+// Device image of the per-tensor metadata: a 64-byte header, fixed-size tables, then two sections whose size
+// depends on the codebooks (DevHeader says how large they are).  What the decoders stage into shared memory is
+//   [pattern | ID_KP table | codebook records]   one bulk copy, kFixedTableBytes
+//   [shape tables]                                 one bulk copy, n_shapes * 256 bytes
+//   [pair tables]                                  one bulk copy, pair_bytes, to an address aligned to pair_align
+//
+// Code shapes.  A canonical code is fixed by how many of its 16 codewords have each length; the 256 codebooks of a
+// tensor share a few dozen such shapes.  The decode tables are stored per shape and work on the symbol's RANK, its
+// position in (length, symbol id) order: the codeword of rank r is the same bit string in every codebook of the
+// shape, and a codebook record carries the symbol -> rank nibbles, which the kernels use to lay out the lane's
+// sixteen dequantised values in rank order.
+//
+// Shape table [256] u8, indexed by the next 8 stream bits (first stream bit in bit 0): length << 4 | rank.
+// Pair table [2^W] u16 (W = 8..12 per shape), indexed by the next W stream bits: two symbols per lookup,
+//   bits 0..3   length of both codewords together           (escape: length of the first)
+//   bits 4..6   zero (room for the sum of two entries)
+//   bits 7..10  rank of the first symbol, i.e. rank << 7 = its byte offset in a [16][32] u32 value table
+//   bits 11..14 rank of the second symbol                   (escape: zero)
+//   bit  15     escape: the W bits end before the second codeword does; the decoder fetches it on its own
+// Shapes get table widths by expected use (from the ID_KP code lengths) and by how much a wider table lowers the
+// escape rate, within kPairBudgetBytes; tables are stored widest first, so each starts at a multiple of its size.
+// If even eight-bit tables for every shape do not fit, there are none (pair_bytes = 0).
 constexpr uint32_t kDevMagic = 0x4F434345u;  // "ECCO"
-constexpr uint32_t kDevVersion = 3;
+constexpr uint32_t kDevVersion = 4;
 struct DevHeader {
     uint32_t magic, version;
     int32_t S, H, e;
     float T;                 // 2^e
     uint32_t total_bytes;
-    uint32_t reserved[9];
+    uint32_t n_shapes;       // distinct code shapes among the codebooks
+    uint32_t shape_bytes;    // n_shapes * 256
+    uint32_t pair_bytes;     // 0: no pair tables
+    uint32_t pair_align;     // size of the widest pair table (a power of two), 0 without pair tables
+    uint32_t off_pair;       // byte offset of the pair tables in the image, a multiple of 16
+    uint32_t hash_lo, hash_hi;   // hash of every staged table (not of e, T): equal hashes = same tables
+    uint32_t reserved[2];
 };
 static_assert(sizeof(DevHeader) == 64, "header is 64 bytes");
 
@@ -36,48 +62,31 @@ constexpr uint32_t kOffPattern = 64;                                  // [64][16
 constexpr uint32_t kPatternBytes = kMaxPatterns * 16 * 2;
 constexpr uint32_t kOffKpLut = kOffPattern + kPatternBytes;           // [4096] u16: kp | len << 8
 constexpr uint32_t kKpLutBytes = (1u << kKpMaxLen) * 2;
-constexpr uint32_t kOffSymLut = kOffKpLut + kKpLutBytes;              // [S*H = 256][256] u8: len << 4 | sym
-constexpr uint32_t kSymLutBytes = kMaxPatterns * kCodebooks * 256;
-constexpr uint32_t kTableBytes = kOffSymLut + kSymLutBytes - kOffPattern;   // 75776: what the decoders stage, a multiple of 16
-// encoder tables for the device-side compressor, after the decode tables
-constexpr uint32_t kOffEncCb = kOffSymLut + kSymLutBytes;             // [256][16] u16: stream-order codeword | length << 8
+// codebook records [S*H = 256] x 16 bytes:
+//   word 0: (pair-table offset >> 9) | shape << 8 | W << 16   (W = 0: the shape has no pair table)
+//   word 1: zero
+//   words 2, 3: rank of symbol s in bits 4s of the 64-bit pair
+constexpr uint32_t kOffCbRec = kOffKpLut + kKpLutBytes;
+constexpr uint32_t kCbRecBytes = kMaxPatterns * kCodebooks * 16;
+constexpr uint32_t kFixedTableBytes = kPatternBytes + kKpLutBytes + kCbRecBytes;   // 14336: what every decoder stages first
+// encoder tables for the device-side compressor
+constexpr uint32_t kOffEncCb = kOffCbRec + kCbRecBytes;               // [256][16] u16: stream-order codeword | length << 8
 constexpr uint32_t kEncCbBytes = kMaxPatterns * kCodebooks * kSymbols * 2;
 constexpr uint32_t kOffEncKp = kOffEncCb + kEncCbBytes;               // [64] u16: stream-order ID_KP codeword | length << 12
 constexpr uint32_t kEncKpBytes = kMaxPatterns * 2;
 constexpr uint32_t kEncBytes = kEncCbBytes + kEncKpBytes;             // 8320, a multiple of 16
-// Tables of the decompress kernel's mixed decoder (table lookups and arithmetic decoding of the canonical
-// code take turns, so that neither the load/store pipe nor the integer pipe carries every symbol).
-// Both work on the symbol's RANK, a relabelling of the 16 symbols per codebook:
-//   rank(s) = (position of s in (length, id) order + rho) mod 16, rho such that an 8-bit codeword's rank is
-//   its own low four bits (rho = 0 without 8-bit codewords).
-// Then rank = (codeword + delta[L]) mod 16 for a codeword of length L, with delta[8] = 0.
-constexpr uint32_t kOffRankLut = kOffEncKp + kEncKpBytes;             // 84160: [256][256] u8: len << 4 | rank, rotated like the symbol tables
-constexpr uint32_t kRankLutBytes = kSymLutBytes;
-constexpr uint32_t kOffArith = kOffRankLut + kRankLutBytes;           // [5][256] u32, one row per word, column = codebook:
-constexpr int kArithWords = 5;                                        //   0, 1: addends of the length compare (see below)
-constexpr uint32_t kArithBytes = kArithWords * kMaxPatterns * kCodebooks * 4;   //   2: delta[2..7], 4 bits each, delta[L] in bits 4(L-2)
-constexpr uint32_t kDevBytes = kOffArith + kArithBytes;               //   3, 4: rank of symbol s in bits 4s of the 64-bit pair
-// Length compare: with b = the next 8 stream bits, first bit on top, and thr[L] = the smallest b whose codeword
-// is longer than L (256 if none), field i of word 0 (bits 10 i ..) holds 256 - thr[2 + i] and field i of word 1
-// (bits 10 i + 1 .., one bit higher so that the two words' result bits do not meet) holds 256 - thr[5 + i],
-// i = 0..2; word 0 also has bits 30 and 31 set.  b * kArithSpread + word 0 and b * 2 kArithSpread + word 1 put
-// b + 256 - thr in every field, whose bit 8 says b >= thr; the codeword length is the number of set bits under
-// kArithGuard | bits 30, 31 of the first and 2 kArithGuard of the second, i.e. 2 + the number of thresholds passed.
-constexpr uint32_t kArithSpread = 1u | (1u << 10) | (1u << 20);
-constexpr uint32_t kArithGuard = (0x100u) | (0x100u << 10) | (0x100u << 20);
-// Both lookup tables are indexed by the next stream bits with the first stream bit in bit 0,
+constexpr uint32_t kOffShapeLut = kOffEncKp + kEncKpBytes;            // [n_shapes][256] u8
+constexpr uint32_t kMaxShapes = kMaxPatterns * kCodebooks;
+constexpr int kPairMinBits = 8, kPairMaxBits = 12;
+constexpr uint32_t kPairBudgetBytes = 64u << 10;
+constexpr uint32_t kMaxDevBytes = kOffShapeLut + kMaxShapes * 256 + kPairBudgetBytes;
+// Both kinds of table are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.
-//
-// Symbol tables are stored with a per-codebook index rotation: the entry for window value i of
-// codebook cb sits at index i ^ lut_rotation(cb).  The rotation touches index bits 2..6, which
-// select the shared-memory bank of a byte entry, so lanes that decode with different codebooks
-// spread over different banks even when their windows agree.
 #ifdef __CUDACC__
 #define ECCO_HD __host__ __device__
 #else
 #define ECCO_HD
 #endif
-ECCO_HD constexpr uint32_t lut_rotation(uint32_t cb) { return ((cb * 11u + (cb >> 3)) & 31u) << 2; }
 
 // Variable-length container: index = u64 total_bits | u64 chunk_base[ceil(n / 4096)] | u32 offset[n];
 // group g starts at stream bit chunk_base[g >> 12] + offset[g].

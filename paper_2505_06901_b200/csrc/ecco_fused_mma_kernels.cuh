@@ -17,6 +17,21 @@ namespace {
 // The [32][16] fp16 staging tile of the second pass (1 KB) lives in rows 0..7 of the warp's bit-stream array: the
 // first pass has consumed them by then, the outlier fields sit in rows 8..15.
 constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
+// value tables first (each at a multiple of 2 KB), then per warp the bit-stream array and the decoded ranks
+__device__ __forceinline__ WarpSmem mma_warp_smem(const Tables& tb, uint32_t nw, uint32_t* stage)
+{
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    WarpSmem ws;
+    ws.tab = tb.warp_base + warp * kTabBytes + lane * 4;
+    *stage = tb.warp_base + nw * kTabBytes + warp * (kBitsBytes + kSymsBytes);          // = rows 0..7 of bits
+    ws.bits = *stage + lane * 4;
+    ws.syms = ws.bits + kBitsBytes;
+    if (warp < nw) {
+        sts_u32(ws.bits + 16 * 128, 0u);
+        sts_u32(ws.bits + 17 * 128, 0u);
+    }
+    return ws;
+}
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&a)[4], uint32_t addr)
 {
@@ -37,18 +52,17 @@ __host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i 
 __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols);
 
 template <class FetchVectors>
-__device__ __forceinline__ void row_dot_mma(const Block& blk, uint32_t smem_base, const WarpSmem& ws, uint32_t stage, float T,
+__device__ __forceinline__ void row_dot_mma(const Block& blk, const Tables& tb, const WarpSmem& ws, uint32_t stage, float T,
                                             bool valid, FetchVectors&& fetch_vectors, float (&acc)[2][4])
 {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = stage + lane * 32;
-    const GroupHeader h = open_group<false>(blk, smem_base, ws, T);
-    uint32_t packed = 0;
+    const GroupHeader h = open_group<kTabHalfBits>(blk, tb, ws, T);
+    RankPacker rk;
     int n_fit = kGroup;
-    const uint32_t end = decode_symbols<false, 16, kBlockBits, 0, kFusedFree>(h, ws, [&](int n, uint32_t, uint32_t sym, bool alive) {
+    const uint32_t end = decode_symbols<false, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t, uint32_t, bool alive, uint32_t pair) {
         if (!alive) n_fit = min(n_fit, n);
-        packed |= sym << ((n & 7) * 4);
-        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+        rk.put(n, pair, ws.syms);
     });
     uint32_t vfrag[16];
     fetch_vectors(vfrag);
@@ -111,41 +125,36 @@ __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* 
 
 // K2m: y[b][n] = sum_k W~[n][k] x[b][k] for 3..8 rows of x.  Units, ownership and the slot-and-ticket
 // reduction are those of the per-warp kernel (unit = 32 rows x one k-block).
-template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+template <int kMaxWarps>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
                      const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
-                     unsigned int* __restrict__ d_tickets, int active_warps)
+                     unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    const uint32_t smem_base = smem_u32(smem);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
-    ws.tab = ws.bits + kBitsBytes;
-    ws.syms = ws.tab + kTabBytes;
-    sts_u32(ws.bits + 16 * 128, 0u);
-    sts_u32(ws.bits + 17 * 128, 0u);
-    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes;      // = rows 0..7 of bits, see kMmaWarpBytes
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
+    uint32_t stage;
+    const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
 
-    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
     const int tiles = (n_out + 31) / 32;
     const int64_t U = static_cast<int64_t>(tiles) * kblocks;
-    const int W = active_warps;
+    const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     const int k = kblocks * kGroup;
     auto block_ptr = [&](int64_t u) {
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
-    dependency_wait();                                     // the previous kernel of the stream has completed
-    release_dependents();
-    issue_tables(smem, d_meta, &bar);
+    issue_tables(tb, d_meta);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!wait_tables(&bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (!wait_tables(tb)) return;
+    const float T = tb.T;
 
     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     // C fragment element (mt, i): row = 16 mt + lane/4 + 8 (i >= 2), column b = (lane%4)*2 + (i & 1)
@@ -197,7 +206,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
         const Block cur = blk;
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         const __half* xk = d_x + static_cast<int>(u % kblocks) * kGroup;
-        row_dot_mma(cur, smem_base, ws, stage, T, tile * 32 + lane < n_out,
+        row_dot_mma(cur, tb, ws, stage, T, tile * 32 + lane < n_out,
                     [&](uint32_t (&v)[16]) { load_vfrag(v, xk, static_cast<size_t>(k), batch); }, acc);
     }
     if (u0 < u1) flush(cur_tile);
@@ -205,40 +214,34 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
 
 // K3m: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for 3..8 query heads per KV head.
 // Unit = (one (batch, kv head), 32 tokens); every working warp owns a contiguous run of units.
-template <int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+template <int kMaxWarps>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
-                            int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores,
-                            int active_warps)
+                            int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    const uint32_t smem_base = smem_u32(smem);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    WarpSmem ws;
-    ws.bits = smem_base + kSmemWarpBase + warp * kMmaWarpBytes + lane * 4;
-    ws.tab = ws.bits + kBitsBytes;
-    ws.syms = ws.tab + kTabBytes;
-    sts_u32(ws.bits + 16 * 128, 0u);
-    sts_u32(ws.bits + 17 * 128, 0u);
-    const uint32_t stage = smem_base + kSmemWarpBase + warp * kMmaWarpBytes;      // = rows 0..7 of bits, see kMmaWarpBytes
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
+    uint32_t stage;
+    const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
 
-    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
     const int tiles = (seq + 31) / 32;
     const int64_t U = static_cast<int64_t>(heads) * tiles;
-    const int W = active_warps;
+    const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     auto block_ptr = [&](int64_t u) {
         const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    dependency_wait();                                     // the previous kernel of the stream has completed
-    release_dependents();
-    issue_tables(smem, d_meta, &bar);
+    issue_tables(tb, d_meta);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!wait_tables(&bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (!wait_tables(tb)) return;
+    const float T = tb.T;
 
     uint32_t vfrag[16];
     int cur_bh = -1;
@@ -248,7 +251,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         const Block cur = blk;
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        row_dot_mma(cur, smem_base, ws, stage, T, t0 + lane < seq,
+        row_dot_mma(cur, tb, ws, stage, T, t0 + lane < seq,
                     [&](uint32_t (&v)[16]) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = vfrag[i];

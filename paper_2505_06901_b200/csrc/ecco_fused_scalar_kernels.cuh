@@ -61,15 +61,14 @@ struct Accum {
 
 // decode one group and accumulate its kV dot products against xs (shared address of xs[0][0])
 template <int kV>
-__device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base, const WarpSmem& ws, float T,
+__device__ __forceinline__ void fused_group(const Block& blk, const Tables& tb, const WarpSmem& ws, float T,
                                             uint32_t xs, Accum<kV>& acc)
 {
-    const GroupHeader h = open_group<true, kFusedRank>(blk, smem_base, ws, T);
-    uint32_t packed = 0;
-    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedArith, kFusedFree>(h, ws, [&](int n, uint32_t v, uint32_t sym, bool) {
+    const GroupHeader h = open_group<kTabFloat>(blk, tb, ws, T);
+    RankPacker rk;
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t pair) {
         acc.fma(n, __uint_as_float(v), xs);
-        packed |= sym << ((n & 7) * 4);
-        if ((n & 7) == 7) { sts_u32(ws.syms + (n >> 3) * 128, packed); packed = 0; }
+        rk.put(n, pair, ws.syms);
     });
     if (end) {
         // outliers replace the mapped value at their location: add (outlier - mapped) * x
@@ -83,8 +82,8 @@ __device__ __forceinline__ void fused_group(const Block& blk, uint32_t smem_base
             if ((upper ? seen_hi : seen_lo) & bit) continue;
             if (upper) seen_hi |= bit; else seen_lo |= bit;
             const uint32_t word = lds_u32(ws.syms + (loc >> 3) * 128);
-            const uint32_t sym = (word >> ((loc & 7u) * 4)) & 15u;
-            const float mapped = __uint_as_float(lds_u32(ws.tab + sym * 128));
+            const uint32_t rank = (word >> ((loc & 7u) * 4)) & 15u;
+            const float mapped = __uint_as_float(lds_u32(ws.tab + rank * 128));
             const float outlier = __half2float(__float2half_rn(fp8_to_float(f >> 7) * T));
             acc.fma_at(loc, outlier - mapped, xs);
         }
@@ -101,17 +100,19 @@ __host__ __device__ __forceinline__ int unit_owner(int64_t U, int G, int64_t u)
     return c;
 }
 
-template <int kWarps>
-__device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
+// per-warp arrays of the scalar fused kernels: value table (fp32), bit-stream array, decoded ranks
+constexpr uint32_t kFusedWarpBytes = kTabBytes + kBitsBytes + kSymsBytes;
+__device__ __forceinline__ WarpSmem fused_warp_smem(const Tables& tb, uint32_t nw)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
-    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
     WarpSmem ws;
-    ws.bits = smem_base + kFusedBase + warp * kWarpBytes + lane * 4;
-    ws.tab = ws.bits + kBitsBytes;
-    ws.syms = ws.tab + kTabBytes;
-    sts_u32(ws.bits + 16 * 128, 0u);
-    sts_u32(ws.bits + 17 * 128, 0u);
+    ws.tab = tb.warp_base + warp * kTabBytes + lane * 4;
+    ws.bits = tb.warp_base + nw * kTabBytes + warp * (kBitsBytes + kSymsBytes) + lane * 4;
+    ws.syms = ws.bits + kBitsBytes;
+    if (warp < nw) {
+        sts_u32(ws.bits + 16 * 128, 0u);
+        sts_u32(ws.bits + 17 * 128, 0u);
+    }
     return ws;
 }
 
@@ -123,40 +124,39 @@ __device__ __forceinline__ WarpSmem fused_warp_smem(uint32_t smem_base)
 // staircase of (warp, tile) pairs) and the last to arrive (ticket counter) adds the slots in warp
 // order: the result does not depend on scheduling.  Workspace: partial[slot][kV][32] floats, then
 // one ticket per 32-row tile.
-template <int kV, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+template <int kV, int kMaxWarps>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
                       const __half* __restrict__ d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
-                      unsigned int* __restrict__ d_tickets, int active_warps)
+                      unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
     constexpr uint32_t kXsBytes = kGroup * kV * 4;
-    const uint32_t smem_base = smem_u32(smem);
-    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes));
+    const WarpSmem ws = fused_warp_smem(tb, nw);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    const uint32_t xs = smem_base + kFusedBase + kWarps * kWarpBytes + warp * kXsBytes;   // this warp's slice
+    const uint32_t xs = tb.warp_base + nw * kFusedWarpBytes + warp * kXsBytes;   // this warp's slice
 
     // W working warps (chosen by the host so that they all get the same number of units, and never
     // more than there are units); warp ids interleave over the CTAs; the other warps idle
-    const int wg = warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x);
+    const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
     const int tiles = (n_out + 31) / 32;
     const int64_t U = static_cast<int64_t>(tiles) * kblocks;
-    const int W = active_warps;
+    const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     const int k = kblocks * kGroup;
     auto block_ptr = [&](int64_t u) {
         const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
-    dependency_wait();                                     // the previous kernel of the stream has completed
-    release_dependents();
-    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
+    issue_tables(tb, d_meta);
     Block blk;
     if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!wait_tables(&bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (!wait_tables(tb)) return;
+    const float T = tb.T;
 
     Accum<kV> acc;
     acc.clear();
@@ -236,7 +236,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         __syncwarp();
         const Block cur = blk;
         if (u + 1 < u1) { ldg_block(blk, block_ptr(u + 1)); load_x(u + 1); }
-        fused_group<kV>(cur, smem_base, ws, T, xs, acc);
+        fused_group<kV>(cur, tb, ws, T, xs, acc);
     }
     if (u0 < u1) flush(cur_tile);
 }
@@ -244,21 +244,23 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
 // K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t].  A work unit is (one (batch, kv
 // head) pair, a chunk of kWarps*32 tokens); units are dealt to persistent CTAs in contiguous runs,
 // the query slice is restaged when the head changes, a thread owns one token.
-template <int kV, int kWarps>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+template <int kV, int kMaxWarps>
+__global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
                         int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    __shared__ uint64_t bar;
-    constexpr int kTokens = kWarps * 32;
-    constexpr uint32_t kWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
-    const uint32_t smem_base = smem_u32(smem);
-    const WarpSmem ws = fused_warp_smem<kWarps>(smem_base);
-    float* xs = reinterpret_cast<float*>(smem + kFusedBase + kWarps * kWarpBytes);
-    const uint32_t xs_addr = smem_u32(xs);
+    dependency_wait();                                     // the previous kernel of the stream has completed
+    release_dependents();
+    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes, kGroup * kV * 4));
+    const int kTokens = nw * 32;                           // tokens per unit: one per thread of the working warps
+    const WarpSmem ws = fused_warp_smem(tb, nw);
+    const uint32_t xs_addr = tb.warp_base + nw * kFusedWarpBytes;
+    float* xs = reinterpret_cast<float*>(smem + (xs_addr - tb.base));
 
     const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
+    const bool working = tid < kTokens;
     const int chunks = (seq + kTokens - 1) / kTokens;
     const int64_t U = static_cast<int64_t>(heads) * chunks;
     const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
@@ -267,13 +269,11 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
-    dependency_wait();                                     // the previous kernel of the stream has completed
-    release_dependents();
-    if (kFusedRank) issue_rank_tables(smem, d_meta, &bar); else issue_tables(smem, d_meta, &bar);
+    issue_tables(tb, d_meta);
     Block blk;
-    if (u0 < u1) ldg_block(blk, block_ptr(u0));
-    if (!wait_tables(&bar)) return;
-    const float T = reinterpret_cast<const DevHeader*>(d_meta)->T;
+    if (u0 < u1 && working) ldg_block(blk, block_ptr(u0));
+    if (!wait_tables(tb)) return;
+    const float T = tb.T;
 
     int cur_bh = -1;
     for (int64_t u = u0; u < u1; ++u) {
@@ -281,18 +281,19 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         if (bh != cur_bh) {
             __syncthreads();                               // everyone is done with the previous head's slice
             // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
-            for (int i = tid; i < kGroup * kV; i += kTokens) {
+            for (int i = tid; i < kGroup * kV; i += static_cast<int>(blockDim.x)) {
                 const int r = i % kV, d = i / kV;
                 xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
             }
             __syncthreads();
             cur_bh = bh;
         }
+        if (!working) continue;                            // warps without room for their arrays only help with the slice
         const Block cur = blk;
         if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
         Accum<kV> acc;
         acc.clear();
-        fused_group<kV>(cur, smem_base, ws, T, xs_addr, acc);
+        fused_group<kV>(cur, tb, ws, T, xs_addr, acc);
         if (t < seq) {
 #pragma unroll
             for (int r = 0; r < kV; ++r)

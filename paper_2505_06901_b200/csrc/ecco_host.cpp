@@ -5,7 +5,9 @@
 #include <atomic>
 #include <cmath>
 #include <cstdint>
+#include <cstdlib>
 #include <cstring>
+#include <memory>
 #include <mutex>
 #include <new>
 #include <numeric>
@@ -133,6 +135,9 @@ struct ecco_meta {
     float pattern_f[kMaxPatterns][kCentroids] = {};
     uint16_t cb_rev[kMaxPatterns][kCodebooks][kSymbols] = {};   // bit-reversed codewords (stream order, lsb first)
     uint16_t kp_rev[kMaxPatterns] = {};
+    // how often the host encoder has picked each codebook with this metadata so far (a hint for the device image:
+    // which code shapes deserve the wide decode tables; all zero = unknown)
+    uint64_t cb_use[kMaxPatterns][kCodebooks] = {};
 };
 
 namespace {
@@ -595,6 +600,8 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
     const float T = std::ldexp(1.0f, m->e);
     const int threads = available_cores();
     std::vector<ecco_stats> part(static_cast<size_t>(threads));
+    struct CbUse { uint64_t n[kMaxPatterns][kCodebooks]; };
+    std::vector<CbUse> use(static_cast<size_t>(threads));
     std::atomic<int> err{0};
     parallel_ranges(n_groups, threads, [&](int t, uint64_t lo, uint64_t hi) {
         Scratch s;
@@ -602,9 +609,12 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
         GroupOut g;
         ecco_stats st;
         std::memset(&st, 0, sizeof st);
+        CbUse& cu = use[static_cast<size_t>(t)];
+        std::memset(&cu, 0, sizeof cu);
         for (uint64_t i = lo; i < hi && !err.load(std::memory_order_relaxed); ++i) {
             int r = encode_group(*m, src + i * kGroup, select, T, s, dst + i * kBlockBytes, g, q);
             if (r) { err = r; break; }
+            cu.n[g.kp][g.hf]++;
             st.n_groups++;
             if (g.n_fit < kGroup) { st.clipped_groups++; st.clipped_values += static_cast<uint64_t>(kGroup - g.n_fit); }
             if (g.n_pad) { st.padded_groups++; st.padded_values += static_cast<uint64_t>(g.n_pad); }
@@ -616,6 +626,9 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
         part[static_cast<size_t>(t)] = st;
     });
     if (err) return err;
+    for (const auto& cu : use)
+        for (int k = 0; k < kMaxPatterns; ++k)
+            for (int h = 0; h < kCodebooks; ++h) m->cb_use[k][h] += cu.n[k][h];
     if (stats) {
         std::memset(stats, 0, sizeof *stats);
         for (const auto& p : part) {
@@ -856,23 +869,111 @@ extern "C" int ecco_calibrate_host(const uint16_t* calib, uint64_t n_groups, con
 // ---------------------------------------------------------------------------------------------
 // C ABI: device image
 // ---------------------------------------------------------------------------------------------
-extern "C" size_t ecco_meta_device_bytes(const ecco_meta* m) { return m ? kDevBytes : 0; }
+namespace {
+
+// code shapes of a metadata set and the plan of its decode tables
+struct ImagePlan {
+    int n_shapes = 0;
+    uint8_t counts[kMaxShapes][kMaxLen + 1] = {};          // shape -> number of codewords per length
+    int shape_of[kMaxPatterns][kCodebooks] = {};
+    int width[kMaxShapes] = {};                            // pair-table index bits per shape, 0 = none
+    uint32_t pair_off[kMaxShapes] = {};                    // byte offset of the shape's pair table in the pair region
+    uint32_t pair_bytes = 0, pair_align = 0;
+    uint32_t total_bytes = 0, off_pair = 0;
+};
+
+// probability that two consecutive codewords of the shape do not both end within W bits, symbols drawn with
+// probability 2^-length (what the code is optimal for)
+double escape_rate(const uint8_t* counts, int W)
+{
+    double esc = 0.0;
+    for (int l0 = kMinLen; l0 <= kMaxLen; ++l0)
+        for (int l1 = kMinLen; l1 <= kMaxLen; ++l1)
+            if (l0 + l1 > W) esc += std::ldexp(static_cast<double>(counts[l0]), -l0) * std::ldexp(static_cast<double>(counts[l1]), -l1);
+    return esc;
+}
+
+void plan_image(const ecco_meta& m, ImagePlan& p)
+{
+    double use[kMaxShapes] = {};
+    uint64_t seen = 0;
+    for (int k = 0; k < m.S; ++k)
+        for (int h = 0; h < kCodebooks; ++h) seen += m.cb_use[k][h];
+    for (int k = 0; k < kMaxPatterns; ++k)
+        for (int h = 0; h < kCodebooks; ++h) {
+            uint8_t c[kMaxLen + 1] = {};
+            if (k < m.S) for (int s = 0; s < kSymbols; ++s) ++c[m.cb_len[k][h][s]];
+            else c[4] = kSymbols;                          // rows of unused patterns decode as sixteen 4-bit codewords
+            int id = -1;
+            for (int i = 0; i < p.n_shapes && id < 0; ++i)
+                if (!std::memcmp(p.counts[i], c, sizeof c)) id = i;
+            if (id < 0) { id = p.n_shapes++; std::memcpy(p.counts[id], c, sizeof c); }
+            p.shape_of[k][h] = id;
+            if (k < m.S)     // expected use: what the encoder has seen, else what the ID_KP code lengths say
+                use[id] += seen ? static_cast<double>(m.cb_use[k][h]) / static_cast<double>(seen)
+                                : std::ldexp(1.0, -m.kp_len[k]) / kCodebooks;
+        }
+    // widths: everyone starts at the minimum; then the upgrade that removes the most escapes per byte, while it fits
+    uint32_t bytes = static_cast<uint32_t>(p.n_shapes) * (2u << kPairMinBits);
+    uint32_t kPairBudgetBytes = ecco::kPairBudgetBytes;
+    if (const char* env = std::getenv("ECCO_PAIR_BUDGET_KB")) kPairBudgetBytes = std::min<uint32_t>(kPairBudgetBytes, static_cast<uint32_t>(std::atoi(env)) << 10);
+    if (bytes <= kPairBudgetBytes) {
+        for (int i = 0; i < p.n_shapes; ++i) p.width[i] = kPairMinBits;
+        for (;;) {
+            int best = -1;
+            double best_gain = 0.0;
+            for (int i = 0; i < p.n_shapes; ++i) {
+                const int W = p.width[i];
+                if (W >= kPairMaxBits || bytes + (2u << W) > kPairBudgetBytes) continue;
+                const double gain = (use[i] + 1e-9) * (escape_rate(p.counts[i], W) - escape_rate(p.counts[i], W + 1)) / static_cast<double>(2u << W);
+                if (best < 0 || gain > best_gain) { best = i; best_gain = gain; }
+            }
+            if (best < 0 || best_gain <= 0.0) break;
+            bytes += 2u << p.width[best];
+            ++p.width[best];
+        }
+        uint32_t off = 0;
+        for (int W = kPairMaxBits; W >= kPairMinBits; --W)      // widest first: every table starts at a multiple of its size
+            for (int i = 0; i < p.n_shapes; ++i)
+                if (p.width[i] == W) { p.pair_off[i] = off; off += 2u << W; if (!p.pair_align) p.pair_align = 2u << W; }
+        p.pair_bytes = off;
+    }
+    p.off_pair = (kOffShapeLut + static_cast<uint32_t>(p.n_shapes) * 256u + 15u) & ~15u;
+    p.total_bytes = p.off_pair + p.pair_bytes;
+}
+
+inline uint64_t fnv1a(const uint8_t* b, size_t n, uint64_t h)
+{
+    for (size_t i = 0; i < n; ++i) { h ^= b[i]; h *= 1099511628211ull; }
+    return h;
+}
+
+}  // namespace
+
+extern "C" size_t ecco_meta_device_bytes(const ecco_meta* m)
+{
+    if (!m) return 0;
+    ecco_meta tmp = *m;
+    if (derive(&tmp)) return 0;
+    ImagePlan* p = new ImagePlan;
+    plan_image(tmp, *p);
+    const size_t n = p->total_bytes;
+    delete p;
+    return n;
+}
 
 extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging, size_t bytes)
 {
     if (!m || !host_staging) return ECCO_ERR_INVALID_ARG;
-    if (bytes < kDevBytes) return ECCO_ERR_INVALID_ARG;
     ecco_meta tmp = *m;
     int rc = derive(&tmp);
     if (rc) return rc;
+    std::unique_ptr<ImagePlan> plan(new ImagePlan);
+    ImagePlan& p = *plan;
+    plan_image(tmp, p);
+    if (bytes < p.total_bytes) return ECCO_ERR_INVALID_ARG;
     uint8_t* base = static_cast<uint8_t*>(host_staging);
-    std::memset(base, 0, kDevBytes);
-    DevHeader h;
-    std::memset(&h, 0, sizeof h);
-    h.magic = kDevMagic; h.version = kDevVersion; h.S = tmp.S; h.H = kCodebooks; h.e = tmp.e;
-    h.T = std::ldexp(1.0f, tmp.e);
-    h.total_bytes = kDevBytes;
-    std::memcpy(base, &h, sizeof h);
+    std::memset(base, 0, p.total_bytes);
     std::memcpy(base + kOffPattern, tmp.pattern, kPatternBytes);
     // ID_KP table: every 12-bit window whose low kp_len bits equal the reversed codeword
     uint16_t* kpl = reinterpret_cast<uint16_t*>(base + kOffKpLut);
@@ -881,18 +982,6 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
         for (uint32_t hi = 0; hi < (1u << (kKpMaxLen - L)); ++hi)
             kpl[tmp.kp_rev[k] | (hi << L)] = static_cast<uint16_t>(k | (L << 8));
     }
-    // symbol tables: every 8-bit window whose low len bits equal the reversed codeword
-    uint8_t* sl = base + kOffSymLut;
-    for (int k = 0; k < tmp.S; ++k)
-        for (int c = 0; c < kCodebooks; ++c) {
-            const uint32_t cb = static_cast<uint32_t>(k) * kCodebooks + c, rot = lut_rotation(cb);
-            uint8_t* t = sl + static_cast<size_t>(cb) * 256;
-            for (int s = 0; s < kSymbols; ++s) {
-                int L = tmp.cb_len[k][c][s];
-                for (uint32_t hi = 0; hi < (1u << (kMaxLen - L)); ++hi)
-                    t[(tmp.cb_rev[k][c][s] | (hi << L)) ^ rot] = static_cast<uint8_t>((L << 4) | s);
-            }
-        }
     // encoder tables: codeword in stream order (first code bit in bit 0) and its length
     uint16_t* ecb = reinterpret_cast<uint16_t*>(base + kOffEncCb);
     uint16_t* ekp = reinterpret_cast<uint16_t*>(base + kOffEncKp);
@@ -903,59 +992,62 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
                 ecb[(static_cast<size_t>(k) * kCodebooks + c) * kSymbols + s] =
                     static_cast<uint16_t>(tmp.cb_rev[k][c][s] | (tmp.cb_len[k][c][s] << 8));
     }
-    // unused pattern rows (S < 64) decode with 4-bit codes so that every table entry is valid
-    for (int k = tmp.S; k < kMaxPatterns; ++k)
-        for (int c = 0; c < kCodebooks; ++c) {
-            uint8_t* t = sl + (static_cast<size_t>(k) * kCodebooks + c) * 256;
-            for (uint32_t i = 0; i < 256; ++i) t[i] = static_cast<uint8_t>((4 << 4) | bit_reverse(i & 15u, 4));
-        }
-    // rank tables and arithmetic-decode constants of the decompress kernel (layout: ecco_format.h)
-    uint8_t* rl = base + kOffRankLut;
-    uint32_t* ar = reinterpret_cast<uint32_t*>(base + kOffArith);
-    const uint32_t n_cb = kMaxPatterns * kCodebooks;
+    // codebook records: shape, pair table, symbol -> rank (rank = position in (length, symbol id) order)
+    uint32_t* rec = reinterpret_cast<uint32_t*>(base + kOffCbRec);
     for (int k = 0; k < kMaxPatterns; ++k)
         for (int c = 0; c < kCodebooks; ++c) {
-            const uint32_t cb = static_cast<uint32_t>(k) * kCodebooks + c, rot = lut_rotation(cb);
-            int len[kSymbols];
-            uint32_t code[kSymbols];                       // codeword value, first code bit on top
-            for (int s = 0; s < kSymbols; ++s) {
-                len[s] = k < tmp.S ? tmp.cb_len[k][c][s] : 4;
-                code[s] = k < tmp.S ? bit_reverse(tmp.cb_rev[k][c][s], len[s]) : static_cast<uint32_t>(s);
-            }
-            // first[L]: smallest codeword of length L; ahead[L]: number of symbols with shorter codewords
-            uint32_t first[kMaxLen + 2] = {0}, count[kMaxLen + 2] = {0}, ahead[kMaxLen + 2] = {0}, thr[kMaxLen + 2] = {0};
-            for (int s = 0; s < kSymbols; ++s) ++count[len[s]];
-            uint32_t next = 0, seen = 0;
-            for (int L = 1; L <= kMaxLen; ++L) {
-                first[L] = next; ahead[L] = seen;
-                thr[L] = (next + count[L]) << (kMaxLen - L);   // <= 256: first window byte past the codewords of length <= L
-                next = (next + count[L]) << 1; seen += count[L];
-            }
-            const uint32_t rho = count[kMaxLen] ? (first[kMaxLen] - ahead[kMaxLen]) & 15u : 0u;
-            uint32_t delta[kMaxLen + 1];
-            for (int L = kMinLen; L <= kMaxLen; ++L) delta[L] = (ahead[L] + rho - first[L]) & 15u;
+            const int sh = p.shape_of[k][c];
             uint64_t rank_of = 0;
-            uint8_t* t = rl + static_cast<size_t>(cb) * 256;
-            for (int s = 0; s < kSymbols; ++s) {
-                const int L = len[s];
-                const uint32_t rank = (code[s] + delta[L]) & 15u;
-                rank_of |= static_cast<uint64_t>(rank) << (4 * s);
-                const uint32_t rev = bit_reverse(code[s], L);
-                for (uint32_t hi = 0; hi < (1u << (kMaxLen - L)); ++hi)
-                    t[(rev | (hi << L)) ^ rot] = static_cast<uint8_t>((L << 4) | rank);
-            }
-            uint32_t w0 = 0xC0000000u, w1 = 0, w2 = 0;
-            for (int i = 0; i < 3; ++i) {
-                w0 |= (256u - thr[2 + i]) << (10 * i);
-                w1 |= (256u - thr[5 + i]) << (10 * i + 1);
-            }
-            for (int L = kMinLen; L < kMaxLen; ++L) w2 |= delta[L] << (4 * (L - kMinLen));
-            ar[0 * n_cb + cb] = w0;
-            ar[1 * n_cb + cb] = w1;
-            ar[2 * n_cb + cb] = w2;
-            ar[3 * n_cb + cb] = static_cast<uint32_t>(rank_of);
-            ar[4 * n_cb + cb] = static_cast<uint32_t>(rank_of >> 32);
+            int rank = 0;
+            for (int L = kMinLen; L <= kMaxLen; ++L)
+                for (int s = 0; s < kSymbols; ++s)
+                    if ((k < tmp.S ? tmp.cb_len[k][c][s] : 4) == L) rank_of |= static_cast<uint64_t>(rank++) << (4 * s);
+            uint32_t* r = rec + (static_cast<size_t>(k) * kCodebooks + c) * 4;
+            r[0] = (p.pair_off[sh] >> 9) | (static_cast<uint32_t>(sh) << 8) | (static_cast<uint32_t>(p.width[sh]) << 16);
+            r[1] = 0;
+            r[2] = static_cast<uint32_t>(rank_of);
+            r[3] = static_cast<uint32_t>(rank_of >> 32);
         }
+    // shape tables, then pair tables built from them
+    for (int sh = 0; sh < p.n_shapes; ++sh) {
+        uint8_t* t = base + kOffShapeLut + static_cast<size_t>(sh) * 256;
+        uint32_t code = 0;
+        int rank = 0;
+        for (int L = kMinLen; L <= kMaxLen; ++L) {
+            for (int i = 0; i < p.counts[sh][L]; ++i, ++code, ++rank) {
+                const uint32_t rev = bit_reverse(code, L);
+                for (uint32_t hi = 0; hi < (1u << (kMaxLen - L)); ++hi) t[rev | (hi << L)] = static_cast<uint8_t>((L << 4) | rank);
+            }
+            code <<= 1;
+        }
+        const int W = p.width[sh];
+        if (!W) continue;
+        uint16_t* pt = reinterpret_cast<uint16_t*>(base + p.off_pair + p.pair_off[sh]);
+        for (uint32_t idx = 0; idx < (1u << W); ++idx) {
+            const uint32_t e0 = t[idx & 255u], l0 = e0 >> 4, r0 = e0 & 15u;
+            const uint32_t room = static_cast<uint32_t>(W) - l0;              // bits of the window after the first codeword
+            const uint32_t e1 = t[(idx >> l0) & 255u], l1 = e1 >> 4, r1 = e1 & 15u;   // bits past the window read as zero
+            // a codeword no longer than the bits on hand is fully inside them, so it is the real one
+            pt[idx] = l1 <= room ? static_cast<uint16_t>((l0 + l1) | (r0 << 7) | (r1 << 11))
+                                 : static_cast<uint16_t>(l0 | (r0 << 7) | 0x8000u);
+        }
+    }
+    DevHeader h;
+    std::memset(&h, 0, sizeof h);
+    h.magic = kDevMagic; h.version = kDevVersion; h.S = tmp.S; h.H = kCodebooks; h.e = tmp.e;
+    h.T = std::ldexp(1.0f, tmp.e);
+    h.total_bytes = p.total_bytes;
+    h.n_shapes = static_cast<uint32_t>(p.n_shapes);
+    h.shape_bytes = static_cast<uint32_t>(p.n_shapes) * 256u;
+    h.pair_bytes = p.pair_bytes;
+    h.pair_align = p.pair_align;
+    h.off_pair = p.off_pair;
+    uint64_t hash = 1469598103934665603ull;
+    hash = fnv1a(base + kOffPattern, kFixedTableBytes, hash);
+    hash = fnv1a(base + kOffShapeLut, p.total_bytes - kOffShapeLut, hash);
+    h.hash_lo = static_cast<uint32_t>(hash);
+    h.hash_hi = static_cast<uint32_t>(hash >> 32);
+    std::memcpy(base, &h, sizeof h);
     return ECCO_OK;
 }
 

@@ -6,16 +6,15 @@
 // groups, not inside a group.  The lanes of a warp advance symbol by symbol in lock step, which
 // keeps every per-symbol index (output position, activation element) uniform across the warp.
 //
-// Shared memory per CTA:
-//   tables   pattern[64][16] fp16 | ID_KP table [4096] u16 | symbol tables [256][256] u8,
-//            brought in by one bulk copy (cp.async.bulk + mbarrier); the tile-store decompress
-//            kernel takes the rank-valued tables and the arithmetic-decode constants instead
-//            (two copies, 80 KB)
-//   per warp bits[18][32] u32   the warp's 32 blocks, word-transposed: lane L's word w at
+// Shared memory per CTA (sizes from the image's header, see ecco_device_core.cuh):
+//   tables   pattern[64][16] fp16 | ID_KP table [4096] u16 | codebook records [256] x 16 B | shape tables
+//            [n_shapes][256] u8 | pair tables, brought in by three bulk copies (cp.async.bulk + mbarrier)
+//   per warp tab[16][32]  u32   per-lane dequantised centroids in rank order (the rank of the abs-max symbol
+//                               holds the abs-max)
+//            bits[18][32] u32   the warp's 32 blocks, word-transposed: lane L's word w at
 //                               [w][L] -> bank L whatever w is (conflict-free refills);
 //                               rows 16 and 17 stay zero (stream bits past 512 read as 0)
-//            tab[16][32]  u32   per-lane dequantised centroids (entry 15 = the abs-max)
-//            syms[16][32] u32   (fused kernels) decoded indices, 8 nibbles per word, for the
+//            syms[16][32] u32   (fused kernels) decoded ranks, 8 nibbles per word, for the
 //                               outlier fix-up
 //
 // Layout of the sources (one translation unit; the .cuh files are included here and nowhere else):
@@ -87,9 +86,16 @@ static bool make_out_map(CUtensorMap* map, void* d_out, uint64_t n_groups)
 }
 
 constexpr int kDecompressTmaWarps = 28;
-// symbols 1 and 3 of every four are decoded arithmetically, 0 and 2 through the byte table: measured best of
-// {none, one, two, three, all} on the 11008x4096 matrix and on a 256 MiB cache (all-table 441 us, this 394 us, all-arithmetic 459 us)
-constexpr uint32_t kDecompressArith = 0b1010;
+
+// every decoding kernel asks for all the shared memory of an SM and lays itself out on the device
+template <class K>
+static int want_all_smem(K kernel, bool* configured)
+{
+    if (*configured) return ECCO_OK;
+    const int rc = set_smem(kernel, kSmemCtaBytes);
+    if (rc == ECCO_OK) *configured = true;
+    return rc;
+}
 
 // tensors of fewer than 32 groups (the tile store's box is 32 rows tall), or when no tensor map can be made
 static int launch_decompress_small(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, void* d_out,
@@ -97,17 +103,12 @@ static int launch_decompress_small(const DeviceInfo& di, const void* d_meta, con
 {
     static thread_local bool configured[64] = {};
     auto kernel = ecco_decompress_kernel<kDecompressWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kDecompressWarps) * (kBitsBytes + kTabBytes);
-    if (!configured[di.device]) {
-        int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
+    int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
     const uint64_t cta_tiles = (n_groups + kDecompressWarps * 32 - 1) / (kDecompressWarps * 32);   // one tile per warp
     const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
-    kernel<<<grid, kDecompressWarps * 32, smem, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_groups,
-                                                          static_cast<uint16_t*>(d_out),
-                                                          balanced_warps((n_groups + 31) / 32, grid * kDecompressWarps));
+    kernel<<<grid, kDecompressWarps * 32, kSmemCtaBytes, stream>>>(static_cast<const uint8_t*>(d_meta), d_blocks, n_groups,
+                                                                   static_cast<uint16_t*>(d_out));
     return check_launch();
 }
 
@@ -115,32 +116,25 @@ static int launch_decompress_small(const DeviceInfo& di, const void* d_meta, con
 static int launch_decompress_batch(const DeviceInfo& di, DecompressBatch& batch, cudaStream_t stream)
 {
     static thread_local bool configured[64] = {};
-    auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps, kDecompressArith>;
-    constexpr size_t smem =
-        ((kSmemRankWarpBase + static_cast<size_t>(kDecompressTmaWarps) * (kBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
-        static_cast<size_t>(kDecompressTmaWarps) * 1024 + 512 + 16;           // + outlier value table + barrier
-    static_assert(smem <= 232448, "227 KB per CTA");
-    if (!configured[di.device]) {
-        int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
-    uint64_t cta_tiles = 0;
-    for (int t = 0; t < batch.n; ++t) {
-        const uint64_t c = (batch.job[t].n_groups + kDecompressTmaWarps * 32 - 1) / (kDecompressTmaWarps * 32);
-        cta_tiles = c > cta_tiles ? c : cta_tiles;
-    }
-    const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
-    for (int t = 0; t < batch.n; ++t)
-        batch.job[t].active_warps = balanced_warps((batch.job[t].n_groups + 31) / 32, grid * kDecompressTmaWarps);
-    return launch_overlapped(kernel, grid, static_cast<unsigned>(kDecompressTmaWarps * 32), smem, stream, batch);
+    auto kernel = ecco_decompress_tma_kernel<kDecompressTmaWarps>;
+    int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
+    uint64_t tiles = 0;
+    for (int t = 0; t < batch.n; ++t) tiles += (batch.job[t].n_groups + 31) / 32;
+    const uint64_t ctas = (tiles + kDecompressTmaWarps - 1) / kDecompressTmaWarps;
+    const unsigned grid = static_cast<unsigned>(ctas < static_cast<uint64_t>(di.sms) ? ctas : di.sms);
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kDecompressTmaWarps * 32), kSmemCtaBytes, stream, batch);
 }
+
+// The tile-store kernel addresses output rows with the 32-bit signed coordinates of the TMA unit: tensors of 2^31 groups
+// (256 GiB of fp16) or more are refused.
+constexpr uint64_t kMaxGroups = (1ull << 31) - 32;
 
 static int check_decompress_args(const void* d_meta, const uint8_t* d_blocks, uint64_t n_groups, const void* d_out)
 {
     if (!d_meta || !d_blocks || !d_out) return ECCO_ERR_INVALID_ARG;
     if (!aligned16(d_meta) || !aligned16(d_blocks) || !aligned16(d_out)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    if (n_groups > kMaxGroups) return ECCO_ERR_INVALID_ARG;
     return ECCO_OK;
 }
 
@@ -192,7 +186,7 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     return ecco_decompress_batch(&item, 1, stream);
 }
 
-constexpr int kVarWarps = 18;
+constexpr int kVarWarps = 24;
 
 extern "C" int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, const void* d_index, uint64_t n_groups, void* d_out,
                                    void* stream)
@@ -200,29 +194,22 @@ extern "C" int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, 
     if (n_groups == 0) return ECCO_OK;
     if (!d_meta || !d_stream || !d_index || !d_out) return ECCO_ERR_INVALID_ARG;
     if (!aligned16(d_meta) || !aligned16(d_stream) || !aligned16(d_out) || (reinterpret_cast<uintptr_t>(d_index) & 7u)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    if (n_groups > kMaxGroups) return ECCO_ERR_INVALID_ARG;
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;
-    // the tile store needs 32 rows: pad the logical row count of tiny tensors is not possible, so they are refused
+    // rows past the end of the tensor are dropped by the tile store, so any n_groups >= 1 works
     CUtensorMap map;
     if (!make_out_map(&map, d_out, n_groups)) return ECCO_ERR_CUDA;
     auto kernel = ecco_var_decompress_kernel<kVarWarps>;
-    constexpr size_t smem =
-        ((kSmemWarpBase + static_cast<size_t>(kVarWarps) * (kVarBitsBytes + kTabBytes) + 1023) & ~static_cast<size_t>(1023)) +
-        static_cast<size_t>(kVarWarps) * 1024;
     static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
+    rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
     const uint64_t cta_tiles = (n_groups + kVarWarps * 32 - 1) / (kVarWarps * 32);
     const unsigned grid = static_cast<unsigned>(cta_tiles < static_cast<uint64_t>(di.sms) ? cta_tiles : di.sms);
-    const uint32_t active = balanced_warps((n_groups + 31) / 32, grid * kVarWarps);
-    return launch_overlapped(kernel, grid, static_cast<unsigned>(kVarWarps * 32), smem, static_cast<cudaStream_t>(stream),
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kVarWarps * 32), kSmemCtaBytes, static_cast<cudaStream_t>(stream),
                              static_cast<const uint8_t*>(d_meta), reinterpret_cast<const uint4*>(d_stream),
-                             static_cast<const uint64_t*>(d_index), n_groups, static_cast<uint16_t*>(d_out), active, map);
+                             static_cast<const uint64_t*>(d_index), n_groups, static_cast<uint16_t*>(d_out), map);
 }
 
 extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch)
@@ -238,24 +225,19 @@ static int launch_gemv_mma(const DeviceInfo& di, const void* d_meta, const uint8
                            const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     auto kernel = ecco_gemv_mma_kernel<kMmaWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kMmaWarps) * kMmaWarpBytes;
     static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
+    int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
     const GemvPlan p = gemv_mma_plan(n_out, kblocks, di.sms < 256 ? di.sms : 256);
     if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-    int rc = zero_tickets(tickets, p.ticket_bytes, stream);
+    rc = zero_tickets(tickets, p.ticket_bytes, stream);
     if (rc) return rc;
-    const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kMmaWarps));
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kMmaWarps * 32), smem, stream,
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kMmaWarps * 32), kSmemCtaBytes, stream,
                              static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), batch, d_y,
-                             partial, tickets, active);
+                             partial, tickets);
 }
 
 // one or two rows of x (batch == kV): the per-warp kernel
@@ -265,24 +247,19 @@ static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint
 {
     constexpr int kFusedWarps = gemv_warp_warps(kV);
     auto kernel = ecco_gemv_warp_kernel<kV, kFusedWarps>;
-    const size_t smem = kFusedBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes + kGroup * kV * 4);
     static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
+    int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
     const GemvPlan p = gemv_warp_plan(n_out, kblocks, kV, di.sms < 256 ? di.sms : 256);
     if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
-    int rc = zero_tickets(tickets, p.ticket_bytes, stream);
+    rc = zero_tickets(tickets, p.ticket_bytes, stream);
     if (rc) return rc;
-    const int active = static_cast<int>(balanced_warps(static_cast<uint64_t>(p.row_tiles) * kblocks, p.grid * kFusedWarps));
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kFusedWarps * 32), smem, stream,
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kFusedWarps * 32), kSmemCtaBytes, stream,
                              static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), d_y, partial,
-                             tickets, active);
+                             tickets);
 }
 
 extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x,
@@ -351,19 +328,16 @@ template <int kV>
 static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* d_kblocks, int batch, int n_kv_heads,
                        int seq, int q_per_kv, const void* d_q, float scale, float* d_scores, cudaStream_t stream)
 {
-    constexpr int kFusedWarps = fused_warps(kV), kFusedRows = kFusedWarps * 32;
+    constexpr int kFusedWarps = fused_warps(kV);
     auto kernel = ecco_attn_scores_kernel<kV, kFusedWarps>;
-    const size_t smem = kFusedBase + static_cast<size_t>(kFusedWarps) * (kBitsBytes + kTabBytes + kSymsBytes) + kGroup * kV * 4;
     static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
+    int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
     const int heads = batch * n_kv_heads;
-    const int64_t units = static_cast<int64_t>(heads) * ((seq + kFusedRows - 1) / kFusedRows);
-    const unsigned grid = balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(di.sms));   // persistent CTAs, same units each
-    return launch_overlapped(kernel, grid, static_cast<unsigned>(kFusedWarps * 32), smem, stream, static_cast<const uint8_t*>(d_meta),
+    // persistent CTAs; the units (a head's tokens in chunks of one per working thread) are split evenly on the device
+    const int64_t most_units = static_cast<int64_t>(heads) * ((seq + 31) / 32);
+    const unsigned grid = static_cast<unsigned>(most_units < di.sms ? most_units : di.sms);
+    return launch_overlapped(kernel, grid, static_cast<unsigned>(kFusedWarps * 32), kSmemCtaBytes, stream, static_cast<const uint8_t*>(d_meta),
                              d_kblocks, heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores);
 }
 
@@ -384,19 +358,14 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
         case 2: return launch_attn<2>(di, d_meta, d_kblocks, batch, n_kv_heads, seq, q_per_kv, d_q, scale, d_scores, s);
         default: {
             auto kernel = ecco_attn_scores_mma_kernel<kMmaWarps>;
-            const size_t smem = kSmemWarpBase + static_cast<size_t>(kMmaWarps) * kMmaWarpBytes;
             static thread_local bool configured[64] = {};
-            if (!configured[di.device]) {
-                rc = set_smem(kernel, smem);
-                if (rc) return rc;
-                configured[di.device] = true;
-            }
+            rc = want_all_smem(kernel, &configured[di.device]);
+            if (rc) return rc;
             const uint64_t units = static_cast<uint64_t>(batch) * n_kv_heads * ((seq + 31) / 32);
             const uint64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
             const unsigned grid = static_cast<unsigned>(ctas < static_cast<uint64_t>(di.sms) ? ctas : di.sms);
-            const int active = static_cast<int>(balanced_warps(units, grid * kMmaWarps));
-            return launch_overlapped(kernel, grid, static_cast<unsigned>(kMmaWarps * 32), smem, s, static_cast<const uint8_t*>(d_meta),
-                                     d_kblocks, batch * n_kv_heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores, active);
+            return launch_overlapped(kernel, grid, static_cast<unsigned>(kMmaWarps * 32), kSmemCtaBytes, s, static_cast<const uint8_t*>(d_meta),
+                                     d_kblocks, batch * n_kv_heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores);
         }
     }
 }
@@ -421,8 +390,9 @@ AvPlan av_plan(int batch, int n_kv_heads, int seq, int q_per_kv, int ctas_max)
     AvPlan p;
     p.warps = av_warps(seq);
     const int heads = batch * n_kv_heads;
-    const int64_t units = static_cast<int64_t>(heads) * ((seq + p.warps * 32 - 1) / (p.warps * 32));
-    p.grid = static_cast<int>(balanced_warps(static_cast<uint64_t>(units), static_cast<uint32_t>(ctas_max)));
+    // at most this many units (fewer when all p.warps warps find room); the device splits what there is evenly
+    const int64_t units = static_cast<int64_t>(heads) * ((seq + 31) / 32);
+    p.grid = static_cast<int>(units < ctas_max ? units : ctas_max);
     auto up = [](size_t v) { return (v + 255) & ~static_cast<size_t>(255); };
     p.stats_bytes = up(static_cast<size_t>(heads) * q_per_kv * sizeof(float2));
     p.partial_bytes = up(static_cast<size_t>(p.grid + heads) * kGroup * 8 * sizeof(float));
@@ -436,14 +406,10 @@ int launch_attn_values(const DeviceInfo& di, const AvPlan& p, const void* d_meta
                        cudaStream_t s)
 {
     auto kernel = ecco_attn_values_kernel<kWarps>;
-    const size_t smem = kSmemWarpBase + static_cast<size_t>(kWarps) * kAvWarpBytes + kGroup * 8 * sizeof(float);
     static thread_local bool configured[64] = {};
-    if (!configured[di.device]) {
-        const int rc = set_smem(kernel, smem);
-        if (rc) return rc;
-        configured[di.device] = true;
-    }
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kWarps * 32), smem, s,
+    const int rc = want_all_smem(kernel, &configured[di.device]);
+    if (rc) return rc;
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kWarps * 32), kSmemCtaBytes, s,
                              static_cast<const uint8_t*>(d_meta), d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets);
 }
 }  // namespace
@@ -492,7 +458,7 @@ extern "C" int ecco_act_decompress(const uint8_t* d_blocks, uint64_t n_groups, v
     if (n_groups == 0) return ECCO_OK;
     if (!d_blocks || !d_out_fp16) return ECCO_ERR_INVALID_ARG;
     if (!aligned16(d_blocks) || (reinterpret_cast<uintptr_t>(d_out_fp16) & 31u)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    if (n_groups > kMaxGroups) return ECCO_ERR_INVALID_ARG;
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;
@@ -507,7 +473,7 @@ extern "C" int ecco_act_compress(const void* d_x_fp16, uint64_t n_groups, uint8_
     if (n_groups == 0) return ECCO_OK;
     if (!d_blocks || !d_x_fp16) return ECCO_ERR_INVALID_ARG;
     if (!aligned16(d_blocks) || (reinterpret_cast<uintptr_t>(d_x_fp16) & 31u)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    if (n_groups > kMaxGroups) return ECCO_ERR_INVALID_ARG;
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;
@@ -523,7 +489,7 @@ extern "C" int ecco_kv_compress(const void* d_meta, const void* d_x_fp16, uint64
     if (n_groups == 0) return ECCO_OK;
     if (!d_meta || !d_x_fp16 || !d_blocks) return ECCO_ERR_INVALID_ARG;
     if (!aligned16(d_meta) || !aligned16(d_x_fp16) || !aligned16(d_blocks)) return ECCO_ERR_ALIGNMENT;
-    if (n_groups > (1ull << 40)) return ECCO_ERR_INVALID_ARG;
+    if (n_groups > kMaxGroups) return ECCO_ERR_INVALID_ARG;
     DeviceInfo di;
     int rc = device_info(&di);
     if (rc) return rc;

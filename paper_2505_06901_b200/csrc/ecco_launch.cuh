@@ -7,14 +7,6 @@ namespace {
 // ---------------------------------------------------------------------------------------------
 // host-side launch helpers
 // ---------------------------------------------------------------------------------------------
-// number of working warps <= w_max such that `units` split evenly: all get ceil(units / w_max) or one less
-inline uint32_t balanced_warps(uint64_t units, uint32_t w_max)
-{
-    if (units <= w_max) return static_cast<uint32_t>(units);
-    const uint64_t per_warp = (units + w_max - 1) / w_max;
-    return static_cast<uint32_t>((units + per_warp - 1) / per_warp);
-}
-
 struct DeviceInfo {
     int device = -1, sms = 0, cc_major = 0;
     bool ok = false;
@@ -94,11 +86,11 @@ int check_launch()
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-constexpr int kDecompressWarps = 32;
-// warps per CTA of the scalar fused kernels (one or two dot products per group): as many as shared memory allows
-constexpr int fused_warps(int) { return 22; }
-// per-warp GEMV: every warp also carries its own slice of x, which leaves room for 22 / 20 warps
-constexpr int gemv_warp_warps(int kV) { return kFusedRank ? (kV >= 2 ? 20 : 21) : (kV >= 2 ? 20 : 22); }
+// Warps per CTA the decoding kernels are launched with (their register budget); how many of them work is decided on
+// the device, from the size of the image's tables.
+constexpr int kDecompressWarps = 28;
+constexpr int fused_warps(int) { return 20; }
+constexpr int gemv_warp_warps(int) { return 20; }
 
 struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
 

@@ -13,6 +13,16 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (run with -m gpu on a B200)")
 
 
+def pytest_terminal_summary(terminalreporter):
+    """Largest errors of the fused calls against the oracle's fp64 results, as measured in this run."""
+    import helpers
+
+    if helpers.FUSED_MAXIMA:
+        terminalreporter.write_line("fused calls, largest error seen: |y - ref| / sum|w x|, plain relative (|ref| >= 0.1 rms)")
+        for label, (scaled, plain) in sorted(helpers.FUSED_MAXIMA.items()):
+            terminalreporter.write_line(f"  {label:24s} {scaled:.3e}  {plain:.3e}")
+
+
 @pytest.fixture(scope="session")
 def eo():
     from oracle import ecco_oracle

@@ -21,3 +21,13 @@ def oracle_meta_from_lib(eo, lmeta):
             for s in range(16):
                 m.cb_len[k][h][s] = int(cb[k, h, s])
     return m
+
+
+# Largest errors the fused calls showed in this run, per label: {label: [max |y - ref| / sum|w x|, max plain relative
+# error where |ref| >= 0.1 rms]}.  conftest.py prints them at the end of the session.
+FUSED_MAXIMA = {}
+
+
+def record_fused(label, scaled, plain):
+    a, b = FUSED_MAXIMA.get(label, (0.0, 0.0))
+    FUSED_MAXIMA[label] = (max(a, float(scaled)), max(b, float(plain)))

@@ -154,81 +154,153 @@ def test_host_calibrator_yields_valid_and_useful_metadata(binding, eo, synth):
         binding.ecco_calibrate_host(cal[:1, :128 * 8].copy(), S=64)   # fewer groups than patterns
 
 
-def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small):
-    """The prebuilt lookup tables, read on the CPU: walking a block with them gives the oracle's
-    symbols and end position (checks table layout and bit order without a GPU)."""
-    ometa = cfg1_small["meta"]
-    lm = lib_meta_from_oracle(binding, ometa)
-    img = binding.ecco_meta_serialize_device(lm)
-    assert img.size == binding.ecco_meta_device_bytes(lm) == 84160 + 65536 + 5120
+OFF_PATTERN, OFF_KP, OFF_REC, OFF_ENC_CB, OFF_ENC_KP, OFF_SHAPE = 64, 2112, 10304, 14400, 22592, 22720
+
+
+def _image_views(img):
+    """The sections of a device image (layout: csrc/ecco_format.h), as numpy views."""
     hdr = img[:64].view(np.uint32)
-    assert hdr[0] == 0x4F434345 and hdr[2] == 64 and hdr[3] == 4 and hdr[4:5].view(np.int32)[0] == ometa.e
-    assert img[20:24].view(np.float32)[0] == 2.0 ** ometa.e
-    pat = img[64:64 + 2048].view(np.float16).reshape(64, 16)
-    assert np.array_equal(pat[:, :15].view(np.uint16), ometa.patterns().view(np.uint16)) and np.all(pat[:, 15] == 0)
-    kpl = img[64 + 2048:64 + 2048 + 8192].view(np.uint16)
-    syml = img[64 + 2048 + 8192:64 + 2048 + 8192 + 65536].reshape(256, 256)
-    enc = img[75840:75840 + 8192].view(np.uint16).reshape(64, 4, 16)
-    assert np.array_equal(enc >> 8, ometa.cb_lengths())                  # encoder table: lengths per (pattern, codebook, symbol)
-    assert np.array_equal(img[84032:84160].view(np.uint16) >> 12, ometa.kp_lengths())
-    assert np.all((syml >> 4) >= 2) and np.all((syml >> 4) <= 8)
-    for g in range(0, 2048, 41):
-        blk = cfg1_small["blocks"][g]
-        _, sym, info = eo.decode_block(ometa, blk)
-        bits = int.from_bytes(blk.tobytes(), "little")
-        e = int(kpl[(bits >> 10) & 0xFFF])
-        assert e & 0xFF == info.kp
-        pos = 10 + (e >> 8)
-        cb = info.kp * 4 + info.hf
-        lut = syml[cb]
-        rot = ((cb * 11 + (cb >> 3)) & 31) << 2          # per-codebook index rotation of the image
-        n = 0
-        while n < 128:
-            t = int(lut[((bits >> pos) & 0xFF) ^ rot])
-            if pos + (t >> 4) > 512:
-                break
-            assert (t & 15) == sym[n]
-            pos += t >> 4
-            n += 1
-        assert n == info.n_fit and pos == info.end_bit
+    n_shapes, shape_bytes, pair_bytes, pair_align, off_pair = (int(v) for v in hdr[7:12])
+    v = dict(hdr=hdr, n_shapes=n_shapes, pair_bytes=pair_bytes, pair_align=pair_align, off_pair=off_pair)
+    assert shape_bytes == n_shapes * 256 and off_pair == (OFF_SHAPE + shape_bytes + 15) // 16 * 16
+    assert img.size == hdr[6] == off_pair + pair_bytes
+    v["pattern"] = img[OFF_PATTERN:OFF_KP].view(np.float16).reshape(64, 16)
+    v["kp"] = img[OFF_KP:OFF_REC].view(np.uint16)
+    v["rec"] = img[OFF_REC:OFF_ENC_CB].view(np.uint32).reshape(256, 4)
+    v["enc_cb"] = img[OFF_ENC_CB:OFF_ENC_KP].view(np.uint16).reshape(64, 4, 16)
+    v["enc_kp"] = img[OFF_ENC_KP:OFF_SHAPE].view(np.uint16)
+    v["shape"] = img[OFF_SHAPE:OFF_SHAPE + shape_bytes].reshape(n_shapes, 256)
+    v["pair"] = img[off_pair:off_pair + pair_bytes]
+    return v
 
 
-def test_device_image_rank_tables_and_arithmetic_constants(binding, eo, cfg1_small):
-    """The mixed decoder's tables against the oracle's canonical codes: for every codebook and every 8-bit
-    window, the rank table has the oracle's codeword length and a rank that is a bijection of the symbol,
-    and the arithmetic route (threshold compare, codeword + delta) lands on the same length and rank."""
+def _walk_with_image_tables(v, blk):
+    """A block decoded the way the kernels do it, in Python: four symbols per step from a window that starts one
+    bit early, two pair-table lookups, escapes completed through the shape table, and the one-symbol-per-lookup
+    walk with the clip test once a step could cross bit 512.  -> (kp, hf, symbols, end bit or 0)."""
+    bits = int.from_bytes(blk.tobytes(), "little")         # stream bit k = bit k of this integer; bits past 511 are zero
+    hf = (bits >> 8) & 3
+    e = int(v["kp"][(bits >> 10) & 0xFFF])
+    kp, pos = e & 0xFF, 10 + (e >> 8)
+    rec = v["rec"][kp * 4 + hf]
+    shape, width, pair_off = (int(rec[0]) >> 8) & 0xFF, int(rec[0]) >> 16, (int(rec[0]) & 0xFF) << 9
+    rank_of = int(rec[2]) | int(rec[3]) << 32
+    sym_of_rank = {(rank_of >> 4 * s) & 15: s for s in range(16)}
+    assert len(sym_of_rank) == 16
+    blut = v["shape"][shape]
+    plut = v["pair"][pair_off:pair_off + (2 << width)].view(np.uint16) if width else None
+    mask = ((1 << width) - 1) << 1
+    ranks, alive = [], True
+
+    def entry(off):                                        # signed 16-bit pair-table entry at byte offset off
+        x = int(plut[off >> 1])
+        return x - 65536 if x & 0x8000 else x
+
+    def resolve(e, p):
+        b = int(blut[(bits >> (p + (e & 15))) & 0xFF])
+        return (e & 0x078F) + (b >> 4) + ((b & 15) << 11)
+
+    for step in range(32):
+        single = plut is None
+        if not single:
+            win = (bits >> (pos - 1)) & 0xFFFFFFFF
+            e0 = entry(win & mask)
+            if e0 < 0:
+                e0 = resolve(e0, pos)
+            e1 = entry((win >> (e0 & 31)) & mask)
+            if e1 < 0:
+                e1 = resolve(e1, pos + (e0 & 31))
+            acc = (e0 + e1) & 0x7F
+            if pos + acc > 512:
+                single = True
+            else:
+                ranks += [(e0 >> 7) & 15, (e0 >> 11) & 15, (e1 >> 7) & 15, (e1 >> 11) & 15]
+                pos += acc
+        if single:
+            for _ in range(4):
+                t = int(blut[(bits >> pos) & 0xFF]) if pos < 520 else int(blut[0])
+                if alive and pos + (t >> 4) <= 512:
+                    ranks.append(t & 15)
+                else:
+                    alive = False
+                pos += t >> 4
+    return kp, hf, [sym_of_rank[r] for r in ranks], pos if alive else 0
+
+
+def test_device_image_tables_decode_like_the_oracle(binding, eo, cfg1_small, kv_small):
+    """The prebuilt lookup tables, read on the CPU: walking a block with them, the way the kernels do, gives the
+    oracle's symbols and end position (checks table layout, bit order, escapes and the clip rule without a GPU)."""
+    for fx in (cfg1_small, kv_small):
+        ometa = fx["meta"]
+        lm = lib_meta_from_oracle(binding, ometa)
+        img = binding.ecco_meta_serialize_device(lm)
+        assert img.size == binding.ecco_meta_device_bytes(lm)
+        v = _image_views(img)
+        hdr = v["hdr"]
+        assert hdr[0] == 0x4F434345 and hdr[1] == 4 and hdr[2] == 64 and hdr[3] == 4 and hdr[4:5].view(np.int32)[0] == ometa.e
+        assert img[20:24].view(np.float32)[0] == 2.0 ** ometa.e
+        assert np.array_equal(v["pattern"][:, :15].view(np.uint16), ometa.patterns().view(np.uint16)) and np.all(v["pattern"][:, 15] == 0)
+        assert np.array_equal(v["enc_cb"] >> 8, ometa.cb_lengths())      # encoder table: lengths per (pattern, codebook, symbol)
+        assert np.array_equal(v["enc_kp"] >> 12, ometa.kp_lengths())
+        assert v["pair_bytes"] > 0 and v["n_shapes"] < 64
+        assert np.all((v["shape"] >> 4) >= 2) and np.all((v["shape"] >> 4) <= 8)
+        escapes = 0
+        for g in range(0, 2048, 13):
+            blk = fx["blocks"][g]
+            _, sym, info = eo.decode_block(ometa, blk)
+            kp, hf, got, end = _walk_with_image_tables(v, blk)
+            assert (kp, hf) == (info.kp, info.hf)
+            assert len(got) == info.n_fit and got == [int(x) for x in sym[:info.n_fit]]
+            assert end == (info.end_bit if info.n_fit == 128 else 0)
+        # random blocks too: whatever the header bits select must decode like the oracle says
+        rb = np.random.Generator(np.random.PCG64(4)).integers(0, 256, size=(150, 64), dtype=np.uint8)
+        for blk in rb:
+            _, sym, info = eo.decode_block(ometa, blk)
+            kp, hf, got, end = _walk_with_image_tables(v, blk)
+            assert (kp, hf) == (info.kp, info.hf) and got == [int(x) for x in sym[:info.n_fit]]
+
+
+def test_device_image_shape_and_pair_tables_against_canonical_codes(binding, eo, cfg1_small):
+    """Every codebook's record, shape table and pair table against the oracle's canonical code: ranks are a
+    bijection of the symbols in (length, id) order; for every 8-bit window the shape table has the codeword's
+    length and rank; for every W-bit window the pair table has both symbols when the second codeword ends inside
+    the window and an escape with the first symbol otherwise; tables are aligned to their size, widest first."""
     ometa = cfg1_small["meta"]
     lm = lib_meta_from_oracle(binding, ometa)
-    img = binding.ecco_meta_serialize_device(lm)
-    syml = img[64 + 2048 + 8192:64 + 2048 + 8192 + 65536].reshape(256, 256)
-    rankl = img[84160:84160 + 65536].reshape(256, 256)
-    ar = img[84160 + 65536:].view(np.uint32).reshape(5, 256)
-    lengths = ometa.cb_lengths()                                   # [pattern][codebook][symbol]
-    spread = 1 | 1 << 10 | 1 << 20
-    guard = 0x100 | 0x100 << 10 | 0x100 << 20
+    v = _image_views(binding.ecco_meta_serialize_device(lm))
+    lengths = ometa.cb_lengths()
+    widths_by_offset = {}
     for cb in range(ometa.S * 4):
         lens = [int(x) for x in lengths[cb // 4, cb % 4]]
         codes, kraft = eo.canonical_codes(lens, 8)
         assert kraft == 256
-        rot = ((cb * 11 + (cb >> 3)) & 31) << 2
-        c1, c2, d, rlo, rhi = (int(ar[i, cb]) for i in range(5))
-        rank_of = rlo | rhi << 32
-        assert sorted((rank_of >> 4 * s) & 15 for s in range(16)) == list(range(16))
-        delta = {L: (d >> 4 * (L - 2)) & 15 for L in range(2, 8)}
-        delta[8] = 0
-        for s in range(16):                                        # every window that starts with the codeword of s
+        rec = v["rec"][cb]
+        shape, width, pair_off = (int(rec[0]) >> 8) & 0xFF, int(rec[0]) >> 16, (int(rec[0]) & 0xFF) << 9
+        rank_of = int(rec[2]) | int(rec[3]) << 32
+        order = sorted(range(16), key=lambda s: (lens[s], s))
+        assert [(rank_of >> 4 * s) & 15 for s in order] == list(range(16))
+        want_len, want_rank = np.zeros(256, np.int64), np.zeros(256, np.int64)
+        for s in range(16):
             L, code = lens[s], int(codes[s])
             for rest in range(1 << (8 - L)):
-                b = code << (8 - L) | rest                         # first stream bit on top
-                i = int(f"{b:08b}"[::-1], 2)                       # the same window, first stream bit in bit 0
-                assert int(syml[cb, i ^ rot]) == (L << 4 | s)
-                assert int(rankl[cb, i ^ rot]) == (L << 4 | ((rank_of >> 4 * s) & 15))
-                m = ((b * spread + c1) & 0xFFFFFFFF & (guard | 0xC0000000)) | ((b * 2 * spread + c2) & 0xFFFFFFFF & (2 * guard))
-                assert bin(m).count("1") == L
-                assert ((b >> (8 - L)) + delta[L]) & 15 == (rank_of >> 4 * s) & 15
-    # rows of unused patterns decode as sixteen 4-bit codewords in every table
-    for cb in range(ometa.S * 4, 256):
-        assert np.all(rankl[cb] >> 4 == 4) and np.all(syml[cb] >> 4 == 4)
+                i = int(f"{code << (8 - L) | rest:08b}"[::-1], 2)     # the window with the first stream bit in bit 0
+                want_len[i], want_rank[i] = L, (rank_of >> 4 * s) & 15
+        assert np.array_equal(v["shape"][shape] >> 4, want_len) and np.array_equal(v["shape"][shape] & 15, want_rank)
+        assert 8 <= width <= 12 and pair_off % (2 << width) == 0
+        widths_by_offset[pair_off] = width
+        pt = v["pair"][pair_off:pair_off + (2 << width)].view(np.uint16).astype(np.int64)
+        idx = np.arange(1 << width)
+        l0, r0 = want_len[idx & 255], want_rank[idx & 255]
+        rest = idx >> l0
+        l1, r1 = want_len[rest & 255], want_rank[rest & 255]
+        fits = l0 + l1 <= width
+        assert np.array_equal(pt[fits], (l0 + l1 + (r0 << 7) + (r1 << 11))[fits])
+        assert np.array_equal(pt[~fits], (l0 + (r0 << 7) + 0x8000)[~fits])
+        assert fits.mean() > 0.5
+    offs = sorted(widths_by_offset)
+    assert offs[0] == 0 and all(widths_by_offset[a] >= widths_by_offset[b] for a, b in zip(offs, offs[1:]))
+    assert v["pair_align"] == 2 << widths_by_offset[0]
+    assert sum(2 << w for w in widths_by_offset.values()) == v["pair_bytes"] <= 64 * 1024
 
 
 def _complete_length_multisets():
@@ -248,54 +320,30 @@ def _complete_length_multisets():
     return out
 
 
-def test_rank_tables_and_arithmetic_constants_for_every_code_shape(binding, eo):
-    """The mixed decoder's tables over EVERY admissible shape of a 2..8-bit code on 16 symbols (all multisets of
-    lengths with Kraft sum 1, lengths dealt to the symbols at random): for all 256 window bytes the arithmetic
-    route gives the canonical code's length, and codeword + delta is a bijection onto the ranks that agrees with
-    the rank table.  The expected lengths and codewords come from the oracle's canonical-code routine."""
+def test_device_image_for_every_code_shape(binding, eo):
+    """EVERY admissible shape of a 2..8-bit code on 16 symbols (all multisets of lengths with Kraft sum 1, lengths
+    dealt to the symbols at random), 120 at a time (so that they fit pair tables of at least eight bits) and all
+    255 in one image (which then has no pair tables): blocks of random bits walked with the image's tables decode
+    like the oracle's."""
     shapes = _complete_length_multisets()
-    assert len(shapes) > 200 and (0, 0, 16, 0, 0, 0, 0) in shapes and (3, 0, 3, 0, 2, 0, 8) in shapes
+    assert len(shapes) == 255 and (0, 0, 16, 0, 0, 0, 0) in shapes and (3, 0, 3, 0, 2, 0, 8) in shapes
     rng = np.random.Generator(np.random.PCG64(2024))
-    spread = 1 | 1 << 10 | 1 << 20
-    guard = 0x100 | 0x100 << 10 | 0x100 << 20
-    per_meta = 64 * 4
     kp_len = eo.huffman_limited(np.ones(64), 12)
     pat = np.sort(rng.uniform(-1, 1, (64, 15)), axis=1).astype(np.float16)
-    for base in range(0, len(shapes), per_meta):
-        chunk = shapes[base:base + per_meta]
-        cb = np.full((64, 4, 16), 4, dtype=np.uint8)
-        for i, counts in enumerate(chunk):
-            lens = np.repeat(np.arange(2, 9), counts)
-            cb[i // 4, i % 4] = rng.permutation(lens)
+    for chunk, want_pairs in ((shapes[:120], True), (shapes[135:], True), (shapes + shapes[:1], False)):
+        cb = np.zeros((64, 4, 16), dtype=np.uint8)
+        for i in range(256):
+            cb[i // 4, i % 4] = rng.permutation(np.repeat(np.arange(2, 9), chunk[i % len(chunk)]))
         lm = binding.ecco_meta_create(64, -5, pat, cb, kp_len)
-        img = binding.ecco_meta_serialize_device(lm)
-        rankl = img[84160:84160 + 65536].reshape(256, 256)
-        ar = img[84160 + 65536:].view(np.uint32).reshape(5, 256)
-        for i in range(len(chunk)):
-            lens = [int(x) for x in cb[i // 4, i % 4]]
-            codes, kraft = eo.canonical_codes(lens, 8)
-            assert kraft == 256
-            rot = ((i * 11 + (i >> 3)) & 31) << 2
-            c1, c2, d, rlo, rhi = (int(ar[j, i]) for j in range(5))
-            rank_of = rlo | rhi << 32
-            assert sorted((rank_of >> 4 * s) & 15 for s in range(16)) == list(range(16))
-            delta = {L: (d >> 4 * (L - 2)) & 15 for L in range(2, 8)}
-            delta[8] = 0
-            expect_len = np.zeros(256, dtype=np.int64)
-            expect_rank = np.zeros(256, dtype=np.int64)
-            for s in range(16):
-                L, code = lens[s], int(codes[s])
-                lo = code << (8 - L)
-                expect_len[lo:lo + (1 << (8 - L))] = L
-                expect_rank[lo:lo + (1 << (8 - L))] = (rank_of >> 4 * s) & 15
-            assert expect_len.min() >= 2                       # the code is complete: every window byte decodes
-            for b in range(256):
-                m = ((b * spread + c1) & 0xFFFFFFFF & (guard | 0xC0000000)) | ((b * 2 * spread + c2) & 0xFFFFFFFF & (2 * guard))
-                L = bin(m).count("1")
-                assert L == expect_len[b], (chunk[i], b)
-                assert ((b >> (8 - L)) + delta[L]) & 15 == expect_rank[b], (chunk[i], b)
-                rev = int(f"{b:08b}"[::-1], 2)
-                assert int(rankl[i, rev ^ rot]) == (L << 4 | expect_rank[b])
+        v = _image_views(binding.ecco_meta_serialize_device(lm))
+        assert v["n_shapes"] == min(len(chunk), 255) and (v["pair_bytes"] > 0) == want_pairs
+        om = oracle_meta_from_lib(eo, lm)
+        rb = rng.integers(0, 256, size=(300, 64), dtype=np.uint8)
+        for blk in rb:
+            _, sym, info = eo.decode_block(om, blk)
+            kp, hf, got, end = _walk_with_image_tables(v, blk)
+            assert (kp, hf) == (info.kp, info.hf) and got == [int(x) for x in sym[:info.n_fit]]
+            assert end == (info.end_bit if info.n_fit == 128 else 0)
 
 
 def test_variable_length_host_encoder_matches_oracle(binding, eo, cfg1_small, kv_small):
