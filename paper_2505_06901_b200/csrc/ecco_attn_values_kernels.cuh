@@ -64,7 +64,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const int tid = static_cast<int>(threadIdx.x), n_threads = static_cast<int>(blockDim.x);
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
-    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar fused kernels
     const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kGroup * 8 * sizeof(float));
     const int kTokens = static_cast<int>(nw) * 32;         // tokens per unit: one per thread of the working warps
     const bool working = warp < nw;

@@ -155,8 +155,7 @@ ecco_decompress_tma_kernel(const __grid_constant__ DecompressBatch batch)
             const DecompressJob& job = batch.job[c.job];
             return job.blocks + min((g - c.first) * 32 + lane, job.n_groups - 1) * kBlockBytes;
         };
-        Block blk;
-        if (gt < run_tiles) { seek(cur, gt); ldg_block(blk, block_ptr(cur, gt)); }
+        if (gt < run_tiles) { seek(cur, gt); prefetch_block_l2(block_ptr(cur, gt)); }
         if (!wait_tables(tb, static_cast<uint32_t>(run & 1))) return;
         float T = tb.T;
         int t_of_T = t0;
@@ -171,9 +170,13 @@ ecco_decompress_tma_kernel(const __grid_constant__ DecompressBatch batch)
             uint16_t* out = job.out + min(g, n_groups - 1) * kGroup;
             const CUtensorMap* out_map = &job.map;
             const int row0 = static_cast<int>(tile * 32);
+            // The block is fetched when its turn comes, after a prefetch into L2 one tile earlier: holding the next
+            // block in sixteen registers through a whole group would cost four of the 32 warps.
+            Block blk;
+            ldg_block(blk, block_ptr(cur, gt));
             const GroupHeader h = open_group<kTabHalf>(blk, tb, ws, T);
             const uint64_t gn = gt + tile_stride;
-            if (gn < run_tiles) { seek(cur, gn); ldg_block(blk, block_ptr(cur, gn)); }
+            if (gn < run_tiles) { seek(cur, gn); prefetch_block_l2(block_ptr(cur, gn)); }
             uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
             auto stage_rows = [&]() {
                 if (lane == 0) bulk_wait_read0();              // the engine has read the previous tile

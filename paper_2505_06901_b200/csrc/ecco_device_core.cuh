@@ -125,6 +125,11 @@ __device__ __forceinline__ void ldg_block(Block& b, const uint8_t* p)
                  : "=r"(b.w[8]), "=r"(b.w[9]), "=r"(b.w[10]), "=r"(b.w[11]), "=r"(b.w[12]), "=r"(b.w[13]), "=r"(b.w[14]), "=r"(b.w[15])
                  : "l"(p + 32));
 }
+__device__ __forceinline__ void prefetch_block_l2(const uint8_t* p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p + 32));
+}
 __device__ __forceinline__ void stg_v8(void* p, const uint32_t (&r)[8])
 {
     asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
@@ -172,14 +177,15 @@ struct Tables {
     float T;
     uint32_t hash_lo, hash_hi;
 };
-__device__ __forceinline__ Tables plan_tables(uint32_t smem_base, const uint8_t* d_meta)
+// use_pairs = false: the kernel decodes one symbol per lookup and leaves the pair tables out (more room for warps)
+__device__ __forceinline__ Tables plan_tables(uint32_t smem_base, const uint8_t* d_meta, bool use_pairs = true)
 {
     const DevHeader* hd = reinterpret_cast<const DevHeader*>(d_meta);
     Tables tb;
     tb.base = smem_base;
     tb.shape = smem_base + kSmemShapeLut;
     tb.shape_bytes = min(__ldg(&hd->shape_bytes), kMaxShapes * 256u) & ~255u;     // clamped: a bad header cannot overrun shared memory
-    tb.pair_bytes = min(__ldg(&hd->pair_bytes), kPairBudgetBytes) & ~511u;
+    tb.pair_bytes = use_pairs ? min(__ldg(&hd->pair_bytes), kPairBudgetBytes) & ~511u : 0u;
     const uint32_t align = min(max(__ldg(&hd->pair_align), 512u), 2u << kPairMaxBits);
     const uint32_t tables_end = tb.shape + tb.shape_bytes;
     tb.pair = tb.pair_bytes ? (tables_end + align - 1u) & ~(align - 1u) : tables_end;
@@ -371,9 +377,10 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         const uint32_t lo = lds_u32(ws.bits + qi * 128), hi = lds_u32(ws.bits + qi * 128 + 128);
         return lds_u8(h.blut | (__funnelshift_r(lo, hi, q) & 0xffu));
     };
-    // an escape entry completed with its second symbol, fetched at stream position p + (length of the first)
-    auto resolve = [&](int32_t e, uint32_t p) {
-        const uint32_t b = single_at(p + (static_cast<uint32_t>(e) & 15u));
+    // an escape entry completed with its second symbol, which starts `off` bits into the window (off = 1 + the bits
+    // before it); the window has it whole unless off > 24, which takes three 8-bit codewords in a row
+    auto resolve = [&](int32_t e, uint32_t win, uint32_t off, uint32_t p) {
+        const uint32_t b = off <= 24u ? lds_u8(h.blut | ((win >> off) & 0xffu)) : single_at(p + (static_cast<uint32_t>(e) & 15u));
         return static_cast<int32_t>((static_cast<uint32_t>(e) & 0x078fu) + (b >> 4) + ((b & 15u) << 11));
     };
     // Two symbols per lookup, software-pipelined by hand: a warp issues in order and every shared-memory load here is
@@ -406,10 +413,10 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         if (__any_sync(kFull, esc || (kTest && pos + acc > kEndBit))) {
             if (esc) {
                 if (e0 < 0) {
-                    e0 = resolve(e0, pos);
+                    e0 = resolve(e0, win, 1u + (static_cast<uint32_t>(e0) & 15u), pos);
                     e1 = lds_s16(h.plut | (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));
                 }
-                if (e1 < 0) e1 = resolve(e1, pos + (static_cast<uint32_t>(e0) & 31u));
+                if (e1 < 0) e1 = resolve(e1, win, 1u + (static_cast<uint32_t>(e0) & 31u) + (static_cast<uint32_t>(e1) & 15u), pos + (static_cast<uint32_t>(e0) & 31u));
                 acc = static_cast<uint32_t>(e0 + e1) & 0x7fu;
             }
             if (kTest && __any_sync(kFull, pos + acc > kEndBit)) {   // some lane's stream ends in this step
@@ -441,8 +448,12 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         for (int step = kFreeSteps; step < 32; ++step) four_pair(step, cuda::std::true_type{});
         if (pending) deliver(31);
     } else {
+        if (kFreeSteps > 0) {
 #pragma unroll 4
-        for (int step = 0; step < 32; ++step) four_single(step, cuda::std::true_type{});
+            for (int step = 0; step < kFreeSteps; ++step) four_single(step, cuda::std::false_type{});
+        }
+#pragma unroll 4
+        for (int step = kFreeSteps; step < 32; ++step) four_single(step, cuda::std::true_type{});
     }
     return alive ? pos : 0u;
 }

@@ -78,7 +78,7 @@ constexpr uint32_t kEncBytes = kEncCbBytes + kEncKpBytes;             // 8320, a
 constexpr uint32_t kOffShapeLut = kOffEncKp + kEncKpBytes;            // [n_shapes][256] u8
 constexpr uint32_t kMaxShapes = kMaxPatterns * kCodebooks;
 constexpr int kPairMinBits = 8, kPairMaxBits = 12;
-constexpr uint32_t kPairBudgetBytes = 64u << 10;
+constexpr uint32_t kPairBudgetBytes = 80u << 10;
 constexpr uint32_t kMaxDevBytes = kOffShapeLut + kMaxShapes * 256 + kPairBudgetBytes;
 // Both kinds of table are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.

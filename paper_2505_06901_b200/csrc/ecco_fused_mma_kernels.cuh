@@ -135,7 +135,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
-    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
     const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
     uint32_t stage;
     const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
@@ -151,8 +151,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
-    Block blk;
-    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
@@ -203,8 +202,9 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
                 for (int i = 0; i < 4; ++i) acc[mt][i] = 0.0f;
             cur_tile = tile;
         }
-        const Block cur = blk;
-        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        Block cur;                                         // fetched now, prefetched into L2 one unit earlier (see the scalar kernels)
+        ldg_block(cur, block_ptr(u));
+        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
         const __half* xk = d_x + static_cast<int>(u % kblocks) * kGroup;
         row_dot_mma(cur, tb, ws, stage, T, tile * 32 + lane < n_out,
                     [&](uint32_t (&v)[16]) { load_vfrag(v, xk, static_cast<size_t>(k), batch); }, acc);
@@ -223,7 +223,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
-    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
     const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
     uint32_t stage;
     const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
@@ -238,8 +238,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
-    Block blk;
-    if (u0 < u1) ldg_block(blk, block_ptr(u0));
+    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
@@ -248,8 +247,9 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
     for (int64_t u = u0; u < u1; ++u) {
         const int bh = static_cast<int>(u / tiles), t0 = static_cast<int>(u % tiles) * 32;
         if (bh != cur_bh) { load_vfrag(vfrag, d_q + static_cast<size_t>(bh) * q_per_kv * kGroup, kGroup, q_per_kv); cur_bh = bh; }
-        const Block cur = blk;
-        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        Block cur;
+        ldg_block(cur, block_ptr(u));
+        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
         row_dot_mma(cur, tb, ws, stage, T, t0 + lane < seq,
                     [&](uint32_t (&v)[16]) {

@@ -915,8 +915,6 @@ void plan_image(const ecco_meta& m, ImagePlan& p)
         }
     // widths: everyone starts at the minimum; then the upgrade that removes the most escapes per byte, while it fits
     uint32_t bytes = static_cast<uint32_t>(p.n_shapes) * (2u << kPairMinBits);
-    uint32_t kPairBudgetBytes = ecco::kPairBudgetBytes;
-    if (const char* env = std::getenv("ECCO_PAIR_BUDGET_KB")) kPairBudgetBytes = std::min<uint32_t>(kPairBudgetBytes, static_cast<uint32_t>(std::atoi(env)) << 10);
     if (bytes <= kPairBudgetBytes) {
         for (int i = 0; i < p.n_shapes; ++i) p.width[i] = kPairMinBits;
         for (;;) {

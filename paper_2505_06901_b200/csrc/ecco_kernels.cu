@@ -85,7 +85,7 @@ static bool make_out_map(CUtensorMap* map, void* d_out, uint64_t n_groups)
               CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kDecompressTmaWarps = 28;
+constexpr int kDecompressTmaWarps = 32;
 
 // every decoding kernel asks for all the shared memory of an SM and lays itself out on the device
 template <class K>

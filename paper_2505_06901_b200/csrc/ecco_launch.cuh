@@ -89,8 +89,8 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Warps per CTA the decoding kernels are launched with (their register budget); how many of them work is decided on
 // the device, from the size of the image's tables.
 constexpr int kDecompressWarps = 28;
-constexpr int fused_warps(int) { return 20; }
-constexpr int gemv_warp_warps(int) { return 20; }
+constexpr int fused_warps(int) { return 28; }
+constexpr int gemv_warp_warps(int) { return 28; }
 
 struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
 
