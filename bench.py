@@ -2,18 +2,23 @@
 """Benchmark of the Ecco decompression hot path on B200.
 
 One step = one pass of the whole hot path over the Llama-2-7B-shaped configuration:
-  1. ecco_decompress of the 7 compressed projection matrices of one decoder layer,
+  1. ecco_decompress of the 7 compressed projection matrices of one decoder layer (one batched call),
   2. ecco_gemv (fused decode + GEMV) over the same 7 matrices at batch 1,
   3. the same at batch 8,
-  4. ecco_attn_scores over the layer's compressed K cache [8][32][4096][128], one query per sequence.
+  4. ecco_attn_scores over the layer's compressed K cache [8][32][4096][128], one query per sequence,
+  5. ecco_attn_values (softmax . V) over the layer's compressed V cache.
 The headline `value` is the fp16 output rate of segment 1 (decompress output GB/s); the other
-segments are reported beside it (GEMV microseconds per layer, attention-score microseconds).
+segments are reported beside it (GEMV microseconds per layer, attention microseconds).  After the
+headline step a single-GPU run also times the long-context and the 70B-shaped configurations and
+reports them under `other_configs`.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-N > 1 (under torchrun): every rank runs the same step on its own copy of the workload (the blocks of
-a tensor are independent, so the path shards with no data-path collective: weak scaling); the time
-is the maximum over ranks of the device time, the value the sum of the ranks' bytes over that time.
+N > 1: one process per GPU.  Started under torchrun the ranks are taken from its environment; started
+directly, the script re-launches itself under torch.distributed.run with N processes on this node.
+Every rank runs the same step on its own copy of the workload (the blocks of a tensor are independent,
+so the path shards with no data-path collective: weak scaling); the time is the maximum over ranks of
+the device time, the value the sum of the ranks' bytes over that time.
 """
 from __future__ import annotations
 
@@ -35,7 +40,7 @@ G, BLOCK = 128, 64
 METRIC, UNIT = "decompress_output_GBps", "GB/s"
 
 
-def parse_args():
+def parse_args(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
@@ -51,7 +56,27 @@ def parse_args():
                     help="decompress segment: one ecco_decompress_batch call over the step's tensors (default) or one ecco_decompress per tensor")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    return ap.parse_args()
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the cfg5 / cfg4 measurements that follow the headline step")
+    return ap.parse_args(argv)
+
+
+def relaunch_command(args, argv, environ):
+    """--gpus N > 1 without a torchrun environment: the command that starts N ranks of this script on this node
+    (None when no re-launch is needed).  A torchrun environment whose world size contradicts --gpus is an error."""
+    world = environ.get("WORLD_SIZE")
+    if world is not None:
+        if args.gpus != int(world) and args.gpus != 1:
+            raise SystemExit(f"--gpus {args.gpus} contradicts WORLD_SIZE={world}")
+        return None
+    if args.gpus <= 1:
+        return None
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
 
 
 def cores() -> int:
@@ -164,8 +189,9 @@ def run_reference(args):
     }))
 
 
-def cpu_baseline(layer, c: int):
-    """The oracle's decoder on a bounded sample of the benchmark's own blocks (about 15 s of CPU work)."""
+def cpu_baseline(layer, c: int, kv_tensor=None):
+    """The oracle's decoder on a bounded sample of the benchmark's own blocks (about 15 s of CPU work), and its
+    decode + dot product for one GEMV sample and one attention-score sample."""
     from oracle import ecco_oracle as eo
 
     t = layer[0]
@@ -187,9 +213,43 @@ def cpu_baseline(layer, c: int):
     t0 = time.perf_counter()
     eo.decode_threads(om, t.blocks[:n], c)
     dt = time.perf_counter() - t0
-    return {"value": n * G * 2 / dt / 1e9, "unit": UNIT, "cores": c, "kind": "oracle",
-            "sample": f"first {n} groups of tensor '{t.name}' {tuple(t.shape)}, one pass on {c} threads",
-            "groups_per_s": n / dt, "single_core_groups_per_s": rate}
+    out = {"value": n * G * 2 / dt / 1e9, "unit": UNIT, "cores": c, "kind": "oracle",
+           "sample": f"first {n} groups of tensor '{t.name}' {tuple(t.shape)}, one pass on {c} threads",
+           "groups_per_s": n / dt, "single_core_groups_per_s": rate}
+    # the fused calls: the oracle's decode + fp64 dot products on one core, over the first rows of the same tensor
+    # (and the first tokens of the K cache), a few seconds each
+    from paper_2505_06901_b200 import synth
+
+    fused = {}
+    if len(t.shape) == 2:
+        n_out, k = t.shape
+        rows = int(max(32, min(n_out, rate * 3 // (k // G))))
+        x = synth.activations(1, k, 11)
+        t0 = time.perf_counter()
+        eo.gemv(om, t.blocks[: rows * (k // G)], rows, k, x, 1)
+        dt = time.perf_counter() - t0
+        fused["ecco_gemv batch 1"] = {"us_per_layer_equivalent": None, "weights_per_s": rows * k / dt, "cores": 1,
+                                      "sample": f"first {rows} rows of '{t.name}' {tuple(t.shape)}"}
+    if kv_tensor is not None:
+        kb, kh, kseq, _ = kv_tensor.shape
+        S2, e2, pat2, cb2, kp2 = kv_tensor.meta.tables()
+        km = eo.Meta()
+        km.S, km.H, km.e = S2, 4, e2
+        for k_ in range(S2):
+            km.kp_len[k_] = int(kp2[k_])
+            for j in range(15):
+                km.pattern[k_][j] = int(pat2.view(np.uint16)[k_, j])
+            for h in range(4):
+                for s_ in range(16):
+                    km.cb_len[k_][h][s_] = int(cb2[k_, h, s_])
+        toks = int(max(256, min(kseq, rate * 3)))
+        q = synth.queries(1, 1, 13)
+        t0 = time.perf_counter()
+        eo.attn_scores(km, kv_tensor.blocks[:toks], 1, 1, toks, 1, q, 128 ** -0.5)
+        dt = time.perf_counter() - t0
+        fused["ecco_attn_scores"] = {"tokens_per_s": toks / dt, "cores": 1, "sample": f"first {toks} tokens of head 0 of the K cache"}
+    out["fused"] = fused
+    return out
 
 
 # ------------------------------------------------------------------------------------------------
@@ -237,7 +297,11 @@ def build_workload(name, workloads):
     return workloads.config2(), (kt, vt), 1, False, ["decompress", "gemv1", "gemv8", "attn", "attnv"]
 
 
-def run_ours(args):
+def run_ours(args, workload=None, extras=True):
+    """-> the JSON line of one workload as a dict (None on ranks other than 0).  extras = False skips the end-to-end
+    leg, the per-tensor-call figure and the CPU baseline (used for the configurations after the headline step)."""
+    import gc
+
     import torch
 
     from paper_2505_06901_b200 import binding as B
@@ -251,11 +315,13 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
 
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if not dist.is_initialized():
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.lib()
 
     # ---- workload (the same seeded tensors on every rank)
-    wname = ("small5" if args.workload == "cfg5" else "small") if args.small else args.workload
+    workload = workload or args.workload
+    wname = ("small5" if workload == "cfg5" else "small") if args.small else workload
     weights, kvt, q_per_kv, decompress_kv, default_segs = build_workload(wname, workloads)
     kt, vt = kvt if kvt is not None else (None, None)
     segs = [s for s in args.only.split(",") if s] or default_segs
@@ -365,7 +431,7 @@ def run_ours(args):
 
     # ---- end to end through the C ABI with host buffers: H2D of the blocks, decompress, D2H of the fp16
     e2e = None
-    if "decompress" in segs and dec:
+    if "decompress" in segs and dec and extras:
         h_in = [torch.from_numpy(d["t"].blocks).pin_memory() for d in dec]
         h_out = [torch.empty(d["n"] * G, dtype=torch.float16).pin_memory() for d in dec]
 
@@ -442,13 +508,13 @@ def run_ours(args):
             del blocks, out
 
     if rank != 0:
-        if dist is not None:
+        if dist is not None and extras:
             dist.destroy_process_group()
-        return
+        return None
 
     # the same tensors through one ecco_decompress call each, for the record
     single_us = None
-    if "decompress" in segs and dec and args.decompress_calls == "batch":
+    if "decompress" in segs and dec and args.decompress_calls == "batch" and extras:
         for _ in range(3):
             seg_decompress_single()
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -474,23 +540,25 @@ def run_ours(args):
         with open(tp) as f:
             ncu_consts = json.load(f)
         traffic = ncu_consts["decompress_dram"]["dram_bytes_per_group"] * groups / n_launch
-    # What really limits the decoder are the SM's issue slots and its load/store pipe.  Their ceilings come from the
-    # unit counts and the clock (4 warp instructions and 1 wavefront per clock per SM); the per-symbol costs are ncu
-    # counters of this kernel (profiles/), the symbol rate is this run's.
+    # What really limits the decoder are the SM's issue slots and its load/store pipe.  Their ceilings were measured
+    # on this GPU with small probe kernels (warp instructions per clock per SM: 4.0 for adds and FFMA, 2.0 for the
+    # logic / shift / permute / multiply-add instructions the decoder is made of; one shared-memory wavefront per
+    # clock); the per-symbol costs are ncu counters of this kernel, the symbol rate is this run's.
     sm_limits = None
     if "decompress_sm" in ncu_consts and dec_ms > 0:
-        c = ncu_consts["decompress_sm"]
+        c, m = ncu_consts["decompress_sm"], ncu_consts["measured_sm_rates"]
         props = torch.cuda.get_device_properties(local)
         sms, ghz = props.multi_processor_count, ((clocks or {}).get("sm_mhz") or 0) / 1e3
         if ghz > 0:
             warp_symbols_per_s = groups * (G / 32) * args.steps / (dec_ms / 1e3)
             sm_limits = {
-                "issue": {"bound": "alu", "unit": "G warp-instr/s", "peak": sms * 4 * ghz,
+                "issue": {"bound": "alu", "unit": "G warp-instr/s", "peak": sms * m["issue_warp_instr_per_clk_sm"] * ghz,
                           "achieved": warp_symbols_per_s * c["warp_instructions_per_warp_symbol"] / 1e9},
-                "lsu": {"bound": "lsu", "unit": "G wavefronts/s", "peak": sms * 1 * ghz,
+                "lsu": {"bound": "lsu", "unit": "G wavefronts/s", "peak": sms * m["lsu_wavefronts_per_clk_sm"] * ghz,
                         "achieved": warp_symbols_per_s * c["lsu_wavefronts_per_warp_symbol"] / 1e9},
                 "per_warp_symbol": {"instructions": c["warp_instructions_per_warp_symbol"], "wavefronts": c["lsu_wavefronts_per_warp_symbol"]},
-                "source": "paper_2505_06901_b200/ncu_constants.json (from profiles/ecco_decompress_tma_kernel_cfg5_dram.md); peaks = SMs x units x sampled SM clock",
+                "measured_rates": m,
+                "source": "per-symbol costs: ncu capture of this kernel (paper_2505_06901_b200/ncu_constants.json); peaks = SMs x measured rate x sampled SM clock",
             }
             for k in ("issue", "lsu"):
                 sm_limits[k]["frac"] = sm_limits[k]["achieved"] / sm_limits[k]["peak"]
@@ -545,11 +613,27 @@ def run_ours(args):
         line["note"] = "--only without decompress: the segment of the headline metric was not timed; see segments_us_per_step"
     if sweep is not None:
         line["stream_sweep"] = sweep
-    if world == 1 and not args.no_cpu_baseline and dec:
-        line["cpu_baseline"] = cpu_baseline([d["t"] for d in dec], cores())
-    print(json.dumps(line))
-    if dist is not None:
+    if world == 1 and not args.no_cpu_baseline and dec and extras:
+        line["cpu_baseline"] = cpu_baseline([d["t"] for d in dec], cores(), kt)
+    if dist is not None and extras:
         dist.destroy_process_group()
+    del mats, dec, kv, dec_items
+    gc.collect()
+    torch.cuda.empty_cache()
+    return line
+
+
+def other_config_summary(line):
+    """What the default run keeps of a cfg4 / cfg5 measurement."""
+    if line is None:
+        return None
+    keep = {"workload": line["config"]["workload"], "steps": line["steps"], "decompress_output_GBps": line["value"],
+            "segments_us_per_step": {k: v for k, v in line["segments_us_per_step"].items() if v > 5.0},
+            "kernels": line["kernels"], "clocks": line["clocks"],
+            "roofline_frac": line["roofline"]["frac"] if line.get("roofline") else None}
+    if "stream_sweep" in line:
+        keep["stream_sweep"] = line["stream_sweep"]
+    return keep
 
 
 def run_var(args):
@@ -735,8 +819,13 @@ def run_act2x(args):
         dist.destroy_process_group()
 
 
-if __name__ == "__main__":
-    a = parse_args()
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
+    a = parse_args(argv)
+    cmd = relaunch_command(a, argv, os.environ)
+    if cmd is not None:                                    # --gpus N without torchrun: start the N ranks here
+        env = dict(os.environ, NCCL_DEBUG=os.environ.get("NCCL_DEBUG", "WARN"))
+        raise SystemExit(subprocess.call(cmd, env=env))
     if a.impl == "reference":
         run_reference(a)
     elif a.workload == "act2x":
@@ -744,4 +833,17 @@ if __name__ == "__main__":
     elif a.workload == "var":
         run_var(a)
     else:
-        run_ours(a)
+        world = int(os.environ.get("WORLD_SIZE", "1"))
+        others = a.workload == "cfg2" and not a.small and not a.only and not a.no_other_configs and world == 1
+        line = run_ours(a)
+        if line is not None and others:
+            # the long-context and the 70B-shaped configurations, outside the headline step (fewer steps, no end-to-end leg)
+            short = argparse.Namespace(**vars(a))
+            short.steps, short.warmup = max(3, min(a.steps, 10)), 3
+            line["other_configs"] = {w: other_config_summary(run_ours(short, workload=w, extras=False)) for w in ("cfg5", "cfg4")}
+        if line is not None:
+            print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

@@ -49,6 +49,29 @@ def test_single_process_is_identity():
     assert distutil.aggregate_throughput(10.0, 2.0, 1) == 5.0
 
 
+def test_gpus_flag_relaunches_under_torchrun_only_when_needed():
+    """`bench.py --gpus N` started directly must start N ranks itself; under torchrun it must not, and a world size
+    that contradicts the flag is an error."""
+    import importlib.util
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(root, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    argv = ["--gpus", "4", "--steps", "7", "--warmup", "3"]
+    cmd = bench.relaunch_command(bench.parse_args(argv), argv, {})
+    assert cmd[:3] == [sys.executable, "-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-len(argv) - 1].endswith("bench.py") and cmd[-len(argv):] == argv
+    assert 1024 < int(cmd[cmd.index("--master-port") + 1]) < 65536
+    assert bench.relaunch_command(bench.parse_args(argv), argv, {"WORLD_SIZE": "4", "RANK": "1"}) is None
+    assert bench.relaunch_command(bench.parse_args([]), [], {}) is None
+    assert bench.relaunch_command(bench.parse_args(["--gpus", "1"]), ["--gpus", "1"], {}) is None
+    with pytest.raises(SystemExit):
+        bench.relaunch_command(bench.parse_args(argv), argv, {"WORLD_SIZE": "2"})
+
+
 def test_reference_arm_prints_one_contract_line():
     """`bench.py --impl reference` (the oracle, CPU only) prints exactly one JSON line with the contract's keys."""
     import json
