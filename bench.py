@@ -600,7 +600,7 @@ def run_ours(args, workload=None, extras=True):
         "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
                      "algorithmic_bytes_per_launch": alg_bytes_per_launch, "avg_launch_us": avg_launch_s * 1e6,
-                     "note": "kernel of the headline metric; limited by the SM load/store pipe, see kernels[] and profiles/"},
+                     "note": "kernel of the headline metric; limited by the SM (issue slots and load/store pipe), not by HBM: see kernels[] and sm_limits"},
         "kernels": kernels,
     }
     if sm_limits is not None:

@@ -160,7 +160,9 @@ int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_
  * of ECCO_STATIC_WORKSPACE_BYTES inside the library's device image (every GPU that loads the
  * library carries it until the process exits) instead of a caller buffer.  The call allocates
  * nothing.  A shape whose plan needs more scratch than that is refused with ECCO_ERR_WORKSPACE
- * before anything is launched (for scale: batch 8 on an 11008 x 4096 matrix needs about 3.3 MB).
+ * before anything is launched.  For scale, on a 148-SM part: batch 8 on an 11008 x 4096 matrix needs 3.99 MB, which
+ * fits; batch 1 or 2 on the same matrix 0.6 / 1.1 MB; a matrix with more than about 12 000 output rows at batch 3..8
+ * (for instance 28672 x 8192) does not fit and is refused.
  * The first call on each device looks up the array's device address (with that device current);
  * make that first call outside any stream capture.  All calls on a device share the one array:
  * it still holds the previous call's values when the next call starts (each call clears the part
@@ -245,6 +247,11 @@ int ecco_last_cuda_error(void);        /* cudaError_t of the last ECCO_ERR_CUDA 
 int ecco_device_status(void);
 /* Number of kernels the library has launched in this process (diagnostic counter). */
 uint64_t ecco_kernel_launch_count(void);
+/* Test aid for the give-up path of the bounded device-side wait (Sec. 4.2's "loaded once" staging waits on a
+ * barrier that a bulk copy completes): launches one small CTA on `stream` that arms such a barrier for bytes
+ * no copy will deliver -- nothing is in flight and nothing can hang --, polls it a few hundred times, gives up and
+ * returns normally.  Afterwards ecco_device_status() reports ECCO_ERR_DEVICE_TIMEOUT once. */
+int ecco_test_wait_timeout(void* stream);
 
 #ifdef __cplusplus
 }

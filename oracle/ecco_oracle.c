@@ -24,8 +24,7 @@
  *   Consumers: decode-phase GEMV and attention scores QK^T/sqrt(d) (Sec. 2.1) in fp64.
  *
  * Where the paper is silent (bit order inside the block, FP8 flavour, tie rules, pad cap)
- * the readings are the ones listed in the repository's design notes; each is marked
- * "reading:" below.
+ * a reading had to be chosen; each is marked "reading:" where it is used below.
  *
  * Pins (tests/test_oracle_*.py): FP16/FP8 conversion against numpy / torch exhaustively;
  * exact dequantisation; DP k-means against brute force; Kraft equality, prefix-freeness,

@@ -36,7 +36,7 @@ EXPORTS = [
     "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
     "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress",
     "ecco_var_stream_bytes_bound", "ecco_var_index_bytes", "ecco_var_encode_host", "ecco_var_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
-    "ecco_kernel_launch_count",
+    "ecco_kernel_launch_count", "ecco_test_wait_timeout",
 ]
 
 
@@ -114,6 +114,7 @@ def lib():
         L.ecco_last_cuda_error.restype = C.c_int
         L.ecco_device_status.restype = C.c_int
         L.ecco_kernel_launch_count.restype = u64
+        L.ecco_test_wait_timeout.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -335,3 +336,8 @@ def ecco_device_status() -> int:
 
 def ecco_kernel_launch_count() -> int:
     return int(lib().ecco_kernel_launch_count())
+
+
+def ecco_test_wait_timeout(stream=None) -> None:
+    """Test aid: one small kernel whose bounded wait runs out (see include/ecco.h)."""
+    _check(lib().ecco_test_wait_timeout(_stream(stream)), "ecco_test_wait_timeout")

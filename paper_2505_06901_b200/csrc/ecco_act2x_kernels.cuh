@@ -23,7 +23,7 @@ ecco_act_decompress_kernel(const uint4* __restrict__ d_blocks, uint64_t n_chunks
     for (uint64_t r = 0, c = static_cast<uint64_t>(blockIdx.x) * blockDim.x + threadIdx.x; r < rounds; ++r, c += stride) {
         const bool ok = c < n_chunks;                       // whole warps stay in the loop for the shuffles
         uint4 b = make_uint4(0, 0, 0, 0);
-        if (ok) asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(d_blocks + c));
+        if (ok) asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(b.x), "=r"(b.y), "=r"(b.z), "=r"(b.w) : "l"(d_blocks + c));
         const uint32_t bits16 = top_bits(b.x) | (top_bits(b.y) << 4) | (top_bits(b.z) << 8) | (top_bits(b.w) << 12);
         const uint32_t lane = threadIdx.x & 31u;
         const uint32_t scale_bits = __shfl_sync(0xffffffffu, bits16, lane & ~3u);          // chunk 0 of the group
@@ -61,7 +61,7 @@ ecco_act_compress_kernel(const uint4* __restrict__ d_x, uint64_t n_chunks, uint4
         const bool ok = c < n_chunks;
         uint32_t h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         if (ok)
-            asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+            asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                          : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3]), "=r"(h[4]), "=r"(h[5]), "=r"(h[6]), "=r"(h[7])
                          : "l"(d_x + c * 2));
         float x[16];

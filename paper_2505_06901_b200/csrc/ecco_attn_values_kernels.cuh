@@ -18,7 +18,7 @@ namespace {
 // The result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
-ecco_softmax_stats_kernel(const float* __restrict__ d_scores, int rows, int seq, float2* __restrict__ d_stats)
+ecco_softmax_stats_kernel(const float* d_scores, int rows, int seq, float2* d_stats)
 {
     const int row = static_cast<int>(blockIdx.x) * 8 + static_cast<int>(threadIdx.x >> 5), lane = static_cast<int>(threadIdx.x & 31u);
     dependency_wait();                                     // the scores may come from the previous kernel of the stream
@@ -26,11 +26,11 @@ ecco_softmax_stats_kernel(const float* __restrict__ d_scores, int rows, int seq,
     if (row >= rows) return;
     const float* s = d_scores + static_cast<size_t>(row) * seq;
     float mx = -INFINITY;
-    for (int t = lane; t < seq; t += 32) mx = fmaxf(mx, s[t]);
+    for (int t = lane; t < seq; t += 32) mx = fmaxf(mx, __ldcg(s + t));    // the scores may come from the previous kernel: coherent loads
 #pragma unroll
     for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     float sum = 0.0f;
-    for (int t = lane; t < seq; t += 32) sum += expf(s[t] - mx);
+    for (int t = lane; t < seq; t += 32) sum += expf(__ldcg(s + t) - mx);
 #pragma unroll
     for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
     if (lane == 0) d_stats[row] = make_float2(mx, 1.0f / sum);
@@ -56,7 +56,7 @@ constexpr float kProbScale = 32768.0f, kProbUnscale = 1.0f / 32768.0f;      // p
 template <int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_vblocks, int heads, int seq,
-                        int q_per_kv, const float* __restrict__ d_scores, const float2* __restrict__ d_stats,
+                        int q_per_kv, const float* d_scores, const float2* d_stats,
                         float* __restrict__ d_out, float* __restrict__ d_partial, unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -164,7 +164,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         const int t = tile_base + static_cast<int>(lane);
         if (bh != cur_bh) {
             if (cur_bh >= 0) { flush(cur_bh); clear_acc(); }
-            if (tid < 8) stats_s[tid] = tid < q_per_kv ? d_stats[static_cast<size_t>(bh) * q_per_kv + tid] : make_float2(0.0f, 0.0f);
+            if (tid < 8) stats_s[tid] = tid < q_per_kv ? __ldcg(d_stats + static_cast<size_t>(bh) * q_per_kv + tid) : make_float2(0.0f, 0.0f);
             __syncthreads();
             cur_bh = bh;
         }
@@ -184,8 +184,8 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             for (int j = 0; j < 4; ++j) {
                 const int tk = tile_base + static_cast<int>(lane & 3u) * 2 + 8 * j;
                 float p0 = 0.0f, p1 = 0.0f;
-                if (r < q_per_kv && tk < seq) p0 = __expf(srow[tk] - st.x) * to_p;
-                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(srow[tk + 1] - st.x) * to_p;
+                if (r < q_per_kv && tk < seq) p0 = __expf(__ldcg(srow + tk) - st.x) * to_p;
+                if (r < q_per_kv && tk + 1 < seq) p1 = __expf(__ldcg(srow + tk + 1) - st.x) * to_p;
                 const __half h0 = __float2half_rn(p0), h1 = __float2half_rn(p1);
                 const __half l0 = __float2half_rn(p0 - __half2float(h0)), l1 = __float2half_rn(p1 - __half2float(h1));
                 p_hi[j] = static_cast<uint32_t>(__half_as_ushort(h0)) | (static_cast<uint32_t>(__half_as_ushort(h1)) << 16);

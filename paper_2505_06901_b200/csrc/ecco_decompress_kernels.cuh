@@ -286,7 +286,7 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     };
     auto load_chunk = [&](uint64_t c) {
         uint4 v = make_uint4(0, 0, 0, 0);
-        if (c < stream_chunks) asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d_stream + c));
+        if (c < stream_chunks) asm volatile("ld.global.cg.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(d_stream + c));
         return v;
     };
     Span cur = {0, 0, 0, 0};

@@ -114,14 +114,16 @@ __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
     return v;
 }
 __device__ __forceinline__ void sts_u32(uint32_t addr, uint32_t v) { asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory"); }
-// one 64-byte block = two 32-byte loads per lane: every load instruction asks for whole sectors
+// one 64-byte block = two 32-byte loads per lane: every load instruction asks for whole sectors.  Plain (coherent)
+// loads that bypass L1: under the overlapped launches the blocks may have been written by the previous kernel of the
+// stream (the online compressor), and the non-coherent path is only for data that nobody writes while a kernel lives.
 struct Block { uint32_t w[16]; };
 __device__ __forceinline__ void ldg_block(Block& b, const uint8_t* p)
 {
-    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+    asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(b.w[0]), "=r"(b.w[1]), "=r"(b.w[2]), "=r"(b.w[3]), "=r"(b.w[4]), "=r"(b.w[5]), "=r"(b.w[6]), "=r"(b.w[7])
                  : "l"(p));
-    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+    asm volatile("ld.global.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                  : "=r"(b.w[8]), "=r"(b.w[9]), "=r"(b.w[10]), "=r"(b.w[11]), "=r"(b.w[12]), "=r"(b.w[13]), "=r"(b.w[14]), "=r"(b.w[15])
                  : "l"(p + 32));
 }
@@ -221,18 +223,20 @@ __device__ __forceinline__ void issue_tables(const Tables& tb, const uint8_t* d_
         if (tb.pair_bytes) bulk_g2s(tb.pair, d_meta + __ldg(&hd->off_pair), tb.pair_bytes, bar);
     }
 }
-__device__ __forceinline__ bool wait_tables(const Tables& tb, uint32_t parity = 0)
+// Bounded wait of the whole CTA on a barrier word: at most 2 * limit polls per thread (the second round is a last
+// chance for a copy in flight), then the CTA gives up together, records ECCO_ERR_DEVICE_TIMEOUT and returns false.
+__device__ __forceinline__ bool bounded_wait(uint32_t bar, uint32_t parity, int limit)
 {
-    const uint32_t bar = tb.base;
     __syncthreads();                             // the barrier word is initialised
     bool done = false;
-    for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, parity);
-    if (!done)                                   // second, bounded chance for the copy in flight
-        for (int i = 0; i < kWaitLimit && !done; ++i) done = mbar_try_wait(bar, parity);
+    for (int i = 0; i < limit && !done; ++i) done = mbar_try_wait(bar, parity);
+    if (!done)
+        for (int i = 0; i < limit && !done; ++i) done = mbar_try_wait(bar, parity);
     const bool all = __syncthreads_and(done);
     if (!all && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_DEVICE_TIMEOUT);
     return all;
 }
+__device__ __forceinline__ bool wait_tables(const Tables& tb, uint32_t parity = 0) { return bounded_wait(tb.base, parity, kWaitLimit); }
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may become resident
 // while the previous kernel in the stream is still draining.  dependency_wait() returns once that kernel has
 // completed and its writes are visible (at once if there is no such overlap); every kernel executes it before

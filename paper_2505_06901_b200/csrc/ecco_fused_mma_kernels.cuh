@@ -117,7 +117,7 @@ __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* 
     const uint2* p = reinterpret_cast<const uint2*>(base + static_cast<size_t>(min(col, n_cols - 1)) * col_stride) + (lane & 3);
 #pragma unroll
     for (int c = 0; c < 8; ++c) {
-        const uint2 v = col < n_cols ? __ldg(p + c * 4) : make_uint2(0u, 0u);     // k = 16c + 4 (lane%4) .. + 3
+        const uint2 v = col < n_cols ? __ldcg(p + c * 4) : make_uint2(0u, 0u);     // k = 16c + 4 (lane%4) .. + 3
         vfrag[2 * c] = v.x;                                // tile columns 2q, 2q+1
         vfrag[2 * c + 1] = v.y;                            // tile columns 2q+8, 2q+9
     }
@@ -128,7 +128,7 @@ __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* 
 template <int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                     const __half* __restrict__ d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+                     const __half* d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
                      unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -217,7 +217,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
 template <int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
-                            int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
+                            int q_per_kv, const __half* d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);

@@ -161,7 +161,7 @@ __device__ __forceinline__ WarpSmem fused_warp_smem(const Tables& tb, uint32_t n
 template <int kV, int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                      const __half* __restrict__ d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
+                      const __half* d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
                       unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -243,7 +243,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         const int kb = static_cast<int>(u % kblocks);
 #pragma unroll
         for (int b = 0; b < kV; ++b)
-            xraw[b] = __ldg(reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4));
+            xraw[b] = __ldcg(reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4));
     };
     if (u0 < u1) load_x(u0);
     int cur_tile = static_cast<int>(u0 / kblocks);
@@ -283,7 +283,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
 template <int kV, int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
-                        int q_per_kv, const __half* __restrict__ d_q, float scale, float* __restrict__ d_scores)
+                        int q_per_kv, const __half* d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     dependency_wait();                                     // the previous kernel of the stream has completed
@@ -318,7 +318,7 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
             for (int i = tid; i < kGroup * kV; i += static_cast<int>(blockDim.x)) {
                 const int r = i % kV, d = i / kV;
-                xs[i] = (r < q_per_kv) ? scale * __half2float(d_q[(static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d]) : 0.0f;
+                xs[i] = (r < q_per_kv) ? scale * __half2float(__ldcg(d_q + (static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d)) : 0.0f;
             }
             __syncthreads();
             cur_bh = bh;

@@ -54,6 +54,30 @@ extern "C" int ecco_device_status(void)
     return st;
 }
 
+// Diagnostics: the give-up path of the bounded wait, exercised without anything that could hang.  The kernel arms a
+// barrier with a byte count that no copy will ever deliver (nothing is in flight, so the CTA may exit at any time),
+// polls it a few hundred times, gives up, records the time-out and returns normally.
+namespace {
+__global__ void ecco_wait_timeout_probe_kernel()
+{
+    __shared__ __align__(8) uint64_t bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        mbar_init(b, 1);
+        mbar_expect_tx(b, 64);
+    }
+    (void)bounded_wait(b, 0, 256);
+}
+}  // namespace
+extern "C" int ecco_test_wait_timeout(void* stream)
+{
+    DeviceInfo di;
+    int rc = device_info(&di);
+    if (rc) return rc;
+    ecco_wait_timeout_probe_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>();
+    return check_launch();
+}
+
 // cuTensorMapEncodeTiled through the runtime's driver entry point query (no link against libcuda)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,

@@ -49,7 +49,7 @@ ecco_kv_compress_kernel(const uint8_t* __restrict__ d_meta, const __half* __rest
     auto fp8 = [&](float v) { return static_cast<uint32_t>(__nv_cvt_float_to_fp8(v * invT, __NV_SATFINITE, __NV_E4M3)); };
 
     for (uint64_t g = static_cast<uint64_t>(blockIdx.x) * kKvWarps + warp; g < n_groups; g += static_cast<uint64_t>(gridDim.x) * kKvWarps) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(d_x + g * kGroup) + lane);
+        const uint2 raw = __ldcg(reinterpret_cast<const uint2*>(d_x + g * kGroup) + lane);
         const uint32_t h16[4] = {raw.x & 0xffffu, raw.x >> 16, raw.y & 0xffffu, raw.y >> 16};
         float x[4];
         uint32_t key[4];                                   // |x| then low index first

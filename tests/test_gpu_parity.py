@@ -279,6 +279,17 @@ def test_decompress_rejects_bad_arguments_on_device(B, cfg1_small):
     assert B.ecco_device_status() == 0
 
 
+def test_bounded_wait_gives_up_and_reports(B, eo, cfg1_small):
+    """The device-side wait on the table copy is bounded: when it runs out the kernel records
+    ECCO_ERR_DEVICE_TIMEOUT and returns, ecco_device_status reports it once, and the context stays usable."""
+    assert B.ecco_device_status() == 0
+    B.ecco_test_wait_timeout()
+    assert B.ecco_device_status() == B.ERR_DEVICE_TIMEOUT
+    assert B.ecco_device_status() == 0                      # reading clears it
+    lm = lib_meta_from_oracle(B, cfg1_small["meta"])
+    assert_bit_exact(gpu_decompress(B, lm, cfg1_small["blocks"][:100]), eo.decode(cfg1_small["meta"], cfg1_small["blocks"][:100]))
+
+
 # ------------------------------------------------------------------ fused GEMV
 @pytest.mark.parametrize("n_out,k,batch", [(256, 1024, 1), (256, 1024, 3), (256, 1024, 8), (100, 1024, 2), (513, 512, 5),
                                            (2048, 128, 1), (64, 4096, 4), (1, 128, 1)])

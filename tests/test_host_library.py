@@ -346,6 +346,49 @@ def test_device_image_for_every_code_shape(binding, eo):
             assert end == (info.end_bit if info.n_fit == 128 else 0)
 
 
+def _oracle_encode_threads(eo, om, x, select):
+    """eo.encode over disjoint ranges of groups from one Python thread per core (ctypes drops the GIL)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    g = x.reshape(-1, 128)
+    n = g.shape[0]
+    threads = max(1, min(len(os.sched_getaffinity(0)), n // 256))
+    bounds = [n * i // threads for i in range(threads + 1)]
+    out = np.zeros((n, 64), dtype=np.uint8)
+
+    def work(i):
+        lo, hi = bounds[i], bounds[i + 1]
+        if hi > lo:
+            out[lo:hi] = eo.encode(om, g[lo:hi], select)[0]
+
+    with ThreadPoolExecutor(threads) as ex:
+        list(ex.map(work, range(threads)))
+    return out
+
+
+def test_host_encoder_matches_oracle_on_samples_of_the_large_configurations(binding, eo, synth):
+    """65 536 groups with the shapes, seeds and distributions of each larger configuration (the first rows of the
+    7B- and 70B-shaped matrices, the first tokens of the two KV caches), encoded with the library's own calibrated
+    metadata: the threaded host encoder and the plain oracle must write the same bytes."""
+    from paper_2505_06901_b200 import workloads as W
+
+    n = 1 << 16
+    cases = [("cfg2 gate", W.calibrate_weights(2, 0.02, True), synth.weight_matrix(n * 128 // 4096, 4096, 1002 * 16 + 4), binding.SELECT_MSE, 0),
+             ("cfg2 down", W.calibrate_weights(2, 0.02, True), synth.weight_matrix(n * 128 // 11008 // 1 + 1, 11008, 1002 * 16 + 6)[:762], binding.SELECT_MSE, 0),
+             ("cfg4 gate", W.calibrate_weights(4, 0.01, False), synth.weight_matrix(n * 128 // 8192, 8192, 1004 * 16, sigma=0.01, row_scale=False), binding.SELECT_MSE, 0),
+             ("cfg3 K", W.calibrate_kv(3, 32), synth.kv_cache(1, 32, n // 32, 1003 * 16, 3003), binding.SELECT_MINMAX, binding.KEEP_EXPONENT),
+             ("cfg5 K", W.calibrate_kv(5, 8), synth.kv_cache(1, 8, n // 8, 1005 * 16, 3005), binding.SELECT_MINMAX, binding.KEEP_EXPONENT)]
+    for name, base, x, select, keep in cases:
+        S, e, pat, cb, kp = base.tables()
+        lm = binding.ecco_meta_create(S, e, pat, cb, kp)
+        blocks, st = binding.ecco_encode_host(lm, x, select | keep)
+        om = oracle_meta_from_lib(eo, lm)                   # carries the exponent the library fitted (weights) or kept (KV)
+        want = _oracle_encode_threads(eo, om, x, select)
+        bad = np.nonzero((blocks != want).any(axis=1))[0]
+        assert bad.size == 0, (name, bad.size, bad[:5])
+        assert blocks.shape[0] >= 60000 and st.n_groups == blocks.shape[0]
+
+
 def test_variable_length_host_encoder_matches_oracle(binding, eo, cfg1_small, kv_small):
     for fx, key, flags in ((cfg1_small, "w", binding.SELECT_MSE), (kv_small, "k", binding.SELECT_MINMAX | binding.KEEP_EXPONENT)):
         ometa, x = fx["meta"], fx[key]

@@ -44,6 +44,15 @@ def test_roundtrip_bounds_and_field_layout(eo, synth):
     # minimum maps to q = -64, order is preserved
     assert np.all(q[np.arange(x.shape[0]), xf.argmin(1)][scale > 0] == -64)
     assert np.all(np.diff(q[5]) >= 0)
+    # quantisation, recomputed exactly: q = rint((x - zero) * (1 / scale)) in fp32 (the compressor's multiply-and-round
+    # circuit, Sec. 4.3), round half to even, clamped to the 7-bit range -- truncation or round-half-up would fail here
+    x32, s32, z32 = x.astype(np.float32), scale.astype(np.float32)[:, None], zero.astype(np.float32)[:, None]
+    live = (scale > 0)[:, None]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        inv = (np.float32(1.0) / s32).astype(np.float32)
+        want_q = np.clip(np.rint(((x32 - z32).astype(np.float32) * inv).astype(np.float32)), -64, 63)
+    want_q = np.where(live, want_q, 0).astype(np.int32)
+    assert np.array_equal(q, want_q)
     # dequantisation = one fused multiply-add in fp32, one rounding to fp16
     want = (q.astype(np.float64) * scale[:, None] + zero[:, None]).astype(np.float32).astype(np.float16)
     assert np.array_equal(out.astype(np.float16).view(np.uint16), want.view(np.uint16))
