@@ -2,19 +2,13 @@
 // Part of the one translation unit ecco_kernels.cu; included from there only.
 #pragma once
 
-#ifndef ECCO_FUSED_PAIRS
-#define ECCO_FUSED_PAIRS 0
-#endif
 namespace {
-constexpr bool kFusedPairs = ECCO_FUSED_PAIRS != 0;
-#ifndef ECCO_FUSED_HALFTAB
-#define ECCO_FUSED_HALFTAB 0
-#endif
-#ifndef ECCO_FUSED_LOCALRANKS
-#define ECCO_FUSED_LOCALRANKS 0
-#endif
-constexpr TabKind kFusedTab = ECCO_FUSED_HALFTAB ? kTabHalf : kTabFloat;
-__device__ __forceinline__ float fused_value(uint32_t v) { return ECCO_FUSED_HALFTAB ? __half2float(__ushort_as_half(static_cast<unsigned short>(v))) : __uint_as_float(v); }
+
+// The fused kernels decode one symbol per lookup (shape tables only) and leave the pair tables out of shared memory:
+// measured on the 7B-shaped matrices and the cfg-3 K cache, the room the pair tables take (fewer resident warps) costs
+// them as much as two-symbol lookups save, and on KV caches, whose codebooks spread over three dozen code shapes,
+// escapes make the pair path the slower one.
+constexpr bool kFusedPairs = false;
 
 // ---------------------------------------------------------------------------------------------
 // K2/K3: fused consumers.  kV = number of dot products per group (batch rows of x, or query
@@ -76,27 +70,11 @@ template <int kV>
 __device__ __forceinline__ void fused_group(const Block& blk, const Tables& tb, const WarpSmem& ws, float T,
                                             uint32_t xs, Accum<kV>& acc)
 {
-    const GroupHeader h = open_group<kFusedTab>(blk, tb, ws, T);
-#if ECCO_FUSED_LOCALRANKS
-    uint32_t ranks[16];                                     // thread-local: indexed by the step, so it lives in local memory
-    uint32_t word = 0;
-#else
+    const GroupHeader h = open_group<kTabFloat>(blk, tb, ws, T);
     RankPacker rk;
-#endif
-    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree, kFusedTab>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t pair) {
-        acc.fma(n, fused_value(v), xs);
-#if ECCO_FUSED_LOCALRANKS
-        if (!(n & 1)) {
-            switch ((n & 7) >> 1) {
-                case 0: word = pair; break;
-                case 1: word = prmt(word, pair, 0x3240u); break;
-                case 2: word = prmt(word, pair, 0x3410u); break;
-                default: word = prmt(word, pair, 0x4210u); ranks[n >> 3] = word; break;
-            }
-        }
-#else
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t pair) {
+        acc.fma(n, __uint_as_float(v), xs);
         rk.put(n, pair, ws.syms);
-#endif
     });
     if (end) {
         // outliers replace the mapped value at their location: add (outlier - mapped) * x
@@ -109,13 +87,9 @@ __device__ __forceinline__ void fused_group(const Block& blk, const Tables& tb, 
             const bool upper = loc >= 64u;
             if ((upper ? seen_hi : seen_lo) & bit) continue;
             if (upper) seen_hi |= bit; else seen_lo |= bit;
-#if ECCO_FUSED_LOCALRANKS
-            const uint32_t w = ranks[loc >> 3];
-#else
-            const uint32_t w = lds_u32(ws.syms + (loc >> 3) * 128);
-#endif
-            const uint32_t rank = (w >> ((loc & 7u) * 4)) & 15u;
-            const float mapped = fused_value(lds_tab<kFusedTab>(ws.tab + rank * 128));
+            const uint32_t word = lds_u32(ws.syms + (loc >> 3) * 128);
+            const uint32_t rank = (word >> ((loc & 7u) * 4)) & 15u;
+            const float mapped = __uint_as_float(lds_u32(ws.tab + rank * 128));
             const float outlier = __half2float(__float2half_rn(fp8_to_float(f >> 7) * T));
             acc.fma_at(loc, outlier - mapped, xs);
         }
@@ -133,15 +107,13 @@ __host__ __device__ __forceinline__ int unit_owner(int64_t U, int G, int64_t u)
 }
 
 // per-warp arrays of the scalar fused kernels: value table (fp32), bit-stream array, decoded ranks
-constexpr uint32_t kFusedSyms = ECCO_FUSED_LOCALRANKS ? 0u : kSymsBytes;
-constexpr uint32_t kFusedWarpBytes = (ECCO_FUSED_HALFTAB ? kTabBytes / 2 : kTabBytes) + kBitsBytes + kFusedSyms;
-constexpr uint32_t kFusedTail = ECCO_FUSED_HALFTAB ? kTabBytes / 2 : 0u;       // an odd warp count leaves half a table unused
+constexpr uint32_t kFusedWarpBytes = kTabBytes + kBitsBytes + kSymsBytes;
 __device__ __forceinline__ WarpSmem fused_warp_smem(const Tables& tb, uint32_t nw)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     WarpSmem ws;
-    ws.tab = tab_column<kFusedTab>(tb.warp_base, warp, lane);
-    ws.bits = tb.warp_base + tab_bytes<kFusedTab>(nw) + warp * (kBitsBytes + kFusedSyms) + lane * 4;
+    ws.tab = tab_column<kTabFloat>(tb.warp_base, warp, lane);
+    ws.bits = tb.warp_base + nw * kTabBytes + warp * (kBitsBytes + kSymsBytes) + lane * 4;
     ws.syms = ws.bits + kBitsBytes;
     if (warp < nw) {
         sts_u32(ws.bits + 16 * 128, 0u);
@@ -169,10 +141,10 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
-    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes, kFusedTail));
+    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes));
     const WarpSmem ws = fused_warp_smem(tb, nw);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    const uint32_t xs = tb.warp_base + tab_bytes<kFusedTab>(nw) + nw * (kBitsBytes + kFusedSyms) + warp * kXsBytes;   // this warp's slice
+    const uint32_t xs = tb.warp_base + nw * kFusedWarpBytes + warp * kXsBytes;   // this warp's slice
 
     // W working warps (chosen by the host so that they all get the same number of units, and never
     // more than there are units); warp ids interleave over the CTAs; the other warps idle
@@ -289,10 +261,10 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
-    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes, kGroup * kV * 4 + kFusedTail));
+    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes, kGroup * kV * 4));
     const int kTokens = nw * 32;                           // tokens per unit: one per thread of the working warps
     const WarpSmem ws = fused_warp_smem(tb, nw);
-    const uint32_t xs_addr = tb.warp_base + tab_bytes<kFusedTab>(nw) + nw * (kBitsBytes + kFusedSyms);
+    const uint32_t xs_addr = tb.warp_base + nw * kFusedWarpBytes;
     float* xs = reinterpret_cast<float*>(smem + (xs_addr - tb.base));
 
     const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
