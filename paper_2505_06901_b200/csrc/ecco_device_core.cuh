@@ -271,8 +271,8 @@ struct WarpSmem {
 
 struct GroupHeader {
     uint32_t pos;       // first bit of the coded indices
-    uint32_t blut;      // shared address of the shape table of (ID_KP, ID_HF): 256-byte aligned
-    uint32_t plut;      // shared address of its pair table (aligned to the table's size)
+    uint32_t blut;      // shared address of the shape table of (ID_KP, ID_HF) (256-byte aligned), OR-ed with its rotation
+    uint32_t plut;      // shared address of its pair table (aligned to the table's size), OR-ed with its rotation
     uint32_t mask;      // ((1 << W) - 1) << 1: byte offset of a pair-table entry from a window that starts one bit early
 };
 
@@ -293,8 +293,9 @@ __device__ __forceinline__ GroupHeader open_header(uint32_t hdr, uint32_t first_
     const uint32_t cb = kp * kCodebooks + hf;
     uint4 rec;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(rec.x), "=r"(rec.y), "=r"(rec.z), "=r"(rec.w) : "r"(tb.base + kSmemCbRec + cb * 16));
-    h.blut = tb.shape + ((rec.x >> 8) & 0xffu) * 256u;
-    h.plut = tb.pair + ((rec.x & 0xffu) << 9);
+    const uint32_t shape = (rec.x >> 8) & 0xffu, rot = table_rotation(shape);   // entry of window i at offset (size * i) ^ rot
+    h.blut = (tb.shape + shape * 256u) | rot;
+    h.plut = (tb.pair + ((rec.x & 0xffu) << 9)) | rot;
     h.mask = ((1u << (rec.x >> 16)) - 1u) << 1;
     const float top = fp8_to_float(qs) * T;           // FP8 -> FP16 range by the power-of-two factor
     const float s = fabsf(top);
@@ -356,7 +357,7 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         uint32_t e[4], end[4], acc = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            e[j] = lds_u8(h.blut | ((win >> acc) & 0xffu));
+            e[j] = lds_u8(h.blut ^ ((win >> acc) & 0xffu));
             acc += e[j] >> 4;
             end[j] = acc;
         }
@@ -379,12 +380,12 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
     auto single_at = [&](uint32_t q) {
         const uint32_t qi = min(q >> 5, kLastRow);
         const uint32_t lo = lds_u32(ws.bits + qi * 128), hi = lds_u32(ws.bits + qi * 128 + 128);
-        return lds_u8(h.blut | (__funnelshift_r(lo, hi, q) & 0xffu));
+        return lds_u8(h.blut ^ (__funnelshift_r(lo, hi, q) & 0xffu));
     };
     // an escape entry completed with its second symbol, which starts `off` bits into the window (off = 1 + the bits
     // before it); the window has it whole unless off > 24, which takes three 8-bit codewords in a row
     auto resolve = [&](int32_t e, uint32_t win, uint32_t off, uint32_t p) {
-        const uint32_t b = off <= 24u ? lds_u8(h.blut | ((win >> off) & 0xffu)) : single_at(p + (static_cast<uint32_t>(e) & 15u));
+        const uint32_t b = off <= 24u ? lds_u8(h.blut ^ ((win >> off) & 0xffu)) : single_at(p + (static_cast<uint32_t>(e) & 15u));
         return static_cast<int32_t>((static_cast<uint32_t>(e) & 0x078fu) + (b >> 4) + ((b & 15u) << 11));
     };
     // Two symbols per lookup, software-pipelined by hand: a warp issues in order and every shared-memory load here is
@@ -409,16 +410,16 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
     auto four_pair = [&](int step, auto tested) {
         constexpr bool kTest = decltype(tested)::value;
         const uint32_t win = __funnelshift_r(lo, hi, pos - 1u);
-        int32_t e0 = lds_s16(h.plut | (win & h.mask));
+        int32_t e0 = lds_s16(h.plut ^ (win & h.mask));
         if (pending) deliver(step - 1);                                // while the lookup is in flight
-        int32_t e1 = lds_s16(h.plut | (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));   // shift by e0 mod 32 = its length field
+        int32_t e1 = lds_s16(h.plut ^ (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));   // shift by e0 mod 32 = its length field
         const bool esc = (e0 | e1) < 0;
         uint32_t acc = static_cast<uint32_t>(e0 + e1) & 0x7fu;      // bits consumed by the four symbols (if no escape)
         if (__any_sync(kFull, esc || (kTest && pos + acc > kEndBit))) {
             if (esc) {
                 if (e0 < 0) {
                     e0 = resolve(e0, win, 1u + (static_cast<uint32_t>(e0) & 15u), pos);
-                    e1 = lds_s16(h.plut | (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));
+                    e1 = lds_s16(h.plut ^ (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));
                 }
                 if (e1 < 0) e1 = resolve(e1, win, 1u + (static_cast<uint32_t>(e0) & 31u) + (static_cast<uint32_t>(e1) & 15u), pos + (static_cast<uint32_t>(e0) & 31u));
                 acc = static_cast<uint32_t>(e0 + e1) & 0x7fu;

@@ -82,11 +82,17 @@ constexpr uint32_t kPairBudgetBytes = 80u << 10;
 constexpr uint32_t kMaxDevBytes = kOffShapeLut + kMaxShapes * 256 + kPairBudgetBytes;
 // Both kinds of table are indexed by the next stream bits with the first stream bit in bit 0,
 // i.e. by the bit-reversed codeword followed by whatever comes next.
+//
+// Both are stored with a per-shape rotation: the entry for window value i sits at byte offset
+// (entry size * i) ^ table_rotation(shape).  The rotation touches offset bits 2..6, which select the
+// shared-memory bank, so lanes that decode with different shapes spread over different banks even when
+// their windows agree (neighbouring groups often start with the same few codewords).
 #ifdef __CUDACC__
 #define ECCO_HD __host__ __device__
 #else
 #define ECCO_HD
 #endif
+ECCO_HD constexpr uint32_t table_rotation(uint32_t shape) { return ((shape * 11u + (shape >> 3)) & 31u) << 2; }
 
 // Variable-length container: index = u64 total_bits | u64 chunk_base[ceil(n / 4096)] | u32 offset[n];
 // group g starts at stream bit chunk_base[g >> 12] + offset[g].

@@ -1008,7 +1008,7 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
         }
     // shape tables, then pair tables built from them
     for (int sh = 0; sh < p.n_shapes; ++sh) {
-        uint8_t* t = base + kOffShapeLut + static_cast<size_t>(sh) * 256;
+        uint8_t t[256];                                    // the shape table in natural order
         uint32_t code = 0;
         int rank = 0;
         for (int L = kMinLen; L <= kMaxLen; ++L) {
@@ -1018,6 +1018,9 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
             }
             code <<= 1;
         }
+        const uint32_t rot = table_rotation(static_cast<uint32_t>(sh));
+        uint8_t* st = base + kOffShapeLut + static_cast<size_t>(sh) * 256;
+        for (uint32_t i = 0; i < 256; ++i) st[i ^ rot] = t[i];
         const int W = p.width[sh];
         if (!W) continue;
         uint16_t* pt = reinterpret_cast<uint16_t*>(base + p.off_pair + p.pair_off[sh]);
@@ -1026,8 +1029,8 @@ extern "C" int ecco_meta_serialize_device(const ecco_meta* m, void* host_staging
             const uint32_t room = static_cast<uint32_t>(W) - l0;              // bits of the window after the first codeword
             const uint32_t e1 = t[(idx >> l0) & 255u], l1 = e1 >> 4, r1 = e1 & 15u;   // bits past the window read as zero
             // a codeword no longer than the bits on hand is fully inside them, so it is the real one
-            pt[idx] = l1 <= room ? static_cast<uint16_t>((l0 + l1) | (r0 << 7) | (r1 << 11))
-                                 : static_cast<uint16_t>(l0 | (r0 << 7) | 0x8000u);
+            pt[idx ^ (rot >> 1)] = l1 <= room ? static_cast<uint16_t>((l0 + l1) | (r0 << 7) | (r1 << 11))
+                                              : static_cast<uint16_t>(l0 | (r0 << 7) | 0x8000u);
         }
     }
     DevHeader h;

@@ -174,6 +174,11 @@ def _image_views(img):
     return v
 
 
+def _rotation(shape):
+    """Byte-offset rotation of the tables of a shape (csrc/ecco_format.h: table_rotation)."""
+    return ((shape * 11 + (shape >> 3)) & 31) << 2
+
+
 def _walk_with_image_tables(v, blk):
     """A block decoded the way the kernels do it, in Python: four symbols per step from a window that starts one
     bit early, two pair-table lookups, escapes completed through the shape table, and the one-symbol-per-lookup
@@ -187,13 +192,14 @@ def _walk_with_image_tables(v, blk):
     rank_of = int(rec[2]) | int(rec[3]) << 32
     sym_of_rank = {(rank_of >> 4 * s) & 15: s for s in range(16)}
     assert len(sym_of_rank) == 16
-    blut = v["shape"][shape]
+    rot = _rotation(shape)                                 # tables are stored rotated: window i at byte offset (size * i) ^ rot
+    blut = v["shape"][shape][np.arange(256) ^ rot]
     plut = v["pair"][pair_off:pair_off + (2 << width)].view(np.uint16) if width else None
     mask = ((1 << width) - 1) << 1
     ranks, alive = [], True
 
     def entry(off):                                        # signed 16-bit pair-table entry at byte offset off
-        x = int(plut[off >> 1])
+        x = int(plut[(off ^ rot) >> 1])
         return x - 65536 if x & 0x8000 else x
 
     def resolve(e, p):
@@ -285,11 +291,13 @@ def test_device_image_shape_and_pair_tables_against_canonical_codes(binding, eo,
             for rest in range(1 << (8 - L)):
                 i = int(f"{code << (8 - L) | rest:08b}"[::-1], 2)     # the window with the first stream bit in bit 0
                 want_len[i], want_rank[i] = L, (rank_of >> 4 * s) & 15
-        assert np.array_equal(v["shape"][shape] >> 4, want_len) and np.array_equal(v["shape"][shape] & 15, want_rank)
+        rot = _rotation(shape)
+        table = v["shape"][shape][np.arange(256) ^ rot]
+        assert np.array_equal(table >> 4, want_len) and np.array_equal(table & 15, want_rank)
         assert 8 <= width <= 12 and pair_off % (2 << width) == 0
         widths_by_offset[pair_off] = width
-        pt = v["pair"][pair_off:pair_off + (2 << width)].view(np.uint16).astype(np.int64)
         idx = np.arange(1 << width)
+        pt = v["pair"][pair_off:pair_off + (2 << width)].view(np.uint16).astype(np.int64)[idx ^ (rot >> 1)]
         l0, r0 = want_len[idx & 255], want_rank[idx & 255]
         rest = idx >> l0
         l1, r1 = want_len[rest & 255], want_rank[rest & 255]
