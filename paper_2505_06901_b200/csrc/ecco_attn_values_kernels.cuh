@@ -96,8 +96,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
-    Block blk;
-    if (u0 < u1 && working) ldg_block(blk, block_ptr(u0));
+    if (u0 < u1 && working) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
@@ -192,8 +191,9 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                 p_lo[j] = static_cast<uint32_t>(__half_as_ushort(l0)) | (static_cast<uint32_t>(__half_as_ushort(l1)) << 16);
             }
         }
-        const Block cur = blk;
-        if (u + 1 < u1) ldg_block(blk, block_ptr(u + 1));
+        Block cur;                                         // fetched now, prefetched into L2 one unit earlier
+        ldg_block(cur, block_ptr(u));
+        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
         const bool valid = t < seq;                        // lanes past the end stage zeros (their p is zero too)
         const GroupHeader h = open_group<kTabHalfBits>(cur, tb, ws, T);
         // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
