@@ -213,6 +213,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
         }
         // pass 2: per 16-dim chunk map the indices, patch the outliers in the tile, contract on the tensor cores
+#pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
             uint32_t r8[8];
             const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
@@ -243,17 +244,10 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                 const uint32_t tok = (lane >> 4) * 8 + (lane & 7u) + 16 * ks, half = (lane >> 3) & 1u;
                 ldmatrix_x4_trans(a[ks], stage + tok * 32 + ((half ^ ((tok >> 2) & 1u)) << 4));
             }
-            // ch is uniform but not a compile-time constant: pick the accumulator set by uniform branches so
-            // that it stays in registers
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                if (ch == k) {
-#pragma unroll
-                    for (int ks = 0; ks < 2; ++ks) {
-                        mma_16816(acc[k], a[ks], p_hi[2 * ks], p_hi[2 * ks + 1]);
-                        mma_16816(acc[k], a[ks], p_lo[2 * ks], p_lo[2 * ks + 1]);
-                    }
-                }
+            for (int ks = 0; ks < 2; ++ks) {
+                mma_16816(acc[ch], a[ks], p_hi[2 * ks], p_hi[2 * ks + 1]);
+                mma_16816(acc[ch], a[ks], p_lo[2 * ks], p_lo[2 * ks + 1]);
             }
         }
     }
