@@ -228,7 +228,8 @@ def cpu_baseline(layer, c: int, kv_tensor=None):
         t0 = time.perf_counter()
         eo.gemv(om, t.blocks[: rows * (k // G)], rows, k, x, 1)
         dt = time.perf_counter() - t0
-        fused["ecco_gemv batch 1"] = {"us_per_layer_equivalent": None, "weights_per_s": rows * k / dt, "cores": 1,
+        layer_weights = sum(int(np.prod(m.shape)) for m in layer if len(m.shape) == 2)
+        fused["ecco_gemv batch 1"] = {"us_per_layer_equivalent": layer_weights * dt / (rows * k) * 1e6, "weights_per_s": rows * k / dt, "cores": 1,
                                       "sample": f"first {rows} rows of '{t.name}' {tuple(t.shape)}"}
     if kv_tensor is not None:
         kb, kh, kseq, _ = kv_tensor.shape

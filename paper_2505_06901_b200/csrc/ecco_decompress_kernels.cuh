@@ -246,7 +246,9 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
 
     dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
-    const Tables tb = plan_tables(smem_u32(smem), d_meta);
+    // one symbol per lookup: a warp's 40-row stream array takes 5 KB, and 28 warps beside the shape tables measured
+    // as fast as 20 beside the pair tables
+    const Tables tb = plan_tables(smem_u32(smem), d_meta, false);
     const uint32_t nw = warps_that_fit(tb, kVarWarpBytes, kTabBytes / 2);
     WarpSmem ws;
     ws.tab = tab_column<kTabHalf>(tb.warp_base, warp, lane);

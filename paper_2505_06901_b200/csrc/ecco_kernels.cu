@@ -210,7 +210,7 @@ extern "C" int ecco_decompress(const void* d_meta, const uint8_t* d_blocks, uint
     return ecco_decompress_batch(&item, 1, stream);
 }
 
-constexpr int kVarWarps = 24;
+constexpr int kVarWarps = 28;
 
 extern "C" int ecco_var_decompress(const void* d_meta, const uint8_t* d_stream, const void* d_index, uint64_t n_groups, void* d_out,
                                    void* stream)
