@@ -27,7 +27,10 @@
  *
  * Stream order: the usual one.  Internally the kernels are launched so that one may become
  * resident while the previous kernel of the stream is still draining, but each waits for that
- * kernel to complete before its first access to memory, so only launch latency overlaps.
+ * kernel to complete before its first access to memory, so only launch latency overlaps.  The
+ * one thing a kernel reads before that wait is the metadata image: d_meta must be filled by a
+ * copy (cudaMemcpy / cudaMemcpyAsync, which the stream orders as usual), not written by a kernel
+ * that is still running when the call is issued.
  */
 #ifndef ECCO_H_
 #define ECCO_H_

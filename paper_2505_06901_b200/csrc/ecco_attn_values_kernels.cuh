@@ -62,7 +62,6 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     const int tid = static_cast<int>(threadIdx.x), n_threads = static_cast<int>(blockDim.x);
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar fused kernels
     const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kGroup * 8 * sizeof(float));
@@ -96,6 +95,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         return d_vblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     if (u0 < u1 && working) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;

@@ -112,7 +112,9 @@ ecco_decompress_tma_kernel(const __grid_constant__ DecompressBatch batch)
     const uint32_t smem_base = smem_u32(smem);
     const uint32_t swz = ((lane >> 2) & 1u) << 4;                               // 32-byte swizzle: bit 4 ^= bit 7
 
-    dependency_wait();
+    // The metadata images are written by the host only, never by a kernel of this library, and this kernel can
+    // start early only behind a kernel that releases its dependents, i.e. one of this library: the tables of the
+    // first run are fetched before the wait on the previous kernel, everything else after it.
     release_dependents();
     auto hash_of = [&](int t) {
         const DevHeader* hd = reinterpret_cast<const DevHeader*>(batch.job[t].meta);
@@ -155,6 +157,7 @@ ecco_decompress_tma_kernel(const __grid_constant__ DecompressBatch batch)
             const DecompressJob& job = batch.job[c.job];
             return job.blocks + min((g - c.first) * 32 + lane, job.n_groups - 1) * kBlockBytes;
         };
+        if (run == 0) dependency_wait();                   // blocks and output: only after the previous kernel has completed
         if (gt < run_tiles) { seek(cur, gt); prefetch_block_l2(block_ptr(cur, gt)); }
         if (!wait_tables(tb, static_cast<uint32_t>(run & 1))) return;
         float T = tb.T;
@@ -244,7 +247,6 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     extern __shared__ __align__(1024) uint8_t smem[];
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
 
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     // one symbol per lookup: a warp's 40-row stream array takes 5 KB, and 28 warps beside the shape tables measured
     // as fast as 20 beside the pair tables
@@ -260,6 +262,7 @@ ecco_var_decompress_kernel(const uint8_t* __restrict__ d_meta, const uint4* __re
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     const uint64_t total_bits = d_index[0];
     const uint64_t stream_chunks = (total_bits + 127) >> 7;
     const uint64_t* chunk_base = d_index + 1;

@@ -240,8 +240,11 @@ __device__ __forceinline__ bool wait_tables(const Tables& tb, uint32_t parity = 
 // Programmatic dependent launch: a kernel launched with the stream-serialisation attribute may become resident
 // while the previous kernel in the stream is still draining.  dependency_wait() returns once that kernel has
 // completed and its writes are visible (at once if there is no such overlap); every kernel executes it before
-// its first access to global memory, so stream order is what it is without the attribute and only launch and
-// prologue overlap.  release_dependents() lets the next kernel of the stream do the same with respect to this one.
+// its first access to global memory other than the metadata image, so stream order is what it is without the
+// attribute and only launch, table fetch and prologue overlap.  The image is the exception because no kernel writes
+// it: it reaches the device by a copy, which is a stream operation of its own (a kernel behind a copy starts after
+// it), and a kernel can start early only behind one that releases its dependents, i.e. one of this file.
+// release_dependents() lets the next kernel of the stream do the same with respect to this one.
 __device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
@@ -407,11 +410,14 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
         sink(step * 4 + 2, pv[2], (pu1 >> 7) & 15u, true, pu1 >> 7);
         sink(step * 4 + 3, pv[3], (pu1 >> 11) & 15u, true, 0u);
     };
-    auto four_pair = [&](int step, auto tested) {
+    // owed: 0 = nothing to deliver (first step), 1 = the previous step is always owed (steps without the clip test
+    // after the first), 2 = look at `pending`
+    auto four_pair = [&](int step, auto tested, auto owed) {
         constexpr bool kTest = decltype(tested)::value;
+        constexpr int kOwed = decltype(owed)::value;
         const uint32_t win = __funnelshift_r(lo, hi, pos - 1u);
         int32_t e0 = lds_s16(h.plut ^ (win & h.mask));
-        if (pending) deliver(step - 1);                                // while the lookup is in flight
+        if (kOwed == 1 || (kOwed == 2 && pending)) deliver(step - 1);  // while the lookup is in flight
         int32_t e1 = lds_s16(h.plut ^ (__funnelshift_r(win, 0u, static_cast<uint32_t>(e0)) & h.mask));   // shift by e0 mod 32 = its length field
         const bool esc = (e0 | e1) < 0;
         uint32_t acc = static_cast<uint32_t>(e0 + e1) & 0x7fu;      // bits consumed by the four symbols (if no escape)
@@ -445,12 +451,16 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
     };
     if (pairs) {
         load_window(cuda::std::false_type{});
+        using Never = cuda::std::integral_constant<int, 0>;
+        using Always = cuda::std::integral_constant<int, 1>;
+        using Check = cuda::std::integral_constant<int, 2>;
         if (kFreeSteps > 0) {
+            four_pair(0, cuda::std::false_type{}, Never{});
 #pragma unroll 4
-            for (int step = 0; step < kFreeSteps; ++step) four_pair(step, cuda::std::false_type{});
+            for (int step = 1; step < kFreeSteps; ++step) four_pair(step, cuda::std::false_type{}, Always{});
         }
 #pragma unroll 4
-        for (int step = kFreeSteps; step < 32; ++step) four_pair(step, cuda::std::true_type{});
+        for (int step = kFreeSteps; step < 32; ++step) four_pair(step, cuda::std::true_type{}, Check{});
         if (pending) deliver(31);
     } else {
         if (kFreeSteps > 0) {

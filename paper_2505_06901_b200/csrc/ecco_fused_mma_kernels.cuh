@@ -133,7 +133,6 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
     const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
@@ -151,6 +150,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
@@ -221,7 +221,6 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
     const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
@@ -238,6 +237,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;

@@ -138,7 +138,6 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr uint32_t kXsBytes = kGroup * kV * 4;
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
     const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes));
@@ -159,6 +158,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
@@ -258,7 +258,6 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                         int q_per_kv, const __half* d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
-    dependency_wait();                                     // the previous kernel of the stream has completed
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
     const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes, kGroup * kV * 4));
@@ -278,6 +277,7 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
+    dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     if (u0 < u1 && working) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
