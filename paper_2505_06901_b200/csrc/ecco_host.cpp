@@ -135,9 +135,6 @@ struct ecco_meta {
     float pattern_f[kMaxPatterns][kCentroids] = {};
     uint16_t cb_rev[kMaxPatterns][kCodebooks][kSymbols] = {};   // bit-reversed codewords (stream order, lsb first)
     uint16_t kp_rev[kMaxPatterns] = {};
-    // how often the host encoder has picked each codebook with this metadata so far (a hint for the device image:
-    // which code shapes deserve the wide decode tables; all zero = unknown)
-    uint64_t cb_use[kMaxPatterns][kCodebooks] = {};
 };
 
 namespace {
@@ -600,8 +597,6 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
     const float T = std::ldexp(1.0f, m->e);
     const int threads = available_cores();
     std::vector<ecco_stats> part(static_cast<size_t>(threads));
-    struct CbUse { uint64_t n[kMaxPatterns][kCodebooks]; };
-    std::vector<CbUse> use(static_cast<size_t>(threads));
     std::atomic<int> err{0};
     parallel_ranges(n_groups, threads, [&](int t, uint64_t lo, uint64_t hi) {
         Scratch s;
@@ -609,12 +604,9 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
         GroupOut g;
         ecco_stats st;
         std::memset(&st, 0, sizeof st);
-        CbUse& cu = use[static_cast<size_t>(t)];
-        std::memset(&cu, 0, sizeof cu);
         for (uint64_t i = lo; i < hi && !err.load(std::memory_order_relaxed); ++i) {
             int r = encode_group(*m, src + i * kGroup, select, T, s, dst + i * kBlockBytes, g, q);
             if (r) { err = r; break; }
-            cu.n[g.kp][g.hf]++;
             st.n_groups++;
             if (g.n_fit < kGroup) { st.clipped_groups++; st.clipped_values += static_cast<uint64_t>(kGroup - g.n_fit); }
             if (g.n_pad) { st.padded_groups++; st.padded_values += static_cast<uint64_t>(g.n_pad); }
@@ -626,9 +618,6 @@ extern "C" int ecco_encode_host(ecco_meta* m, const uint16_t* src, uint64_t n_gr
         part[static_cast<size_t>(t)] = st;
     });
     if (err) return err;
-    for (const auto& cu : use)
-        for (int k = 0; k < kMaxPatterns; ++k)
-            for (int h = 0; h < kCodebooks; ++h) m->cb_use[k][h] += cu.n[k][h];
     if (stats) {
         std::memset(stats, 0, sizeof *stats);
         for (const auto& p : part) {
@@ -895,10 +884,10 @@ double escape_rate(const uint8_t* counts, int W)
 
 void plan_image(const ecco_meta& m, ImagePlan& p)
 {
+    // Expected use of a shape: what the ID_KP code lengths say about its patterns (a pattern coded in L bits is
+    // used about 2^-L of the time), the four codebooks of a pattern alike.  A function of the metadata alone, so
+    // that tensors encoded with the same patterns and codebooks get the same tables, hence the same table hash.
     double use[kMaxShapes] = {};
-    uint64_t seen = 0;
-    for (int k = 0; k < m.S; ++k)
-        for (int h = 0; h < kCodebooks; ++h) seen += m.cb_use[k][h];
     for (int k = 0; k < kMaxPatterns; ++k)
         for (int h = 0; h < kCodebooks; ++h) {
             uint8_t c[kMaxLen + 1] = {};
@@ -909,9 +898,7 @@ void plan_image(const ecco_meta& m, ImagePlan& p)
                 if (!std::memcmp(p.counts[i], c, sizeof c)) id = i;
             if (id < 0) { id = p.n_shapes++; std::memcpy(p.counts[id], c, sizeof c); }
             p.shape_of[k][h] = id;
-            if (k < m.S)     // expected use: what the encoder has seen, else what the ID_KP code lengths say
-                use[id] += seen ? static_cast<double>(m.cb_use[k][h]) / static_cast<double>(seen)
-                                : std::ldexp(1.0, -m.kp_len[k]) / kCodebooks;
+            if (k < m.S) use[id] += std::ldexp(1.0, -m.kp_len[k]) / kCodebooks;
         }
     // widths: everyone starts at the minimum; then the upgrade that removes the most escapes per byte, while it fits
     uint32_t bytes = static_cast<uint32_t>(p.n_shapes) * (2u << kPairMinBits);

@@ -311,6 +311,28 @@ def test_device_image_shape_and_pair_tables_against_canonical_codes(binding, eo,
     assert sum(2 << w for w in widths_by_offset.values()) == v["pair_bytes"] <= 80 * 1024
 
 
+def test_device_image_tables_depend_on_the_metadata_only(binding, eo, cfg1_small):
+    """Tensors encoded with the same patterns and codebooks must get the same decode tables and the same table hash
+    (ecco_decompress_batch decodes consecutive tensors of equal hash as one run), whatever was encoded with the
+    metadata before the image was made and whatever exponent the tensor got."""
+    fresh = lib_meta_from_oracle(binding, cfg1_small["meta"])
+    used = lib_meta_from_oracle(binding, cfg1_small["meta"])
+    skewed = (cfg1_small["w"].astype(np.float32) ** 3 * 50.0).astype(np.float16)     # other codebook choices, other exponent
+    binding.ecco_encode_host(used, skewed, binding.SELECT_MSE)
+    assert used.tables()[1] != fresh.tables()[1]
+    a, b = binding.ecco_meta_serialize_device(fresh), binding.ecco_meta_serialize_device(used)
+    va, vb = _image_views(a), _image_views(b)
+    assert a.size == b.size and np.array_equal(va["hdr"][12:14], vb["hdr"][12:14])
+    assert np.array_equal(a[OFF_PATTERN:], b[OFF_PATTERN:])          # everything but the header (exponent, T)
+    other = lib_meta_from_oracle(binding, cfg1_small["meta"])
+    S, e, pat, cb, kp = other.tables()
+    cb = cb.copy()
+    cb[0, 0] = cb[0, 0][::-1]                                         # same lengths on other symbols: another code
+    changed = binding.ecco_meta_create(S, e, pat, cb, kp)
+    vc = _image_views(binding.ecco_meta_serialize_device(changed))
+    assert not np.array_equal(va["hdr"][12:14], vc["hdr"][12:14])
+
+
 def _complete_length_multisets():
     """Every way to give 16 symbols code lengths in 2..8 with Kraft sum exactly 1, as counts per length."""
     out = []
