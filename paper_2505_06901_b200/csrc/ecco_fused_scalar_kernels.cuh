@@ -249,59 +249,71 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
     if (u0 < u1) flush(cur_tile);
 }
 
-// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t].  A work unit is (one (batch, kv
-// head) pair, a chunk of kWarps*32 tokens); units are dealt to persistent CTAs in contiguous runs,
-// the query slice is restaged when the head changes, a thread owns one token.
+// K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for one or two query heads per KV head.
+// Built like K2: a work unit is (one (batch, kv head) pair, 32 consecutive tokens), a lane owns one token, every
+// working warp owns a contiguous run of units and keeps its own query slice (pre-multiplied by scale, restaged
+// when the head changes), so warps never meet at a barrier and a ragged sequence length costs at most one
+// partly filled unit per head.
 template <int kV, int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
 ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_kblocks, int heads, int seq,
                         int q_per_kv, const __half* d_q, float scale, float* __restrict__ d_scores)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
+    constexpr uint32_t kXsBytes = kGroup * kV * 4;
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
-    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes, kGroup * kV * 4));
-    const int kTokens = nw * 32;                           // tokens per unit: one per thread of the working warps
+    const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes));
     const WarpSmem ws = fused_warp_smem(tb, nw);
-    const uint32_t xs_addr = tb.warp_base + nw * kFusedWarpBytes;
-    float* xs = reinterpret_cast<float*>(smem + (xs_addr - tb.base));
+    const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
+    const uint32_t xs = tb.warp_base + nw * kFusedWarpBytes + warp * kXsBytes;   // this warp's slice: xs[d][r]
 
-    const int G = gridDim.x, c = blockIdx.x, tid = static_cast<int>(threadIdx.x);
-    const bool working = tid < kTokens;
-    const int chunks = (seq + kTokens - 1) / kTokens;
-    const int64_t U = static_cast<int64_t>(heads) * chunks;
-    const int64_t u0 = unit_begin(U, G, c), u1 = unit_begin(U, G, c + 1);
+    const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
+    const int tiles = (seq + 31) / 32;
+    const int64_t U = static_cast<int64_t>(heads) * tiles;
+    const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
+    const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     // lanes past the end of the sequence decode its last token again and store nothing
     auto block_ptr = [&](int64_t u) {
-        const int bh = static_cast<int>(u / chunks), t = min(static_cast<int>(u % chunks) * kTokens + tid, seq - 1);
+        const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
         return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
     };
     issue_tables(tb, d_meta);
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
-    if (u0 < u1 && working) prefetch_block_l2(block_ptr(u0));
+    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
     int cur_bh = -1;
     for (int64_t u = u0; u < u1; ++u) {
-        const int bh = static_cast<int>(u / chunks), t = static_cast<int>(u % chunks) * kTokens + tid;
+        const int bh = static_cast<int>(u / tiles), t = static_cast<int>(u % tiles) * 32 + lane;
         if (bh != cur_bh) {
-            __syncthreads();                               // everyone is done with the previous head's slice
-            // q[b][h*q_per_kv + r][d] -> xs[d][r], pre-multiplied by scale; heads beyond q_per_kv are zero
-            for (int i = tid; i < kGroup * kV; i += static_cast<int>(blockDim.x)) {
-                const int r = i % kV, d = i / kV;
-                xs[i] = (r < q_per_kv) ? scale * __half2float(__ldcg(d_q + (static_cast<size_t>(bh) * q_per_kv + r) * kGroup + d)) : 0.0f;
+            // lane l stages q[b][h*q_per_kv + r][4l .. 4l+3] * scale as fp32, layout xs[d][r]; heads beyond q_per_kv are zero
+            float v[kV][4];
+#pragma unroll
+            for (int r = 0; r < kV; ++r) {
+                uint2 raw = make_uint2(0u, 0u);
+                if (r < q_per_kv) raw = __ldcg(reinterpret_cast<const uint2*>(d_q + (static_cast<size_t>(bh) * q_per_kv + r) * kGroup) + lane);
+                const __half2 h0 = *reinterpret_cast<const __half2*>(&raw.x), h1 = *reinterpret_cast<const __half2*>(&raw.y);
+                v[r][0] = scale * __low2float(h0); v[r][1] = scale * __high2float(h0);
+                v[r][2] = scale * __low2float(h1); v[r][3] = scale * __high2float(h1);
             }
-            __syncthreads();
+            __syncwarp();                                  // every lane is done with the previous head's slice
+            if constexpr (kV == 1) {
+                sts_v4(xs + lane * 16, __float_as_uint(v[0][0]), __float_as_uint(v[0][1]), __float_as_uint(v[0][2]), __float_as_uint(v[0][3]));
+            } else {
+                sts_v4(xs + lane * 32, __float_as_uint(v[0][0]), __float_as_uint(v[1][0]), __float_as_uint(v[0][1]), __float_as_uint(v[1][1]));
+                sts_v4(xs + lane * 32 + 16, __float_as_uint(v[0][2]), __float_as_uint(v[1][2]), __float_as_uint(v[0][3]), __float_as_uint(v[1][3]));
+            }
+            __syncwarp();
             cur_bh = bh;
         }
-        if (!working) continue;                            // warps without room for their arrays only help with the slice
         Block cur;
         ldg_block(cur, block_ptr(u));
         if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
         Accum<kV> acc;
         acc.clear();
-        fused_group<kV>(cur, tb, ws, T, xs_addr, acc);
+        fused_group<kV>(cur, tb, ws, T, xs, acc);
         if (t < seq) {
 #pragma unroll
             for (int r = 0; r < kV; ++r)

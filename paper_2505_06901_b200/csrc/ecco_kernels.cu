@@ -358,9 +358,10 @@ static int launch_attn(const DeviceInfo& di, const void* d_meta, const uint8_t* 
     int rc = want_all_smem(kernel, &configured[di.device]);
     if (rc) return rc;
     const int heads = batch * n_kv_heads;
-    // persistent CTAs; the units (a head's tokens in chunks of one per working thread) are split evenly on the device
-    const int64_t most_units = static_cast<int64_t>(heads) * ((seq + 31) / 32);
-    const unsigned grid = static_cast<unsigned>(most_units < di.sms ? most_units : di.sms);
+    // persistent CTAs; the units (32 tokens of a head) are split evenly over the working warps on the device
+    const int64_t units = static_cast<int64_t>(heads) * ((seq + 31) / 32);
+    const int64_t ctas = (units + kFusedWarps - 1) / kFusedWarps;
+    const unsigned grid = static_cast<unsigned>(ctas < di.sms ? ctas : di.sms);
     return launch_overlapped(kernel, grid, static_cast<unsigned>(kFusedWarps * 32), kSmemCtaBytes, stream, static_cast<const uint8_t*>(d_meta),
                              d_kblocks, heads, seq, q_per_kv, static_cast<const __half*>(d_q), scale, d_scores);
 }
