@@ -64,7 +64,8 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const int tid = static_cast<int>(threadIdx.x), n_threads = static_cast<int>(blockDim.x);
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar fused kernels
-    const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kGroup * 8 * sizeof(float));
+    constexpr uint32_t kSlotFloats = kGroup * 8, kSlots = (kMaxWarps + 1) / 2;      // reduction slots: see flush
+    const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kSlots * kSlotFloats * sizeof(float));
     const int kTokens = static_cast<int>(nw) * 32;         // tokens per unit: one per thread of the working warps
     const bool working = warp < nw;
     // small CTA-wide words in the misc area at the start of shared memory (the barrier word is its first)
@@ -81,7 +82,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     }
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
     const uint32_t my_row = stage + lane * 32;
-    float* out_s = reinterpret_cast<float*>(smem + (tb.warp_base - tb.base) + nw * kAvWarpBytes);    // [128 dims][8 heads]
+    float* out_s = reinterpret_cast<float*>(smem + (tb.warp_base - tb.base) + nw * kAvWarpBytes);    // slots of [128 dims][8 heads]
 
     const int chunks = (seq + kTokens - 1) / kTokens;
     const int64_t U = static_cast<int64_t>(heads) * chunks;
@@ -109,23 +110,31 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     };
     clear_acc();
 
-    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in warp order, then
-    // either store (this CTA owns the whole head) or hand a partial to the slot-and-ticket reduction
+    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in a fixed order (the first half of
+    // the warps write a slot each, the second half add theirs to the slot of the warp half the count below, then
+    // the slots are added in slot order), then either store (this CTA owns the whole head) or hand a partial to the
+    // slot-and-ticket reduction
     auto flush = [&](int bh) {
-        for (int i = tid; i < kGroup * 8; i += n_threads) out_s[i] = 0.0f;
+        const uint32_t half = (nw + 1u) >> 1;
+        auto my_elements = [&](float* slot, bool add) {
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
+                    const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
+                    const float v = acc[ch][j] * kProbUnscale;
+                    slot[dim * 8 + head] = add ? slot[dim * 8 + head] + v : v;
+                }
+        };
+        if (warp < half) my_elements(out_s + warp * kSlotFloats, false);
         __syncthreads();
-        for (int w = 0; w < static_cast<int>(nw); ++w) {
-            if (static_cast<int>(warp) == w) {
-#pragma unroll
-                for (int ch = 0; ch < 8; ++ch)
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
-                        const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
-                        out_s[dim * 8 + head] += acc[ch][j] * kProbUnscale;
-                    }
-            }
-            __syncthreads();
+        if (warp >= half && warp < nw) my_elements(out_s + (warp - half) * kSlotFloats, true);
+        __syncthreads();
+        for (int i = tid; i < static_cast<int>(kSlotFloats); i += n_threads) {   // thread i keeps element i from here on
+            float sum = out_s[i];
+            for (uint32_t sl = 1; sl < half; ++sl) sum += out_s[sl * kSlotFloats + i];
+            out_s[i] = sum;
         }
         const int c_lo = unit_owner(U, G, static_cast<int64_t>(bh) * chunks);
         const int c_hi = unit_owner(U, G, static_cast<int64_t>(bh + 1) * chunks - 1);
