@@ -190,16 +190,24 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
             if (row_ok) {
 #pragma unroll
                 for (int b = 0; b < kV; ++b) {
-                    // slots are added in warp order whatever the arrival order; loads go out sixteen at a time
+                    // slots are added in warp order whatever the arrival order; loads go out thirty-two at a time (a
+                    // 4096-wide row is 32 k-blocks: one round trip to L2 instead of two at the end of the kernel)
                     const float* slot = d_partial + (static_cast<size_t>(w_lo + tile) * kV + b) * 32 + lane;
                     float sum = 0.0f;
                     int ww = w_lo;
-                    for (; ww + 16 <= w_hi + 1; ww += 16, slot += 16 * kV * 32) {
-                        float v[16];
+                    for (; ww + 32 <= w_hi + 1; ww += 32, slot += 32 * kV * 32) {
+                        float v[32];
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) v[i] = __ldcg(slot + i * kV * 32);
+                        for (int i = 0; i < 32; ++i) v[i] = __ldcg(slot + i * kV * 32);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) sum += v[i];
+                        for (int i = 0; i < 32; ++i) sum += v[i];
+                    }
+                    for (; ww + 8 <= w_hi + 1; ww += 8, slot += 8 * kV * 32) {
+                        float v[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) v[i] = __ldcg(slot + i * kV * 32);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) sum += v[i];
                     }
                     for (; ww <= w_hi; ++ww, slot += kV * 32) sum += __ldcg(slot);
                     d_y[static_cast<size_t>(b) * n_out + row] = sum;
