@@ -154,6 +154,29 @@ size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t batch);
 int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x_fp16,
               int32_t batch, float* d_y, void* d_workspace, size_t workspace_bytes, void* stream);
 
+/* The same for several matrices in one call: y_i = W~_i x_i for up to ECCO_MAX_GEMV_ITEMS matrices that are
+ * independent of each other (the q, k and v projections of a decoder layer, which read the same x; gate and up).  The
+ * work of all matrices is dealt out to the SMs as one, so launch, table fetch and tail are paid once and small
+ * matrices fill the machine together.  All items must have been encoded with the same patterns and codebooks (equal
+ * decode tables; the per-tensor exponent may differ) and use the same batch; x and y are per item and may be shared
+ * between items only for x.  The result is reproducible (the same call gives the same bits) and equals that of
+ * ecco_gemv on each item up to fp32 rounding: a row's sum over k is cut into partial sums at other places.  `items` is a
+ * HOST array read before the call returns.  Errors of the arguments are found before anything is launched; items
+ * whose tables differ from those of the first are detected on the device: nothing is computed and
+ * ecco_device_status() then reports ECCO_ERR_INVALID_ARG.  Workspace as for ecco_gemv, sized by
+ * ecco_gemv_batch_workspace_bytes for the same items. */
+#define ECCO_MAX_GEMV_ITEMS 8
+typedef struct ecco_gemv_item {
+    const void* d_meta;        /* device: metadata image of this matrix */
+    const uint8_t* d_blocks;   /* device: 64 * n_out * (k / 128) bytes */
+    int32_t n_out, k;
+    const void* d_x_fp16;      /* device: fp16 [batch][k] */
+    float* d_y;                /* device: fp32 [batch][n_out] */
+} ecco_gemv_item;
+size_t ecco_gemv_batch_workspace_bytes(const ecco_gemv_item* items, int32_t n_items, int32_t batch);
+int ecco_gemv_batch(const ecco_gemv_item* items, int32_t n_items, int32_t batch, void* d_workspace,
+                    size_t workspace_bytes, void* stream);
+
 /* Allocation-free variant of ecco_gemv.  The paper has no counterpart: this entry point exists for
  * callers that are not allowed to obtain device memory at the time they need the product -- a
  * layer plugged into an inference engine whose memory plan was fixed when the engine was built, a

@@ -33,7 +33,7 @@ ERR_DEVICE_TIMEOUT = -8
 EXPORTS = [
     "ecco_calibrate_host", "ecco_meta_create", "ecco_meta_get", "ecco_meta_free", "ecco_encode_host",
     "ecco_meta_device_bytes", "ecco_meta_serialize_device", "ecco_decompress", "ecco_decompress_batch", "ecco_gemv_workspace_bytes",
-    "ecco_gemv", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
+    "ecco_gemv", "ecco_gemv_batch_workspace_bytes", "ecco_gemv_batch", "ecco_gemv_static_ws", "ecco_attn_scores", "ecco_act_compress", "ecco_act_decompress",
     "ecco_attn_values_workspace_bytes", "ecco_attn_values", "ecco_kv_compress",
     "ecco_var_stream_bytes_bound", "ecco_var_index_bytes", "ecco_var_encode_host", "ecco_var_decompress", "ecco_error_string", "ecco_last_cuda_error", "ecco_device_status",
     "ecco_kernel_launch_count", "ecco_test_wait_timeout",
@@ -43,6 +43,12 @@ EXPORTS = [
 class DecompressItem(C.Structure):
     """ecco_decompress_item of include/ecco.h."""
     _fields_ = [("d_meta", C.c_void_p), ("d_blocks", C.c_void_p), ("n_groups", C.c_uint64), ("d_out_fp16", C.c_void_p)]
+
+
+class GemvItem(C.Structure):
+    """ecco_gemv_item of include/ecco.h."""
+    _fields_ = [("d_meta", C.c_void_p), ("d_blocks", C.c_void_p), ("n_out", C.c_int32), ("k", C.c_int32),
+                ("d_x_fp16", C.c_void_p), ("d_y", C.c_void_p)]
 
 
 class EccoError(RuntimeError):
@@ -96,6 +102,9 @@ def lib():
         L.ecco_gemv_workspace_bytes.restype = sz
         L.ecco_gemv.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, sz, vp]
         L.ecco_gemv_static_ws.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+        L.ecco_gemv_batch_workspace_bytes.argtypes = [C.POINTER(GemvItem), i32, i32]
+        L.ecco_gemv_batch_workspace_bytes.restype = sz
+        L.ecco_gemv_batch.argtypes = [C.POINTER(GemvItem), i32, i32, vp, sz, vp]
         L.ecco_attn_scores.argtypes = [vp, vp, i32, i32, i32, i32, vp, C.c_float, vp, vp]
         L.ecco_attn_values_workspace_bytes.argtypes = [i32, i32, i32, i32]
         L.ecco_attn_values_workspace_bytes.restype = sz
@@ -277,6 +286,28 @@ def ecco_gemv(d_meta, d_blocks, n_out: int, k: int, d_x_fp16, batch: int, d_y, d
     _check(lib().ecco_gemv(_ptr(d_meta), _ptr(d_blocks), n_out, k, _ptr(d_x_fp16), batch, _ptr(d_y),
                            _ptr(d_workspace) if d_workspace is not None else None, workspace_bytes, _stream(stream)),
            "ecco_gemv")
+
+
+def _gemv_items(items):
+    arr = (GemvItem * max(len(items), 1))()
+    for i, (d_meta, d_blocks, n_out, k, d_x, d_y) in enumerate(items):
+        arr[i].d_meta, arr[i].d_blocks, arr[i].n_out, arr[i].k = _ptr(d_meta), _ptr(d_blocks), n_out, k
+        arr[i].d_x_fp16, arr[i].d_y = _ptr(d_x), _ptr(d_y)
+    return arr
+
+
+def ecco_gemv_batch_workspace_bytes(items, batch: int) -> int:
+    """items: sequence of (d_meta, d_blocks, n_out, k, d_x_fp16, d_y) (pointers may be None here)."""
+    arr = (GemvItem * max(len(items), 1))()
+    for i, it in enumerate(items):
+        arr[i].n_out, arr[i].k = it[2], it[3]
+    return int(lib().ecco_gemv_batch_workspace_bytes(arr, len(items), batch))
+
+
+def ecco_gemv_batch(items, batch: int, d_workspace, workspace_bytes: int, stream=None) -> None:
+    """items: sequence of (d_meta, d_blocks, n_out, k, d_x_fp16, d_y); one call for all of them (see include/ecco.h)."""
+    _check(lib().ecco_gemv_batch(_gemv_items(items), len(items), batch, _ptr(d_workspace) if d_workspace is not None else None,
+                                 workspace_bytes, _stream(stream)), "ecco_gemv_batch")
 
 
 STATIC_WORKSPACE_BYTES = 4 << 20

@@ -123,44 +123,44 @@ __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* 
     }
 }
 
-// K2m: y[b][n] = sum_k W~[n][k] x[b][k] for 3..8 rows of x.  Units, ownership and the slot-and-ticket
-// reduction are those of the per-warp kernel (unit = 32 rows x one k-block).
+// K2m: y[b][n] = sum_k W~[n][k] x[b][k] for 3..8 rows of x.  Units (over all matrices of the call), ownership and the
+// slot-and-ticket reduction are those of the per-warp kernel (unit = 32 rows x one k-block).
 template <int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
-ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                     const __half* d_x, int batch, float* __restrict__ d_y, float* __restrict__ d_partial,
+ecco_gemv_mma_kernel(const __grid_constant__ GemvBatch batch, int n_cols, float* __restrict__ d_partial,
                      unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     release_dependents();
+    const uint8_t* d_meta = batch.job[0].meta;
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
     const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
     uint32_t stage;
     const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
 
     const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
-    const int tiles = (n_out + 31) / 32;
-    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    const int64_t U = batch.units;
     const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
-    const int k = kblocks * kGroup;
-    auto block_ptr = [&](int64_t u) {
-        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);
-        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
-    };
     issue_tables(tb, d_meta);
+    if (!same_tables(batch, tb)) return;                   // images are host-written: readable before the wait
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
-    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
+    GemvPos pos = {0, 0, 0};
+    if (u0 < u1) { pos = gemv_pos_of(batch, u0); prefetch_block_l2(gemv_block_ptr(batch, pos, lane)); }
     if (!wait_tables(tb)) return;
-    const float T = tb.T;
+    if (u0 >= u1) return;
 
     float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
     // C fragment element (mt, i): row = 16 mt + lane/4 + 8 (i >= 2), column b = (lane%4)*2 + (i & 1)
-    auto flush = [&](int tile) {
-        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
-        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
-        float* mine = d_partial + static_cast<size_t>(wg + tile) * 8 * 32;
+    auto flush = [&](int jf, int tile) {
+        const GemvJob& jb = batch.job[jf];
+        const int n_out = jb.n_out, kblocks = jb.kblocks, gtile = jb.tile_first + tile;
+        float* d_y = jb.y;
+        const int64_t g0 = jb.unit_first + static_cast<int64_t>(tile) * kblocks;
+        const int w_lo = unit_owner(U, W, g0);
+        const int w_hi = unit_owner(U, W, g0 + kblocks - 1);
+        float* mine = d_partial + static_cast<size_t>(wg + gtile) * 8 * 32;
         if (w_lo != w_hi) {
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
@@ -170,7 +170,7 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
             __threadfence();
             __syncwarp();
             unsigned int t = 0;
-            if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+            if (lane == 0) t = atomicAdd(&d_tickets[gtile], 1u);
             t = __shfl_sync(0xffffffffu, t, 0);
             if (t != static_cast<unsigned int>(w_hi - w_lo)) return;
             __threadfence();
@@ -184,32 +184,38 @@ ecco_gemv_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restri
                 float sum = acc[mt][i];
                 if (w_lo != w_hi) {                        // slots in warp order, whatever the arrival order
                     sum = 0.0f;
-                    for (int ww = w_lo; ww <= w_hi; ++ww) sum += __ldcg(d_partial + (static_cast<size_t>(ww + tile) * 8 + b) * 32 + r);
+                    for (int ww = w_lo; ww <= w_hi; ++ww) sum += __ldcg(d_partial + (static_cast<size_t>(ww + gtile) * 8 + b) * 32 + r);
                 }
-                if (row < n_out && b < batch) d_y[static_cast<size_t>(b) * n_out + row] = sum;
+                if (row < n_out && b < n_cols) d_y[static_cast<size_t>(b) * n_out + row] = sum;
             }
-        if (w_lo != w_hi && lane == 0) d_tickets[tile] = 0;
+        if (w_lo != w_hi && lane == 0) d_tickets[gtile] = 0;
     };
 
-    int cur_tile = static_cast<int>(u0 / kblocks);
+    int cur_j = pos.j, cur_tile = pos.tile;
+    float T = __ldg(&reinterpret_cast<const DevHeader*>(batch.job[pos.j].meta)->T);
     for (int64_t u = u0; u < u1; ++u) {
-        const int tile = static_cast<int>(u / kblocks);
-        if (tile != cur_tile) {
-            flush(cur_tile);
+        const GemvJob& jb = batch.job[pos.j];
+        const int tile = pos.tile;
+        if (pos.j != cur_j || tile != cur_tile) {
+            flush(cur_j, cur_tile);
 #pragma unroll
             for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) acc[mt][i] = 0.0f;
+            if (pos.j != cur_j) T = __ldg(&reinterpret_cast<const DevHeader*>(jb.meta)->T);
+            cur_j = pos.j;
             cur_tile = tile;
         }
         Block cur;                                         // fetched now, prefetched into L2 one unit earlier (see the scalar kernels)
-        ldg_block(cur, block_ptr(u));
-        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
-        const __half* xk = d_x + static_cast<int>(u % kblocks) * kGroup;
-        row_dot_mma(cur, tb, ws, stage, T, tile * 32 + lane < n_out,
-                    [&](uint32_t (&v)[16]) { load_vfrag(v, xk, static_cast<size_t>(k), batch); }, acc);
+        ldg_block(cur, gemv_block_ptr(batch, pos, lane));
+        const __half* xk = jb.x + pos.kb * kGroup;
+        const size_t k = static_cast<size_t>(jb.kblocks) * kGroup;
+        const bool valid = tile * 32 + lane < jb.n_out;
+        if (u + 1 < u1) { pos = gemv_pos_next(batch, pos); prefetch_block_l2(gemv_block_ptr(batch, pos, lane)); }
+        row_dot_mma(cur, tb, ws, stage, T, valid,
+                    [&](uint32_t (&v)[16]) { load_vfrag(v, xk, k, n_cols); }, acc);
     }
-    if (u0 < u1) flush(cur_tile);
+    flush(cur_j, cur_tile);
 }
 
 // K3m: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for 3..8 query heads per KV head.

@@ -122,54 +122,110 @@ __device__ __forceinline__ WarpSmem fused_warp_smem(const Tables& tb, uint32_t n
     return ws;
 }
 
+// One call of the fused GEMV may cover several matrices (ecco_gemv_batch): the units of all of them form one unit
+// space, dealt out to the working warps as one, so that a group of small matrices pays one launch, one table fetch and
+// one tail.  All matrices of a call share the decode tables (equal table hash; only the exponent differs).
+constexpr int kMaxGemvJobs = 8;
+struct GemvJob {
+    const uint8_t* meta;       // metadata image of this matrix (its exponent factor T is read from here)
+    const uint8_t* blocks;
+    const __half* x;           // [kV or batch][k]
+    float* y;                  // [batch][n_out]
+    int32_t n_out, kblocks;
+    int32_t tile_first;        // first 32-row tile of this matrix in the call's tile space (tickets and slots)
+    int32_t reserved;
+    int64_t unit_first;        // first unit of this matrix in the call's unit space
+};
+struct GemvBatch {
+    int32_t n, reserved;
+    int64_t units;             // of all matrices
+    GemvJob job[kMaxGemvJobs];
+};
+// true (uniformly over the grid) if every matrix of the call carries the tables of the first
+__device__ __forceinline__ bool same_tables(const GemvBatch& batch, const Tables& tb)
+{
+    bool same = true;
+    for (int t = 1; t < batch.n; ++t) {
+        const DevHeader* hd = reinterpret_cast<const DevHeader*>(batch.job[t].meta);
+        same = same && __ldg(&hd->hash_lo) == tb.hash_lo && __ldg(&hd->hash_hi) == tb.hash_hi;
+    }
+    if (!same && threadIdx.x == 0) atomicExch(&g_device_status, ECCO_ERR_INVALID_ARG);
+    return same;
+}
+
+// Where a unit sits: matrix, 32-row tile and k-block.  Units are visited in order, so the position is advanced by one
+// instead of being divided out of the unit number every time.
+struct GemvPos { int j, tile, kb; };
+__device__ __forceinline__ GemvPos gemv_pos_of(const GemvBatch& batch, int64_t u)
+{
+    GemvPos p = {0, 0, 0};
+    while (p.j + 1 < batch.n && u >= batch.job[p.j + 1].unit_first) ++p.j;
+    const int64_t lu = u - batch.job[p.j].unit_first;
+    p.tile = static_cast<int>(lu / batch.job[p.j].kblocks);
+    p.kb = static_cast<int>(lu % batch.job[p.j].kblocks);
+    return p;
+}
+__device__ __forceinline__ GemvPos gemv_pos_next(const GemvBatch& batch, GemvPos p)
+{
+    if (++p.kb == batch.job[p.j].kblocks) {
+        p.kb = 0;
+        if (++p.tile == (batch.job[p.j].n_out + 31) / 32) { p.tile = 0; ++p.j; }
+    }
+    return p;
+}
+__device__ __forceinline__ const uint8_t* gemv_block_ptr(const GemvBatch& batch, const GemvPos& p, int lane)
+{
+    const GemvJob& jb = batch.job[p.j];
+    const int row = min(p.tile * 32 + lane, jb.n_out - 1);                         // rows past the end: repeat the last
+    return jb.blocks + (static_cast<uint64_t>(row) * jb.kblocks + p.kb) * kBlockBytes;
+}
+
 // K2 for one or two rows of x: the slice is small enough (512 B or 1 KB) for every warp to keep
 // its own, so warps never meet at a barrier.  A work unit is (32 consecutive rows, one k-block),
-// numbered row-tile major; every working warp owns a contiguous run of units and keeps its rows'
-// partial sums in registers along k.  When a row tile is shared by several warps each writes its
+// numbered matrix by matrix, row-tile major; every working warp owns a contiguous run of units and keeps its
+// rows' partial sums in registers along k.  When a row tile is shared by several warps each writes its
 // partial sums to its own workspace slot (slot = global warp id + row tile: unique along the
 // staircase of (warp, tile) pairs) and the last to arrive (ticket counter) adds the slots in warp
 // order: the result does not depend on scheduling.  Workspace: partial[slot][kV][32] floats, then
 // one ticket per 32-row tile.
 template <int kV, int kMaxWarps>
 __global__ void __launch_bounds__(kMaxWarps * 32, 1)
-ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restrict__ d_blocks, int n_out, int kblocks,
-                      const __half* d_x, float* __restrict__ d_y, float* __restrict__ d_partial,
-                      unsigned int* __restrict__ d_tickets)
+ecco_gemv_warp_kernel(const __grid_constant__ GemvBatch batch, float* __restrict__ d_partial, unsigned int* __restrict__ d_tickets)
 {
     extern __shared__ __align__(1024) uint8_t smem[];
     constexpr uint32_t kXsBytes = kGroup * kV * 4;
     release_dependents();
+    const uint8_t* d_meta = batch.job[0].meta;
     const Tables tb = plan_tables(smem_u32(smem), d_meta, kFusedPairs);
     const int nw = static_cast<int>(warps_that_fit(tb, kFusedWarpBytes + kXsBytes));
     const WarpSmem ws = fused_warp_smem(tb, nw);
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     const uint32_t xs = tb.warp_base + nw * kFusedWarpBytes + warp * kXsBytes;   // this warp's slice
 
-    // W working warps (chosen by the host so that they all get the same number of units, and never
-    // more than there are units); warp ids interleave over the CTAs; the other warps idle
+    // W working warps (chosen so that they all get the same number of units, and never more than there are
+    // units); warp ids interleave over the CTAs; the other warps idle
     const int wg = warp < nw ? warp * static_cast<int>(gridDim.x) + static_cast<int>(blockIdx.x) : INT_MAX;
-    const int tiles = (n_out + 31) / 32;
-    const int64_t U = static_cast<int64_t>(tiles) * kblocks;
+    const int64_t U = batch.units;
     const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
-    const int k = kblocks * kGroup;
-    auto block_ptr = [&](int64_t u) {
-        const int row = min(static_cast<int>(u / kblocks) * 32 + lane, n_out - 1);     // rows past the end: repeat the last
-        return d_blocks + (static_cast<uint64_t>(row) * kblocks + static_cast<int>(u % kblocks)) * kBlockBytes;
-    };
     issue_tables(tb, d_meta);
+    if (!same_tables(batch, tb)) return;                   // images are host-written: readable before the wait
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
-    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
+    GemvPos pos = {0, 0, 0};
+    if (u0 < u1) { pos = gemv_pos_of(batch, u0); prefetch_block_l2(gemv_block_ptr(batch, pos, lane)); }
     if (!wait_tables(tb)) return;
-    const float T = tb.T;
 
     Accum<kV> acc;
     acc.clear();
-    auto flush = [&](int tile) {
+    auto flush = [&](int jf, int tile) {
+        const GemvJob& jb = batch.job[jf];
+        const int n_out = jb.n_out, kblocks = jb.kblocks, gtile = jb.tile_first + tile;
+        float* d_y = jb.y;
         const int row = tile * 32 + lane;
         const bool row_ok = row < n_out;
-        const int w_lo = unit_owner(U, W, static_cast<int64_t>(tile) * kblocks);
-        const int w_hi = unit_owner(U, W, static_cast<int64_t>(tile + 1) * kblocks - 1);
+        const int64_t g0 = jb.unit_first + static_cast<int64_t>(tile) * kblocks;
+        const int w_lo = unit_owner(U, W, g0);
+        const int w_hi = unit_owner(U, W, g0 + kblocks - 1);
         if (w_lo == w_hi) {
             if (row_ok) {
 #pragma unroll
@@ -177,13 +233,13 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
             }
             return;
         }
-        float* mine = d_partial + static_cast<size_t>(wg + tile) * kV * 32;
+        float* mine = d_partial + static_cast<size_t>(wg + gtile) * kV * 32;
 #pragma unroll
         for (int b = 0; b < kV; ++b) mine[b * 32 + lane] = acc.a[b];
         __threadfence();
         __syncwarp();
         unsigned int t = 0;
-        if (lane == 0) t = atomicAdd(&d_tickets[tile], 1u);
+        if (lane == 0) t = atomicAdd(&d_tickets[gtile], 1u);
         t = __shfl_sync(0xffffffffu, t, 0);
         if (t == static_cast<unsigned int>(w_hi - w_lo)) {  // last of the warps that share this tile
             __threadfence();
@@ -192,7 +248,7 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
                 for (int b = 0; b < kV; ++b) {
                     // slots are added in warp order whatever the arrival order; loads go out thirty-two at a time (a
                     // 4096-wide row is 32 k-blocks: one round trip to L2 instead of two at the end of the kernel)
-                    const float* slot = d_partial + (static_cast<size_t>(w_lo + tile) * kV + b) * 32 + lane;
+                    const float* slot = d_partial + (static_cast<size_t>(w_lo + gtile) * kV + b) * 32 + lane;
                     float sum = 0.0f;
                     int ww = w_lo;
                     for (; ww + 32 <= w_hi + 1; ww += 32, slot += 32 * kV * 32) {
@@ -213,23 +269,31 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
                     d_y[static_cast<size_t>(b) * n_out + row] = sum;
                 }
             }
-            if (lane == 0) d_tickets[tile] = 0;
+            if (lane == 0) d_tickets[gtile] = 0;
         }
     };
 
     // x for a unit is fetched one unit ahead, like the block
     uint2 xraw[kV];
-    auto load_x = [&](int64_t u) {
-        const int kb = static_cast<int>(u % kblocks);
+    auto load_x = [&](const GemvPos& p) {
+        const GemvJob& jb = batch.job[p.j];
+        const size_t k = static_cast<size_t>(jb.kblocks) * kGroup;
 #pragma unroll
         for (int b = 0; b < kV; ++b)
-            xraw[b] = __ldcg(reinterpret_cast<const uint2*>(d_x + static_cast<size_t>(b) * k + kb * kGroup + lane * 4));
+            xraw[b] = __ldcg(reinterpret_cast<const uint2*>(jb.x + static_cast<size_t>(b) * k + p.kb * kGroup + lane * 4));
     };
-    if (u0 < u1) load_x(u0);
-    int cur_tile = static_cast<int>(u0 / kblocks);
+    if (u0 >= u1) return;
+    load_x(pos);
+    int cur_j = pos.j, cur_tile = pos.tile;
+    float T = __ldg(&reinterpret_cast<const DevHeader*>(batch.job[pos.j].meta)->T);
     for (int64_t u = u0; u < u1; ++u) {
-        const int tile = static_cast<int>(u / kblocks);
-        if (tile != cur_tile) { flush(cur_tile); acc.clear(); cur_tile = tile; }
+        if (pos.j != cur_j || pos.tile != cur_tile) {
+            flush(cur_j, cur_tile);
+            acc.clear();
+            if (pos.j != cur_j) T = __ldg(&reinterpret_cast<const DevHeader*>(batch.job[pos.j].meta)->T);
+            cur_j = pos.j;
+            cur_tile = pos.tile;
+        }
         // this warp's slice: lane l converts x[b][kb*128 + 4l .. 4l+3] to fp32, layout xs[i][b]
         __syncwarp();
         {
@@ -250,11 +314,15 @@ ecco_gemv_warp_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __restr
         // the block is fetched when its turn comes (it was prefetched into L2 one unit earlier): holding the next
         // one in sixteen registers through a whole group costs more in resident warps than the fetch costs here
         Block cur;
-        ldg_block(cur, block_ptr(u));
-        if (u + 1 < u1) { prefetch_block_l2(block_ptr(u + 1)); load_x(u + 1); }
+        ldg_block(cur, gemv_block_ptr(batch, pos, lane));
+        if (u + 1 < u1) {
+            pos = gemv_pos_next(batch, pos);
+            prefetch_block_l2(gemv_block_ptr(batch, pos, lane));
+            load_x(pos);
+        }
         fused_group<kV>(cur, tb, ws, T, xs, acc);
     }
-    if (u0 < u1) flush(cur_tile);
+    flush(cur_j, cur_tile);
 }
 
 // K3: scores[b][hq][t] = scale * q[b][hq] . K~[b][hq / q_per_kv][t] for one or two query heads per KV head.

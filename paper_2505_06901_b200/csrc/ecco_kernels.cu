@@ -240,50 +240,89 @@ extern "C" size_t ecco_gemv_workspace_bytes(int32_t n_out, int32_t k, int32_t ba
 {
     if (n_out <= 0 || k <= 0 || k % kGroup || batch < 1 || batch > ECCO_MAX_BATCH) return 0;
     // sized for the largest plan any supported device can ask for (at most 256 persistent CTAs)
-    const GemvPlan p = pad_v(batch) <= 2 ? gemv_warp_plan(n_out, k / kGroup, pad_v(batch), 256) : gemv_mma_plan(n_out, k / kGroup, 256);
+    const int row_tiles = (n_out + 31) / 32;
+    const GemvPlan p = gemv_plan_for(static_cast<int64_t>(row_tiles) * (k / kGroup), row_tiles, pad_v(batch), 256);
     return p.partial_bytes + p.ticket_bytes;
 }
 
+// the matrices of one call with their places in the call's unit and tile spaces
+struct GemvCall {
+    GemvBatch b;
+    int row_tiles;
+};
+static void gemv_call_begin(GemvCall* c)
+{
+    std::memset(c, 0, sizeof *c);
+}
+static void gemv_call_add(GemvCall* c, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks, const void* d_x, float* d_y)
+{
+    GemvJob& j = c->b.job[c->b.n++];
+    j.meta = static_cast<const uint8_t*>(d_meta);
+    j.blocks = d_blocks;
+    j.x = static_cast<const __half*>(d_x);
+    j.y = d_y;
+    j.n_out = n_out;
+    j.kblocks = kblocks;
+    j.tile_first = c->row_tiles;
+    j.unit_first = c->b.units;
+    const int tiles = (n_out + 31) / 32;
+    c->row_tiles += tiles;
+    c->b.units += static_cast<int64_t>(tiles) * kblocks;
+}
+
 // three to eight rows of x: the tensor-core kernel
-static int launch_gemv_mma(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
-                           const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+static int launch_gemv_mma_call(const DeviceInfo& di, const GemvCall& c, int batch, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     auto kernel = ecco_gemv_mma_kernel<kMmaWarps>;
     static thread_local bool configured[64] = {};
     int rc = want_all_smem(kernel, &configured[di.device]);
     if (rc) return rc;
-    const GemvPlan p = gemv_mma_plan(n_out, kblocks, di.sms < 256 ? di.sms : 256);
+    const GemvPlan p = gemv_plan_for(c.b.units, c.row_tiles, 8, di.sms < 256 ? di.sms : 256);
     if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
     rc = zero_tickets(tickets, p.ticket_bytes, stream);
     if (rc) return rc;
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kMmaWarps * 32), kSmemCtaBytes, stream,
-                             static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), batch, d_y,
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kMmaWarps * 32), kSmemCtaBytes, stream, c.b, batch,
                              partial, tickets);
+}
+static int launch_gemv_mma(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
+                           const void* d_x, int batch, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+{
+    GemvCall c;
+    gemv_call_begin(&c);
+    gemv_call_add(&c, d_meta, d_blocks, n_out, kblocks, d_x, d_y);
+    return launch_gemv_mma_call(di, c, batch, d_ws, ws_bytes, stream);
 }
 
 // one or two rows of x (batch == kV): the per-warp kernel
 template <int kV>
-static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
-                            const void* d_x, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+static int launch_gemv_warp_call(const DeviceInfo& di, const GemvCall& c, void* d_ws, size_t ws_bytes, cudaStream_t stream)
 {
     constexpr int kFusedWarps = gemv_warp_warps(kV);
     auto kernel = ecco_gemv_warp_kernel<kV, kFusedWarps>;
     static thread_local bool configured[64] = {};
     int rc = want_all_smem(kernel, &configured[di.device]);
     if (rc) return rc;
-    const GemvPlan p = gemv_warp_plan(n_out, kblocks, kV, di.sms < 256 ? di.sms : 256);
+    const GemvPlan p = gemv_plan_for(c.b.units, c.row_tiles, kV, di.sms < 256 ? di.sms : 256);
     if (!d_ws || !aligned16(d_ws)) return d_ws ? ECCO_ERR_ALIGNMENT : ECCO_ERR_WORKSPACE;
     if (ws_bytes < p.partial_bytes + p.ticket_bytes) return ECCO_ERR_WORKSPACE;
     float* partial = static_cast<float*>(d_ws);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(static_cast<uint8_t*>(d_ws) + p.partial_bytes);
     rc = zero_tickets(tickets, p.ticket_bytes, stream);
     if (rc) return rc;
-    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kFusedWarps * 32), kSmemCtaBytes, stream,
-                             static_cast<const uint8_t*>(d_meta), d_blocks, n_out, kblocks, static_cast<const __half*>(d_x), d_y, partial,
-                             tickets);
+    return launch_overlapped(kernel, static_cast<unsigned>(p.grid), static_cast<unsigned>(kFusedWarps * 32), kSmemCtaBytes, stream, c.b,
+                             partial, tickets);
+}
+template <int kV>
+static int launch_gemv_warp(const DeviceInfo& di, const void* d_meta, const uint8_t* d_blocks, int n_out, int kblocks,
+                            const void* d_x, float* d_y, void* d_ws, size_t ws_bytes, cudaStream_t stream)
+{
+    GemvCall c;
+    gemv_call_begin(&c);
+    gemv_call_add(&c, d_meta, d_blocks, n_out, kblocks, d_x, d_y);
+    return launch_gemv_warp_call<kV>(di, c, d_ws, ws_bytes, stream);
 }
 
 extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_out, int32_t k, const void* d_x,
@@ -301,6 +340,58 @@ extern "C" int ecco_gemv(const void* d_meta, const uint8_t* d_blocks, int32_t n_
         case 1: return launch_gemv_warp<1>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
         case 2: return launch_gemv_warp<2>(di, d_meta, d_blocks, n_out, kblocks, d_x, d_y, d_workspace, workspace_bytes, s);
         default: return launch_gemv_mma(di, d_meta, d_blocks, n_out, kblocks, d_x, batch, d_y, d_workspace, workspace_bytes, s);
+    }
+}
+
+// several matrices in one call: one unit space, one launch
+static int check_gemv_items(const ecco_gemv_item* items, int32_t n_items, int32_t batch)
+{
+    if (!items || n_items < 1 || n_items > ECCO_MAX_GEMV_ITEMS || batch < 1 || batch > ECCO_MAX_BATCH) return ECCO_ERR_INVALID_ARG;
+    for (int i = 0; i < n_items; ++i) {
+        const ecco_gemv_item& it = items[i];
+        if (!it.d_meta || !it.d_blocks || !it.d_x_fp16 || !it.d_y) return ECCO_ERR_INVALID_ARG;
+        if (it.n_out <= 0 || it.k <= 0 || it.k % kGroup) return ECCO_ERR_INVALID_ARG;
+        if (!aligned16(it.d_meta) || !aligned16(it.d_blocks) || !aligned16(it.d_x_fp16) || !aligned16(it.d_y)) return ECCO_ERR_ALIGNMENT;
+    }
+    return ECCO_OK;
+}
+static void gemv_call_from_items(GemvCall* c, const ecco_gemv_item* items, int32_t n_items)
+{
+    gemv_call_begin(c);
+    for (int i = 0; i < n_items; ++i)
+        gemv_call_add(c, items[i].d_meta, items[i].d_blocks, items[i].n_out, items[i].k / kGroup, items[i].d_x_fp16, items[i].d_y);
+}
+
+extern "C" size_t ecco_gemv_batch_workspace_bytes(const ecco_gemv_item* items, int32_t n_items, int32_t batch)
+{
+    if (!items || n_items < 1 || n_items > ECCO_MAX_GEMV_ITEMS || batch < 1 || batch > ECCO_MAX_BATCH) return 0;
+    int64_t units = 0, tiles = 0;
+    for (int i = 0; i < n_items; ++i) {
+        if (items[i].n_out <= 0 || items[i].k <= 0 || items[i].k % kGroup) return 0;
+        const int64_t t = (items[i].n_out + 31) / 32;
+        tiles += t;
+        units += t * (items[i].k / kGroup);
+    }
+    if (tiles > INT32_MAX) return 0;
+    const GemvPlan p = gemv_plan_for(units, static_cast<int>(tiles), pad_v(batch), 256);
+    return p.partial_bytes + p.ticket_bytes;
+}
+
+extern "C" int ecco_gemv_batch(const ecco_gemv_item* items, int32_t n_items, int32_t batch, void* d_workspace,
+                               size_t workspace_bytes, void* stream)
+{
+    int rc = check_gemv_items(items, n_items, batch);
+    if (rc) return rc;
+    DeviceInfo di;
+    rc = device_info(&di);
+    if (rc) return rc;
+    GemvCall c;
+    gemv_call_from_items(&c, items, n_items);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (pad_v(batch)) {
+        case 1: return launch_gemv_warp_call<1>(di, c, d_workspace, workspace_bytes, s);
+        case 2: return launch_gemv_warp_call<2>(di, c, d_workspace, workspace_bytes, s);
+        default: return launch_gemv_mma_call(di, c, batch, d_workspace, workspace_bytes, s);
     }
 }
 
@@ -324,7 +415,8 @@ extern "C" int ecco_gemv_static_ws(const void* d_meta, const uint8_t* d_blocks, 
     const int kblocks = k / kGroup, vpad = pad_v(batch);
     // refuse, before any launch, a shape whose plan does not fit the fixed array
     const int ctas = di.sms < 256 ? di.sms : 256;
-    const GemvPlan p = vpad <= 2 ? gemv_warp_plan(n_out, kblocks, vpad, ctas) : gemv_mma_plan(n_out, kblocks, ctas);
+    const int row_tiles = (n_out + 31) / 32;
+    const GemvPlan p = gemv_plan_for(static_cast<int64_t>(row_tiles) * kblocks, row_tiles, vpad, ctas);
     if (p.partial_bytes + p.ticket_bytes > ECCO_STATIC_WORKSPACE_BYTES) return ECCO_ERR_WORKSPACE;
     // one-time set-up per device (the current device is di.device): resolve the array's address
     static std::mutex mu;

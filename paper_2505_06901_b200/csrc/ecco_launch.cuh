@@ -94,33 +94,26 @@ constexpr int gemv_warp_warps(int) { return 28; }
 
 struct GemvPlan { int row_tiles, grid; size_t partial_bytes, ticket_bytes; };
 
-// plan of the per-warp GEMV (one or two rows of x)
-GemvPlan gemv_warp_plan(int n_out, int kblocks, int vpad, int ctas_max)
+// plan of a fused GEMV call over `units` units in `row_tiles` 32-row tiles (all matrices of the call together):
+// persistent CTAs of `warps` warps, one slot of cols x 32 partial sums per (warp, tile) step of the staircase, one
+// ticket per tile
+inline GemvPlan gemv_plan(int64_t units, int row_tiles, int warps, int cols, int ctas_max)
 {
     GemvPlan p;
-    p.row_tiles = (n_out + 31) / 32;
-    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
-    const int64_t ctas = (units + gemv_warp_warps(vpad) - 1) / gemv_warp_warps(vpad);
+    p.row_tiles = row_tiles;
+    const int64_t ctas = (units + warps - 1) / warps;
     p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
-    p.partial_bytes = static_cast<size_t>(p.grid * gemv_warp_warps(vpad) + p.row_tiles) * vpad * 32 * sizeof(float);
-    p.partial_bytes = (p.partial_bytes + 255) & ~static_cast<size_t>(255);
-    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
+    p.partial_bytes = (static_cast<size_t>(p.grid * warps + row_tiles) * cols * 32 * sizeof(float) + 255) & ~static_cast<size_t>(255);
+    p.ticket_bytes = (static_cast<size_t>(row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
     return p;
 }
 
 constexpr int kMmaWarps = 24;
 
-// plan of the tensor-core GEMV (3..8 rows of x): units and slots as in the per-warp kernel, eight columns
-GemvPlan gemv_mma_plan(int n_out, int kblocks, int ctas_max)
+// the per-warp kernel (one or two rows of x: vpad columns) or the tensor-core kernel (3..8 rows: eight columns)
+inline GemvPlan gemv_plan_for(int64_t units, int row_tiles, int vpad, int ctas_max)
 {
-    GemvPlan p;
-    p.row_tiles = (n_out + 31) / 32;
-    const int64_t units = static_cast<int64_t>(p.row_tiles) * kblocks;
-    const int64_t ctas = (units + kMmaWarps - 1) / kMmaWarps;
-    p.grid = static_cast<int>(ctas < ctas_max ? ctas : ctas_max);
-    p.partial_bytes = (static_cast<size_t>(p.grid * kMmaWarps + p.row_tiles) * 8 * 32 * sizeof(float) + 255) & ~static_cast<size_t>(255);
-    p.ticket_bytes = (static_cast<size_t>(p.row_tiles) * sizeof(unsigned int) + 255) & ~static_cast<size_t>(255);
-    return p;
+    return vpad <= 2 ? gemv_plan(units, row_tiles, gemv_warp_warps(vpad), vpad, ctas_max) : gemv_plan(units, row_tiles, kMmaWarps, 8, ctas_max);
 }
 
 inline int pad_v(int v) { return v <= 1 ? 1 : v <= 2 ? 2 : v <= 4 ? 4 : 8; }

@@ -327,6 +327,72 @@ def test_gemv_handles_pads_clips_and_garbage(B, eo, cfg1_small, synth):
     check_fused(got, ref, refabs, "gemv b2 skewed code")
 
 
+@pytest.mark.parametrize("batch", [1, 2, 3, 8])
+def test_gemv_batch_gives_every_item_what_gemv_gives(B, eo, cfg1_small, synth, batch):
+    """Several matrices in one call (shapes that differ in rows and in k, a ragged row count, a one-row matrix, a shared
+    x, per-tensor exponents that differ): every item within the fused tolerance of the oracle and, to rounding, what
+    ecco_gemv gives on it alone (the k range of a row is cut into partial sums at other places, so the last bits may
+    differ); the same call twice gives the same bits.  Eight items is the most one call takes."""
+    meta = cfg1_small["meta"]
+    shapes = [(256, 1024), (100, 1024), (513, 512), (64, 4096), (1, 128), (2048, 128), (31, 256), (96, 1024)]
+    x_shared = synth.activations(batch, 1024, 77)
+    items, keep, want = [], [], []
+    for i, (n_out, k) in enumerate(shapes):
+        n_groups = n_out * (k // 128)
+        blocks = np.roll(np.tile(cfg1_small["blocks"], (-(-n_groups // 2048), 1)), 17 * i, axis=0)[:n_groups]
+        om = meta.copy()
+        om.e = meta.e + (i % 3) - 1                           # same tables, another exponent
+        x = x_shared if k == 1024 else synth.activations(batch, k, 80 + i)
+        d_meta, d_blocks, d_x = B.meta_to_device(lib_meta_from_oracle(B, om)), dev(blocks), dev(x)
+        d_y = torch.full((batch, n_out), float("nan"), dtype=torch.float32, device="cuda")
+        items.append((d_meta, d_blocks, n_out, k, d_x, d_y))
+        keep.append((om, blocks, x))
+        wsb = B.ecco_gemv_workspace_bytes(n_out, k, batch)
+        ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+        d_alone = torch.empty((batch, n_out), dtype=torch.float32, device="cuda")
+        B.ecco_gemv(d_meta, d_blocks, n_out, k, d_x, batch, d_alone, ws, wsb)
+        want.append(d_alone)
+    wsb = B.ecco_gemv_batch_workspace_bytes(items, batch)
+    assert wsb > 0
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    first = None
+    for _ in range(2):                                        # the second call starts from a used workspace
+        B.ecco_gemv_batch(items, batch, ws, wsb)
+        torch.cuda.synchronize()
+        assert B.ecco_device_status() == 0
+        outs = [it[5].cpu().numpy() for it in items]
+        if first is not None:
+            assert all(np.array_equal(a, b) for a, b in zip(first, outs))
+        first = outs
+    for (om, blocks, x), it, alone, got in zip(keep, items, want, first):
+        ref, refabs = eo.gemv(om, blocks, it[2], it[3], x, batch)
+        check_fused(got.astype(np.float64), ref, refabs, f"gemv batch-call b{batch}")
+        assert np.all(np.abs(got - alone.cpu().numpy()) <= 1e-5 * refabs + 1e-30)
+    # argument errors stop the call before anything runs; too small a workspace is refused
+    with pytest.raises(B.EccoError) as ei:
+        B.ecco_gemv_batch(items + items[:1], batch, ws, wsb)
+    assert ei.value.code == B.ERR_INVALID_ARG
+    with pytest.raises(B.EccoError) as ei:
+        B.ecco_gemv_batch(items, batch, ws, wsb - 256)
+    assert ei.value.code == B.ERR_WORKSPACE
+    # an item with other decode tables is detected on the device: nothing is written, the status says so
+    S, e, pat, cb, kp = lib_meta_from_oracle(B, meta).tables()
+    cb = cb.copy()
+    cb[0, 0] = cb[0, 0][::-1]
+    other = B.meta_to_device(B.ecco_meta_create(S, e, pat, cb, kp))
+    canary = torch.full((batch, shapes[0][0]), 7.0, dtype=torch.float32, device="cuda")
+    bad = [(items[0][0], items[0][1], items[0][2], items[0][3], items[0][4], canary),
+           (other, items[1][1], items[1][2], items[1][3], items[1][4], items[1][5])]
+    B.ecco_gemv_batch(bad, batch, ws, wsb)
+    torch.cuda.synchronize()
+    assert B.ecco_device_status() == B.ERR_INVALID_ARG
+    assert B.ecco_device_status() == 0                        # reported once
+    assert bool((canary == 7.0).all())
+    B.ecco_gemv_batch(items, batch, ws, wsb)                  # and the next good call is unaffected
+    torch.cuda.synchronize()
+    assert np.array_equal(items[0][5].cpu().numpy(), first[0])
+
+
 def test_gemv_workspace_errors(B, cfg1_small, synth):
     lm = lib_meta_from_oracle(B, cfg1_small["meta"])
     d_meta, d_blocks = B.meta_to_device(lm), dev(cfg1_small["blocks"])
