@@ -238,24 +238,25 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
     const int64_t U = static_cast<int64_t>(heads) * tiles;
     const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
-    auto block_ptr = [&](int64_t u) {
-        const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
-        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    auto block_ptr = [&](int bh, int tile) {
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + min(tile * 32 + lane, seq - 1)) * kBlockBytes;
     };
+    int nbh = static_cast<int>(u0 / tiles), ntile = static_cast<int>(u0 % tiles);     // advanced by one per unit
     issue_tables(tb, d_meta);
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
-    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
+    if (u0 < u1) prefetch_block_l2(block_ptr(nbh, ntile));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
     uint32_t vfrag[16];
     int cur_bh = -1;
     for (int64_t u = u0; u < u1; ++u) {
-        const int bh = static_cast<int>(u / tiles), t0 = static_cast<int>(u % tiles) * 32;
+        const int bh = nbh, t0 = ntile * 32;
         if (bh != cur_bh) { load_vfrag(vfrag, d_q + static_cast<size_t>(bh) * q_per_kv * kGroup, kGroup, q_per_kv); cur_bh = bh; }
         Block cur;
-        ldg_block(cur, block_ptr(u));
-        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
+        ldg_block(cur, block_ptr(nbh, ntile));
+        if (++ntile == tiles) { ntile = 0; ++nbh; }
+        if (u + 1 < u1) prefetch_block_l2(block_ptr(nbh, ntile));
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
         row_dot_mma(cur, tb, ws, stage, T, t0 + lane < seq,
                     [&](uint32_t (&v)[16]) {

@@ -349,20 +349,21 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const int64_t U = static_cast<int64_t>(heads) * tiles;
     const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
-    // lanes past the end of the sequence decode its last token again and store nothing
-    auto block_ptr = [&](int64_t u) {
-        const int bh = static_cast<int>(u / tiles), t = min(static_cast<int>(u % tiles) * 32 + lane, seq - 1);
-        return d_kblocks + (static_cast<uint64_t>(bh) * seq + t) * kBlockBytes;
+    // lanes past the end of the sequence decode its last token again and store nothing; (head, tile) of a unit is
+    // advanced by one per unit instead of divided out of the unit number
+    auto block_ptr = [&](int bh, int tile) {
+        return d_kblocks + (static_cast<uint64_t>(bh) * seq + min(tile * 32 + lane, seq - 1)) * kBlockBytes;
     };
+    int bh = static_cast<int>(u0 / tiles), tile = static_cast<int>(u0 % tiles);
     issue_tables(tb, d_meta);
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
-    if (u0 < u1) prefetch_block_l2(block_ptr(u0));
+    if (u0 < u1) prefetch_block_l2(block_ptr(bh, tile));
     if (!wait_tables(tb)) return;
     const float T = tb.T;
 
     int cur_bh = -1;
     for (int64_t u = u0; u < u1; ++u) {
-        const int bh = static_cast<int>(u / tiles), t = static_cast<int>(u % tiles) * 32 + lane;
+        const int t = tile * 32 + lane;
         if (bh != cur_bh) {
             // lane l stages q[b][h*q_per_kv + r][4l .. 4l+3] * scale as fp32, layout xs[d][r]; heads beyond q_per_kv are zero
             float v[kV][4];
@@ -385,15 +386,17 @@ ecco_attn_scores_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
             cur_bh = bh;
         }
         Block cur;
-        ldg_block(cur, block_ptr(u));
-        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
+        ldg_block(cur, block_ptr(bh, tile));
+        const int out_bh = bh;
+        if (++tile == tiles) { tile = 0; ++bh; }
+        if (u + 1 < u1) prefetch_block_l2(block_ptr(bh, tile));
         Accum<kV> acc;
         acc.clear();
         fused_group<kV>(cur, tb, ws, T, xs, acc);
         if (t < seq) {
 #pragma unroll
             for (int r = 0; r < kV; ++r)
-                if (r < q_per_kv) d_scores[(static_cast<size_t>(bh) * q_per_kv + r) * seq + t] = acc.a[r];
+                if (r < q_per_kv) d_scores[(static_cast<size_t>(out_bh) * q_per_kv + r) * seq + t] = acc.a[r];
         }
     }
 }
