@@ -54,6 +54,9 @@ def parse_args(argv=None):
                          "variable-length container on the cfg2 gate/up/down matrices")
     ap.add_argument("--decompress-calls", choices=["batch", "single"], default="batch",
                     help="decompress segment: one ecco_decompress_batch call over the step's tensors (default) or one ecco_decompress per tensor")
+    ap.add_argument("--gemv-calls", choices=["grouped", "single"], default="grouped",
+                    help="GEMV segments: one ecco_gemv_batch call per group of matrices that a decoder layer can issue together "
+                         "(q+k+v, o, gate+up, down; default) or one ecco_gemv call per matrix")
     ap.add_argument("--only", default="", help="comma list of segments to run: decompress,gemv1,gemv8,attn (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-other-configs", action="store_true", help="skip the cfg5 / cfg4 measurements that follow the headline step")
@@ -259,7 +262,7 @@ def cpu_baseline(layer, c: int, kv_tensor=None):
 WORKLOADS = {
     "cfg2": dict(label="cfg2 llama2-7b decoder layer (q,k,v,o 4096x4096; gate,up 11008x4096; down 4096x11008; 1,581,056 groups) "
                        "+ cfg3 K and V caches [8][32][4096][128]",
-                 step="decompress of the 7 matrices (one ecco_decompress_batch call), gemv batch 1 x7, gemv batch 8 x7, attn_scores x1 (K cache), attn_values x1 (V cache); --only kvcomp times ecco_kv_compress over the whole K cache",
+                 step="decompress of the 7 matrices (one ecco_decompress_batch call), gemv batch 1 over the 7 matrices (four ecco_gemv_batch calls: q+k+v, o, gate+up, down), the same at batch 8, attn_scores x1 (K cache), attn_values x1 (V cache); --only kvcomp times ecco_kv_compress over the whole K cache",
                  l2="inputs larger than L2: each step streams 96.5 MiB of blocks and writes 386 MiB before any tensor is revisited"),
     "cfg4": dict(label="cfg4 llama-70b-shaped MLP weights (gate, up 28672x8192; down 8192x28672; 5,505,024 groups)",
                  step="decompress x3, gemv batch 1 x3; plus a decompress sweep over 64 MiB .. 4 GiB streams (stream_sweep)",
@@ -368,10 +371,36 @@ def run_ours(args, workload=None, extras=True):
         else:
             seg_decompress_single()
 
-    def seg_gemv(b):
+    def seg_gemv_single(b):
         for d in mats:
             B.ecco_gemv(d["meta"], d["blocks"], d["n_out"], d["k"], d["x1" if b == 1 else "x8"], b, d["y1" if b == 1 else "y8"],
                         d["ws"], d["wsb"], stream)
+
+    # The products of a decoder layer that do not depend on each other go out in one ecco_gemv_batch call: q, k and v
+    # read the same activations, and so do gate and up; o and down each wait for what comes before them.
+    by_name = {d["t"].name: d for d in mats}
+    gemv_groups = [[by_name[n] for n in grp if n in by_name] for grp in (("q", "k", "v"), ("o",), ("gate", "up"), ("down",))]
+    gemv_groups = [g for g in gemv_groups if g]
+    if sum(len(g) for g in gemv_groups) != len(mats):
+        gemv_groups = [[d] for d in mats]
+    grouped = {}
+    for b in (1, 8):
+        if b == 8 and not need8:
+            continue
+        calls = []
+        for g in gemv_groups:
+            xk, yk = ("x1", "y1") if b == 1 else ("x8", "y8")
+            items = [(d["meta"], d["blocks"], d["n_out"], d["k"], g[0][xk], d[yk]) for d in g]      # one x for the group
+            nb = B.ecco_gemv_batch_workspace_bytes(items, b)
+            calls.append((items, torch.empty(nb, dtype=torch.uint8, device="cuda"), nb))
+        grouped[b] = calls
+
+    def seg_gemv(b):
+        if args.gemv_calls == "grouped":
+            for items, ws, nb in grouped[b]:
+                B.ecco_gemv_batch(items, b, ws, nb, stream)
+        else:
+            seg_gemv_single(b)
 
     def seg_attn():
         if kv is not None:
@@ -529,6 +558,25 @@ def run_ours(args, workload=None, extras=True):
         (sms_,) = distutil.max_over_ranks([s0.elapsed_time(s1)], dist, "cuda")
         single_us = sms_ * 1e3 / reps
 
+    # the GEMVs through one ecco_gemv call per matrix, for the record
+    gemv_single_us = {}
+    if args.gemv_calls == "grouped" and extras:
+        for b, seg in ((1, "gemv1"), (8, "gemv8")):
+            if seg not in segs or not mats:
+                continue
+            for _ in range(3):
+                seg_gemv_single(b)
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(3, min(args.steps, 20))
+            barrier()
+            s0.record(stream)
+            for _ in range(reps):
+                seg_gemv_single(b)
+            s1.record(stream)
+            barrier()
+            (gms_,) = distutil.max_over_ranks([s0.elapsed_time(s1)], dist, "cuda")
+            gemv_single_us[f"batch{b}"] = gms_ * 1e3 / reps
+
     peak, peak_kind = measured_peaks()
     n_launch = max(1, -(-len(dec) // 8) if args.decompress_calls == "batch" else len(dec))
     avg_launch_s = dec_ms / 1e3 / (args.steps * n_launch) if dec_ms > 0 else float("nan")
@@ -597,6 +645,9 @@ def run_ours(args, workload=None, extras=True):
                                  "attn_values": av_ms / args.steps * 1e3, "kv_compress": kc_ms / args.steps * 1e3},
         "decompress_one_call_per_tensor_us": single_us,
         "gemv_us_per_layer_batch1": g1_ms / args.steps * 1e3 if wname == "cfg2" else None,
+        "gemv_calls": ("ecco_gemv_batch per group: " + ", ".join("+".join(d["t"].name for d in g) for g in gemv_groups))
+                      if args.gemv_calls == "grouped" else "one ecco_gemv per matrix",
+        "gemv_one_call_per_matrix_us": gemv_single_us or None,
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "roofline": {"kernel": "ecco_decompress_tma_kernel", "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": traffic,
