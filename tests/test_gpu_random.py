@@ -119,6 +119,32 @@ def test_random_configurations_match_the_oracle(B, eo, synth):
             ok, worst = fused_ok(y.cpu().numpy().astype(np.float64), ref, refabs, "random gemv")
             if not ok:
                 failures.append((it, "gemv", batch, worst))
+        # several matrices in one ecco_gemv_batch call: the same blocks cut into up to four matrices of random shapes
+        if n >= 33 and it % 2 == 0:
+            batch = int(rng.integers(1, 9))
+            parts, at = [], 0
+            while at < n and len(parts) < 4:
+                kbp = int(rng.choice([1, 2, 4]))
+                rows_p = int(rng.integers(1, max(2, (n - at) // kbp // 2 + 2)))
+                if rows_p * kbp > n - at or (at * 64) % 16:
+                    break
+                parts.append((at, rows_p, kbp))
+                at += rows_p * kbp
+            items, checks = [], []
+            for (g0, rows_p, kbp) in parts:
+                xx = synth.activations(batch, kbp * 128, 31 + it + g0)
+                yb = torch.full((batch, rows_p), float("nan"), dtype=torch.float32, device="cuda")
+                items.append((d_meta, d_b[g0:], rows_p, kbp * 128, dev(xx), yb))
+                checks.append((blocks[g0: g0 + rows_p * kbp], rows_p, kbp * 128, xx, yb))
+            if items:
+                wsb = B.ecco_gemv_batch_workspace_bytes(items, batch)
+                ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+                B.ecco_gemv_batch(items, batch, ws, wsb)
+                for blk, rows_p, kk, xx, yb in checks:
+                    ref, refabs = eo.gemv(m, blk, rows_p, kk, xx, batch)
+                    ok, worst = fused_ok(yb.cpu().numpy().astype(np.float64), ref, refabs, "random gemv batch")
+                    if not ok:
+                        failures.append((it, "gemv_batch", batch, rows_p, kk, worst))
         # attention scores and attention output on a [batch][heads][seq] view
         heads = int(rng.choice([1, 2, 3]))
         seq = n // heads
