@@ -17,23 +17,54 @@ namespace {
 // split into an fp16 head and an fp16 remainder (two MMAs) so that its rounding does not show.
 // The result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------------
+// Row maximum and reciprocal of the row's sum of exponentials, one CTA per row.  One pass: every thread keeps a running
+// (maximum, sum of exp(x - maximum)) over its elements, rescaling the sum when the maximum grows; the pairs are then
+// merged over the warp and over the warps in a fixed order.
+__device__ __forceinline__ void softmax_merge(float& m, float& s, float m2, float s2)
+{
+    const float mn = fmaxf(m, m2);
+    // an empty side has maximum -inf and sum 0: its factor is exp(-inf) = 0 unless both are empty (avoid -inf - -inf)
+    const float f1 = m == mn ? 1.0f : expf(m - mn), f2 = m2 == mn ? 1.0f : expf(m2 - mn);
+    s = s * f1 + s2 * f2;
+    m = mn;
+}
 __global__ void __launch_bounds__(256)
 ecco_softmax_stats_kernel(const float* d_scores, int rows, int seq, float2* d_stats)
 {
-    const int row = static_cast<int>(blockIdx.x) * 8 + static_cast<int>(threadIdx.x >> 5), lane = static_cast<int>(threadIdx.x & 31u);
-    dependency_wait();                                     // the scores may come from the previous kernel of the stream
+    __shared__ float2 part[8];
+    const int row = static_cast<int>(blockIdx.x), tid = static_cast<int>(threadIdx.x), lane = tid & 31, warp = tid >> 5;
     release_dependents();
+    dependency_wait();                                     // the scores may come from the previous kernel of the stream
     if (row >= rows) return;
     const float* s = d_scores + static_cast<size_t>(row) * seq;
-    float mx = -INFINITY;
-    for (int t = lane; t < seq; t += 32) mx = fmaxf(mx, __ldcg(s + t));    // the scores may come from the previous kernel: coherent loads
+    float mx = -INFINITY, sum = 0.0f;
+    auto take = [&](float x) {
+        if (x > mx) { sum = sum * expf(mx - x) + 1.0f; mx = x; }      // exp(-inf) = 0 on the first element
+        else if (x != -INFINITY) sum += expf(x - mx);                  // a masked score (-inf) adds nothing, also before any finite one
+    };
+    // the scores may come from the previous kernel: coherent loads; 16-byte loads where the row allows it
+    if ((reinterpret_cast<uintptr_t>(s) & 15u) == 0) {
+        const float4* s4 = reinterpret_cast<const float4*>(s);
+        for (int i = tid; i < seq / 4; i += 256) {
+            const float4 v = __ldcg(s4 + i);
+            take(v.x); take(v.y); take(v.z); take(v.w);
+        }
+        for (int t = (seq & ~3) + tid; t < seq; t += 256) take(__ldcg(s + t));
+    } else {
+        for (int t = tid; t < seq; t += 256) take(__ldcg(s + t));
+    }
 #pragma unroll
-    for (int o = 16; o; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    float sum = 0.0f;
-    for (int t = lane; t < seq; t += 32) sum += expf(__ldcg(s + t) - mx);
-#pragma unroll
-    for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-    if (lane == 0) d_stats[row] = make_float2(mx, 1.0f / sum);
+    for (int o = 16; o; o >>= 1) {
+        const float m2 = __shfl_xor_sync(0xffffffffu, mx, o), s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+        softmax_merge(mx, sum, m2, s2);
+    }
+    if (lane == 0) part[warp] = make_float2(mx, sum);
+    __syncthreads();
+    if (tid == 0) {
+        float m = part[0].x, t = part[0].y;
+        for (int w = 1; w < 8; ++w) softmax_merge(m, t, part[w].x, part[w].y);
+        d_stats[row] = make_float2(m, 1.0f / t);
+    }
 }
 
 __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&a)[4], uint32_t addr)

@@ -562,7 +562,7 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     rc = zero_tickets(tickets, p.ticket_bytes, s);
     if (rc) return rc;
     const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
-    rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>((rows + 7) / 8), 256u, 0, s, d_scores, rows, seq, stats);
+    rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>(rows), 256u, 0, s, d_scores, rows, seq, stats);
     if (rc) return rc;
     return p.warps == kAvWarpsWide
                ? launch_attn_values<kAvWarpsWide>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s)

@@ -714,6 +714,29 @@ def test_attn_values_keeps_small_probabilities(B, eo, kv_small, synth, qpk):
         assert np.all(err[0, 1] <= 2e-5 * refabs[0, 1])    # evenly spread weights: far inside the bound
 
 
+@pytest.mark.parametrize("seq", [301, 4100])
+def test_attn_values_with_masked_scores(B, eo, kv_small, synth, seq):
+    """Scores of -inf (masked tokens) carry no weight: at the start of a row (before the row statistics have seen any
+    finite score), in the middle, in whole 16-byte chunks and at a ragged end; rows of odd length start at addresses
+    that are not 16-byte aligned."""
+    meta = kv_small["meta"]
+    heads, qpk = 2, 3
+    n = heads * seq
+    blocks = np.tile(kv_small["blocks"], (-(-n // 2048), 1))[:n]
+    rng = np.random.Generator(np.random.PCG64(5 + seq))
+    scores = (rng.standard_normal((1, heads * qpk, seq)) * 2.0).astype(np.float32)
+    scores[0, :, :9] = -np.inf
+    scores[0, 1, 100:164] = -np.inf
+    scores[0, 2, -3:] = -np.inf
+    scores[0, 3, rng.random(seq) < 0.5] = -np.inf
+    scores[0, 4, 1:] = -np.inf
+    scores[0, 4, 0] = 0.5                                  # a single live token, first in the row
+    got = gpu_attn_values(B, lib_meta_from_oracle(B, meta), blocks, 1, heads, seq, qpk, scores)
+    ref, refabs = eo.attn_values(meta, blocks, 1, heads, seq, qpk, scores)
+    assert np.isfinite(ref).all()
+    check_fused(got, ref, refabs, "values masked")
+
+
 # ------------------------------------------------------------------ online KV compressor
 def gpu_kv_compress(B, lmeta, x):
     n = x.size // 128
