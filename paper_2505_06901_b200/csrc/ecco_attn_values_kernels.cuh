@@ -45,7 +45,16 @@ ecco_softmax_stats_kernel(const float* d_scores, int rows, int seq, float2* d_st
     // the scores may come from the previous kernel: coherent loads; 16-byte loads where the row allows it
     if ((reinterpret_cast<uintptr_t>(s) & 15u) == 0) {
         const float4* s4 = reinterpret_cast<const float4*>(s);
-        for (int i = tid; i < seq / 4; i += 256) {
+        const int n4 = seq / 4;
+        int i = tid;
+        for (; i + 3 * 256 < n4; i += 4 * 256) {           // four loads in flight per thread
+            const float4 a = __ldcg(s4 + i), b = __ldcg(s4 + i + 256), c = __ldcg(s4 + i + 512), d = __ldcg(s4 + i + 768);
+            take(a.x); take(a.y); take(a.z); take(a.w);
+            take(b.x); take(b.y); take(b.z); take(b.w);
+            take(c.x); take(c.y); take(c.z); take(c.w);
+            take(d.x); take(d.y); take(d.z); take(d.w);
+        }
+        for (; i < n4; i += 256) {
             const float4 v = __ldcg(s4 + i);
             take(v.x); take(v.y); take(v.z); take(v.w);
         }
