@@ -8,14 +8,12 @@ namespace {
 // K5: attention output over a compressed V cache (Eq. 3: softmax(QK^T / sqrt(d_k)) V).
 // out[b][hq][d] = sum_t p[b][hq][t] * V~[b][hq / q_per_kv][t][d] with p = softmax_t(scores).
 // A thread owns one token (one group) as in K3, but here the sum runs over tokens, i.e. across
-// lanes.  Pass 1 runs the serial Huffman chain and keeps only the 4-bit indices (syms[16][32]);
-// by then the end bit, hence the outliers, are known.  Pass 2 walks the eight 16-dim chunks: map
-// the indices through the lane's table, stage them in a [32 tokens][16 dims] fp16 tile (same
-// swizzle as the decompress staging tile), overwrite the outliers of that chunk in the tile, and
-// contract the tile on the tensor cores: (V tile)^T [16 dims x 32 tokens] x P^T [32 tokens x 8
-// heads] with mma.m16n8k16, fp32 accumulators (4 registers per 16 dims, 32 for the 128 dims).  p is
-// split into an fp16 head and an fp16 remainder (two MMAs) so that its rounding does not show.
-// The result does not depend on scheduling.
+// lanes.  The group is decoded once, values and all, into eight [32 tokens][16 dims] fp16 tiles of the
+// warp (the swizzle of the decompress staging tile); when the end bit is known the outliers are
+// written over their positions in the tiles; then every tile is contracted on the tensor cores:
+// (V tile)^T [16 dims x 32 tokens] x P^T [32 tokens x 8 heads] with mma.m16n8k16, fp32 accumulators
+// (4 registers per 16 dims, 32 for the 128 dims).  p is split into an fp16 head and an fp16 remainder
+// (two MMAs) so that its rounding does not show.  The result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------------
 // Row maximum and reciprocal of the row's sum of exponentials, one CTA per row.  One pass: every thread keeps a running
 // (maximum, sum of exp(x - maximum)) over its elements, rescaling the sum when the maximum grows; the pairs are then
@@ -89,7 +87,9 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-constexpr uint32_t kAvWarpBytes = kBitsBytes + kTabBytes + kSymsBytes + 1024;   // + the [32][16] fp16 tile
+constexpr uint32_t kAvValueBytes = 8 * 1024;                                // eight [32 tokens][16 dims] fp16 tiles
+constexpr uint32_t kAvWarpBytes = kTabBytes / 2 + kAvValueBytes + kBitsBytes;   // half a value table (two warps share one), tiles, bit stream
+constexpr uint32_t kAvSlots = 4;                                            // reduction slots: see flush
 
 constexpr float kProbScale = 32768.0f, kProbUnscale = 1.0f / 32768.0f;      // powers of two: exact
 
@@ -104,25 +104,26 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     const int tid = static_cast<int>(threadIdx.x), n_threads = static_cast<int>(blockDim.x);
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar fused kernels
-    constexpr uint32_t kSlotFloats = kGroup * 8, kSlots = (kMaxWarps + 1) / 2;      // reduction slots: see flush
-    const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kSlots * kSlotFloats * sizeof(float));
+    constexpr uint32_t kSlotFloats = kGroup * 8;
+    const uint32_t nw = warps_that_fit(tb, kAvWarpBytes, kTabBytes / 2 + kAvSlots * kSlotFloats * sizeof(float));
     const int kTokens = static_cast<int>(nw) * 32;         // tokens per unit: one per thread of the working warps
     const bool working = warp < nw;
     // small CTA-wide words in the misc area at the start of shared memory (the barrier word is its first)
     unsigned int& ticket = *reinterpret_cast<unsigned int*>(smem + 32);
     float2* stats_s = reinterpret_cast<float2*>(smem + 64);
     WarpSmem ws;
-    ws.tab = tb.warp_base + warp * kTabBytes + lane * 4;
-    const uint32_t stage = tb.warp_base + nw * kTabBytes + warp * (1024 + kBitsBytes + kSymsBytes);
-    ws.bits = stage + 1024 + lane * 4;
-    ws.syms = ws.bits + kBitsBytes;
+    ws.tab = tab_column<kTabHalf>(tb.warp_base, warp, lane);
+    const uint32_t per_warp = tb.warp_base + tab_bytes<kTabHalf>(nw);
+    const uint32_t vals = per_warp + warp * (kAvValueBytes + kBitsBytes);      // this warp's eight tiles
+    ws.bits = vals + kAvValueBytes + lane * 4;
+    ws.syms = 0;
     if (working) {
         sts_u32(ws.bits + 16 * 128, 0u);
         sts_u32(ws.bits + 17 * 128, 0u);
     }
     const uint32_t swz = ((lane >> 2) & 1u) << 4;
-    const uint32_t my_row = stage + lane * 32;
-    float* out_s = reinterpret_cast<float*>(smem + (tb.warp_base - tb.base) + nw * kAvWarpBytes);    // slots of [128 dims][8 heads]
+    const uint32_t my_row = vals + lane * 32;
+    float* out_s = reinterpret_cast<float*>(smem + (per_warp - tb.base) + nw * (kAvValueBytes + kBitsBytes));    // slots of [128 dims][8 heads]
 
     const int chunks = (seq + kTokens - 1) / kTokens;
     const int64_t U = static_cast<int64_t>(heads) * chunks;
@@ -150,30 +151,30 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     };
     clear_acc();
 
-    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in a fixed order (the first half of
-    // the warps write a slot each, the second half add theirs to the slot of the warp half the count below, then
-    // the slots are added in slot order), then either store (this CTA owns the whole head) or hand a partial to the
-    // slot-and-ticket reduction
+    // all tokens of head bh seen by this CTA are in acc: reduce over the warps in a fixed order (in rounds of
+    // kAvSlots warps: warp w adds its sums to slot w mod kAvSlots, the first round by plain stores; then the slots are
+    // added in slot order), then either store (this CTA owns the whole head) or hand a partial to the slot-and-ticket
+    // reduction
     auto flush = [&](int bh) {
-        const uint32_t half = (nw + 1u) >> 1;
-        auto my_elements = [&](float* slot, bool add) {
+        for (uint32_t first = 0; first < nw; first += kAvSlots) {
+            if (warp >= first && warp < first + kAvSlots && warp < nw) {
+                float* slot = out_s + (warp - first) * kSlotFloats;
 #pragma unroll
-            for (int ch = 0; ch < 8; ++ch)
+                for (int ch = 0; ch < 8; ++ch)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
-                    const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
-                    const float v = acc[ch][j] * kProbUnscale;
-                    slot[dim * 8 + head] = add ? slot[dim * 8 + head] + v : v;
-                }
-        };
-        if (warp < half) my_elements(out_s + warp * kSlotFloats, false);
-        __syncthreads();
-        if (warp >= half && warp < nw) my_elements(out_s + (warp - half) * kSlotFloats, true);
-        __syncthreads();
+                    for (int j = 0; j < 4; ++j) {
+                        const int dim = ch * 16 + static_cast<int>(lane >> 2) + (j >= 2 ? 8 : 0);
+                        const int head = static_cast<int>(lane & 3u) * 2 + (j & 1);
+                        const float v = acc[ch][j] * kProbUnscale;
+                        slot[dim * 8 + head] = first ? slot[dim * 8 + head] + v : v;
+                    }
+            }
+            __syncthreads();
+        }
+        const uint32_t used = min(nw, kAvSlots);
         for (int i = tid; i < static_cast<int>(kSlotFloats); i += n_threads) {   // thread i keeps element i from here on
             float sum = out_s[i];
-            for (uint32_t sl = 1; sl < half; ++sl) sum += out_s[sl * kSlotFloats + i];
+            for (uint32_t sl = 1; sl < used; ++sl) sum += out_s[sl * kSlotFloats + i];
             out_s[i] = sum;
         }
         const int c_lo = unit_owner(U, G, static_cast<int64_t>(bh) * chunks);
@@ -209,7 +210,7 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
     for (int64_t u = u0; u < u1; ++u) {
         const int bh = static_cast<int>(u / chunks);
         const int tile_base = static_cast<int>(u % chunks) * kTokens + static_cast<int>(warp) * 32;
-        const int t = tile_base + static_cast<int>(lane);
+        const bool valid = tile_base + static_cast<int>(lane) < seq;
         if (bh != cur_bh) {
             if (cur_bh >= 0) { flush(cur_bh); clear_acc(); }
             if (tid < 8) stats_s[tid] = tid < q_per_kv ? __ldcg(d_stats + static_cast<size_t>(bh) * q_per_kv + tid) : make_float2(0.0f, 0.0f);
@@ -243,55 +244,45 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         Block cur;                                         // fetched now, prefetched into L2 one unit earlier
         ldg_block(cur, block_ptr(u));
         if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
-        const bool valid = t < seq;                        // lanes past the end stage zeros (their p is zero too)
-        const GroupHeader h = open_group<kTabHalfBits>(cur, tb, ws, T);
-        // pass 1: the serial Huffman chain, indices only (8 per word into syms[16][32])
-        RankPacker rk;
-        int n_fit = kGroup;
-        const uint32_t end = decode_symbols<false, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t, uint32_t, bool alive, uint32_t pair) {
-            if (!alive) n_fit = min(n_fit, n);             // only the clip path can see alive == false
-            rk.put(n, pair, ws.syms);
+        // lanes past the end of the row decode the row's last token again (zeroed below)
+        const GroupHeader h = open_group<kTabHalf>(cur, tb, ws, T);
+        __syncwarp();                                      // the tiles of the previous token tile have been read
+        uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree, kTabHalf>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t) {
+            const int slot = (n & 15) >> 1;                // clipped positions arrive as +0
+            if (n & 1) r[slot] = __byte_perm(r[slot], v, 0x5410); else r[slot] = v;
+            if ((n & 15) == 15) {
+                const uint32_t row = my_row + (n >> 4) * 1024;
+                sts_v4(row + swz, r[0], r[1], r[2], r[3]);
+                sts_v4(row + (swz ^ 16u), r[4], r[5], r[6], r[7]);
+            }
         });
-        if (!valid) n_fit = 0;
-        // outliers of a complete group: which 16-dim chunks they fall into
-        const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
-        uint64_t pads_lo = 0, pads_hi = 0;                 // 16 bits per chunk: which pads fall into it
+        // outliers of a complete group replace the mapped values in the tiles (ascending: a later pad overrides an earlier one)
+        const int n_pad = end ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
         for (int j = 0; j < n_pad; ++j) {
-            const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
-            const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
-            if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+            const uint32_t f = read_pad(ws, j);
+            const uint32_t loc = f & 127u, byte = (loc & 15u) * 2;
+            asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + (loc >> 4) * 1024 + ((byte & 16u) ^ swz) + (byte & 15u)),
+                         "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
         }
-        // pass 2: per 16-dim chunk map the indices, patch the outliers in the tile, contract on the tensor cores
+        if (__any_sync(0xffffffffu, !valid)) {             // a row's ragged last tile: lanes past its end hold zeros (p is
+            if (!valid) {                                  // zero there, but a decoded value need not be finite)
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) {
+                    sts_v4(my_row + ch * 1024, 0u, 0u, 0u, 0u);
+                    sts_v4(my_row + ch * 1024 + 16, 0u, 0u, 0u, 0u);
+                }
+            }
+        }
+        __syncwarp();                                      // tiles complete
+        // per 16-dim chunk: (V tile)^T x P^T on the tensor cores
 #pragma unroll
         for (int ch = 0; ch < 8; ++ch) {
-            uint32_t r8[8];
-            const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
-            const bool whole = ch * 16 + 16 <= n_fit;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
-                uint32_t v = lds_u32(ws.tab + sym * 128);
-                if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;      // clipped positions (and lanes past the end) are +0
-                if (i & 1) r8[i >> 1] |= v << 16; else r8[i >> 1] = v;
-            }
-            __syncwarp();                                  // the previous tile has been read
-            sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
-            sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
-            uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
-            while (mine) {                                 // ascending: a later pad overrides an earlier one
-                const int j = __ffs(static_cast<int>(mine)) - 1;
-                mine &= mine - 1;
-                const uint32_t f = read_pad(ws, j);
-                const uint32_t byte = (f & 15u) * 2;
-                asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
-                             "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
-            }
-            __syncwarp();                                  // tile complete
             uint32_t a[2][4];
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {
                 const uint32_t tok = (lane >> 4) * 8 + (lane & 7u) + 16 * ks, half = (lane >> 3) & 1u;
-                ldmatrix_x4_trans(a[ks], stage + tok * 32 + ((half ^ ((tok >> 2) & 1u)) << 4));
+                ldmatrix_x4_trans(a[ks], vals + ch * 1024 + tok * 32 + ((half ^ ((tok >> 2) & 1u)) << 4));
             }
 #pragma unroll
             for (int ks = 0; ks < 2; ++ks) {

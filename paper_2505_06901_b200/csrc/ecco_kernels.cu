@@ -491,16 +491,9 @@ extern "C" int ecco_attn_scores(const void* d_meta, const uint8_t* d_kblocks, in
 // ecco_attn_values
 // ---------------------------------------------------------------------------------------------
 namespace {
-// Warps per CTA = tokens per unit / 32.  Twenty warps keep more decode chains in flight (96 registers per thread
-// instead of 120), sixteen make a unit of 512 tokens, which divides the usual sequence lengths: the choice goes by
-// how much of the last unit of a row is padding (cfg-5 cache, 32768 tokens: 889 us with 16, 821 us with 20; cfg-3
-// cache, 4096 tokens: 210 us with 16, 223 us with 20).
-constexpr int kAvWarpsNarrow = 16, kAvWarpsWide = 20;
-inline int av_warps(int seq)
-{
-    auto fill = [&](int w) { const int t = 32 * w; return static_cast<double>(seq) / (static_cast<double>((seq + t - 1) / t) * t); };
-    return fill(kAvWarpsWide) * 1.08 > fill(kAvWarpsNarrow) ? kAvWarpsWide : kAvWarpsNarrow;
-}
+// A CTA of ecco_attn_values: sixteen warps is what finds room beside the tables (11.25 KB of shared memory per warp)
+constexpr int kAvWarps = 16;
+inline int av_warps(int) { return kAvWarps; }
 struct AvPlan { int grid, warps; size_t stats_bytes, partial_bytes, ticket_bytes; };
 AvPlan av_plan(int batch, int n_kv_heads, int seq, int q_per_kv, int ctas_max)
 {
@@ -564,9 +557,7 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
     rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>(rows), 256u, 0, s, d_scores, rows, seq, stats);
     if (rc) return rc;
-    return p.warps == kAvWarpsWide
-               ? launch_attn_values<kAvWarpsWide>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s)
-               : launch_attn_values<kAvWarpsNarrow>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s);
+    return launch_attn_values<kAvWarps>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s);
 }
 
 
