@@ -7,25 +7,24 @@ namespace {
 // ---------------------------------------------------------------------------------------------
 // K2m / K3m: the fused consumers for 3 to 8 dot products per group (rows of x, query heads) on the
 // tensor cores.  With eight products per weight the scalar path spends four shared-memory
-// wavefronts and eight FMAs per symbol on the vector operand alone.  Here a group is decoded in
-// two passes as in K5 (indices first; then per 16 values: map, stage a [32 rows][16 k] fp16 tile,
-// patch its outliers) and each tile is contracted against the fp16 vector fragments, which stay
-// in registers for the whole group: C[32 rows][8] += tile[32 x 16] * V[16 x 8], two
-// mma.m16n8k16 per tile, fp32 accumulate (fp16 x fp16 products are exact in fp32).  A warp is
-// independent of the others: no vector slice in shared memory, no block barrier.
+// wavefronts and eight FMAs per symbol on the vector operand alone.  Here a group is decoded once,
+// values and all, into eight [32 rows][16 k] fp16 tiles of the warp (as in K5); when the end bit is
+// known the outliers are written over their positions; then each tile is contracted against the fp16
+// vector fragments: C[32 rows][8] += tile[32 x 16] * V[16 x 8], two mma.m16n8k16 per tile, fp32
+// accumulate (fp16 x fp16 products are exact in fp32).  A warp is independent of the others: no
+// vector slice in shared memory, no block barrier.
 // ---------------------------------------------------------------------------------------------
-// The [32][16] fp16 staging tile of the second pass (1 KB) lives in rows 0..7 of the warp's bit-stream array: the
-// first pass has consumed them by then, the outlier fields sit in rows 8..15.
-constexpr uint32_t kMmaWarpBytes = kBitsBytes + kTabBytes + kSymsBytes;
-// value tables first (each at a multiple of 2 KB), then per warp the bit-stream array and the decoded ranks
-__device__ __forceinline__ WarpSmem mma_warp_smem(const Tables& tb, uint32_t nw, uint32_t* stage)
+constexpr uint32_t kMmaValueBytes = 8 * 1024;                               // eight [32 rows][16 k] fp16 tiles
+constexpr uint32_t kMmaWarpBytes = kTabBytes / 2 + kMmaValueBytes + kBitsBytes;   // half a value table (two warps share one), tiles, bit stream
+// value tables first, then per warp the tiles and the bit-stream array; *vals = the warp's first tile
+__device__ __forceinline__ WarpSmem mma_warp_smem(const Tables& tb, uint32_t nw, uint32_t* vals)
 {
     const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
     WarpSmem ws;
-    ws.tab = tb.warp_base + warp * kTabBytes + lane * 4;
-    *stage = tb.warp_base + nw * kTabBytes + warp * (kBitsBytes + kSymsBytes);          // = rows 0..7 of bits
-    ws.bits = *stage + lane * 4;
-    ws.syms = ws.bits + kBitsBytes;
+    ws.tab = tab_column<kTabHalf>(tb.warp_base, warp, lane);
+    *vals = tb.warp_base + tab_bytes<kTabHalf>(nw) + warp * (kMmaValueBytes + kBitsBytes);
+    ws.bits = *vals + kMmaValueBytes + lane * 4;
+    ws.syms = 0;
     if (warp < nw) {
         sts_u32(ws.bits + 16 * 128, 0u);
         sts_u32(ws.bits + 17 * 128, 0u);
@@ -52,59 +51,43 @@ __host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i 
 __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols);
 
 template <class FetchVectors>
-__device__ __forceinline__ void row_dot_mma(const Block& blk, const Tables& tb, const WarpSmem& ws, uint32_t stage, float T,
-                                            bool valid, FetchVectors&& fetch_vectors, float (&acc)[2][4])
+__device__ __forceinline__ void row_dot_mma(const Block& blk, const Tables& tb, const WarpSmem& ws, uint32_t vals, float T,
+                                            FetchVectors&& fetch_vectors, float (&acc)[2][4])
 {
     const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = stage + lane * 32;
-    const GroupHeader h = open_group<kTabHalfBits>(blk, tb, ws, T);
-    RankPacker rk;
-    int n_fit = kGroup;
-    const uint32_t end = decode_symbols<false, 16, kBlockBits, kFusedFree>(h, ws, tb.pairs, [&](int n, uint32_t, uint32_t, bool alive, uint32_t pair) {
-        if (!alive) n_fit = min(n_fit, n);
-        rk.put(n, pair, ws.syms);
+    const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = vals + lane * 32;
+    const GroupHeader h = open_group<kTabHalf>(blk, tb, ws, T);
+    __syncwarp();                                          // the tiles of the previous group have been read
+    uint32_t r8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree, kTabHalf>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t) {
+        const int col = tile_column(n & 15);               // see load_vfrag; clipped positions arrive as +0
+        if (col & 1) r8[col >> 1] = __byte_perm(r8[col >> 1], v, 0x5410); else r8[col >> 1] = v;   // the even column of a pair comes first
+        if ((n & 15) == 15) {
+            const uint32_t row = my_row + (n >> 4) * 1024;
+            sts_v4(row + swz, r8[0], r8[1], r8[2], r8[3]);
+            sts_v4(row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
+        }
     });
     uint32_t vfrag[16];
     fetch_vectors(vfrag);
-    if (!valid) n_fit = 0;                                 // rows past the end contribute zeros
-    const int n_pad = (end && valid) ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
-    uint64_t pads_lo = 0, pads_hi = 0;                     // 16 bits per chunk: which pads fall into it
+    // outliers of a complete group replace the mapped values in the tiles (ascending: a later pad overrides an earlier
+    // one).  Rows past the end of the matrix or the sequence decode the last one again; their results are not stored.
+    const int n_pad = end ? min(kMaxPads, static_cast<int>((kBlockBits - end) / kPadBits)) : 0;
     for (int j = 0; j < n_pad; ++j) {
-        const uint32_t ch = (read_pad(ws, j) & 127u) >> 4;
-        const uint64_t bit = 1ull << ((ch & 3u) * 16 + j);
-        if (ch < 4) pads_lo |= bit; else pads_hi |= bit;
+        const uint32_t f = read_pad(ws, j);
+        const uint32_t loc = f & 127u, i = loc & 15u;
+        const uint32_t byte = (2u * (i >> 2) + (i & 1u) + 8u * ((i >> 1) & 1u)) * 2u;          // tile_column(i) * 2
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + (loc >> 4) * 1024 + ((byte & 16u) ^ swz) + (byte & 15u)),
+                     "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
     }
+    __syncwarp();                                          // tiles complete
 #pragma unroll
     for (int ch = 0; ch < 8; ++ch) {
-        uint32_t r8[8];
-        const uint32_t w0 = lds_u32(ws.syms + (2 * ch) * 128), w1 = lds_u32(ws.syms + (2 * ch + 1) * 128);
-        const bool whole = ch * 16 + 16 <= n_fit;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            const uint32_t sym = ((i < 8 ? w0 : w1) >> ((i & 7) * 4)) & 15u;
-            uint32_t v = lds_u32(ws.tab + sym * 128);
-            if (!whole) v = (ch * 16 + i < n_fit) ? v : 0u;
-            const int col = tile_column(i);                // see load_vfrag
-            if (col & 1) r8[col >> 1] |= v << 16; else r8[col >> 1] = v;
-        }
-        __syncwarp();                                      // the previous tile has been read
-        sts_v4(my_row + swz, r8[0], r8[1], r8[2], r8[3]);
-        sts_v4(my_row + (swz ^ 16u), r8[4], r8[5], r8[6], r8[7]);
-        uint32_t mine = static_cast<uint32_t>((ch < 4 ? pads_lo : pads_hi) >> ((ch & 3) * 16)) & 0xffffu;
-        while (mine) {                                     // ascending: a later pad overrides an earlier one
-            const int j = __ffs(static_cast<int>(mine)) - 1;
-            mine &= mine - 1;
-            const uint32_t f = read_pad(ws, j);
-            const uint32_t byte = static_cast<uint32_t>(tile_column(static_cast<int>(f & 15u))) * 2;
-            asm volatile("st.shared.u16 [%0], %1;" ::"r"(my_row + ((byte & 16u) ^ swz) + (byte & 15u)),
-                         "h"(static_cast<unsigned short>(f2h_bits(fp8_to_float(f >> 7) * T))) : "memory");
-        }
-        __syncwarp();                                      // tile complete
 #pragma unroll
         for (int mt = 0; mt < 2; ++mt) {
             const uint32_t row = ((lane >> 3) & 1u) * 8 + (lane & 7u) + 16 * mt, half = lane >> 4;
             uint32_t a[4];
-            ldmatrix_x4(a, stage + row * 32 + ((half ^ ((row >> 2) & 1u)) << 4));
+            ldmatrix_x4(a, vals + ch * 1024 + row * 32 + ((half ^ ((row >> 2) & 1u)) << 4));
             mma_16816(acc[mt], a, vfrag[2 * ch], vfrag[2 * ch + 1]);
         }
     }
@@ -135,7 +118,7 @@ ecco_gemv_mma_kernel(const __grid_constant__ GemvBatch batch, int n_cols, float*
     release_dependents();
     const uint8_t* d_meta = batch.job[0].meta;
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
-    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
+    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes, kTabBytes / 2));
     uint32_t stage;
     const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
 
@@ -210,10 +193,8 @@ ecco_gemv_mma_kernel(const __grid_constant__ GemvBatch batch, int n_cols, float*
         ldg_block(cur, gemv_block_ptr(batch, pos, lane));
         const __half* xk = jb.x + pos.kb * kGroup;
         const size_t k = static_cast<size_t>(jb.kblocks) * kGroup;
-        const bool valid = tile * 32 + lane < jb.n_out;
         if (u + 1 < u1) { pos = gemv_pos_next(batch, pos); prefetch_block_l2(gemv_block_ptr(batch, pos, lane)); }
-        row_dot_mma(cur, tb, ws, stage, T, valid,
-                    [&](uint32_t (&v)[16]) { load_vfrag(v, xk, k, n_cols); }, acc);
+        row_dot_mma(cur, tb, ws, stage, T, [&](uint32_t (&v)[16]) { load_vfrag(v, xk, k, n_cols); }, acc);
     }
     flush(cur_j, cur_tile);
 }
@@ -229,7 +210,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
     const int lane = static_cast<int>(threadIdx.x & 31u), warp = static_cast<int>(threadIdx.x >> 5);
     release_dependents();
     const Tables tb = plan_tables(smem_u32(smem), d_meta, false);   // one symbol per lookup: see the scalar kernels
-    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes));
+    const int nw = static_cast<int>(warps_that_fit(tb, kMmaWarpBytes, kTabBytes / 2));
     uint32_t stage;
     const WarpSmem ws = mma_warp_smem(tb, nw, &stage);
 
@@ -258,7 +239,7 @@ ecco_attn_scores_mma_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* _
         if (++ntile == tiles) { ntile = 0; ++nbh; }
         if (u + 1 < u1) prefetch_block_l2(block_ptr(nbh, ntile));
         float acc[2][4] = {{0.f, 0.f, 0.f, 0.f}, {0.f, 0.f, 0.f, 0.f}};
-        row_dot_mma(cur, tb, ws, stage, T, t0 + lane < seq,
+        row_dot_mma(cur, tb, ws, stage, T,
                     [&](uint32_t (&v)[16]) {
 #pragma unroll
                         for (int i = 0; i < 16; ++i) v[i] = vfrag[i];

@@ -108,7 +108,7 @@ inline GemvPlan gemv_plan(int64_t units, int row_tiles, int warps, int cols, int
     return p;
 }
 
-constexpr int kMmaWarps = 24;
+constexpr int kMmaWarps = 20;      // 18 find room beside the tables of a typical image (11.25 KB of shared memory per warp)
 
 // the per-warp kernel (one or two rows of x: vpad columns) or the tensor-core kernel (3..8 rows: eight columns)
 inline GemvPlan gemv_plan_for(int64_t units, int row_tiles, int vpad, int ctas_max)
