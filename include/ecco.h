@@ -186,9 +186,9 @@ int ecco_gemv_batch(const ecco_gemv_item* items, int32_t n_items, int32_t batch,
  * of ECCO_STATIC_WORKSPACE_BYTES inside the library's device image (every GPU that loads the
  * library carries it until the process exits) instead of a caller buffer.  The call allocates
  * nothing.  A shape whose plan needs more scratch than that is refused with ECCO_ERR_WORKSPACE
- * before anything is launched.  For scale, on a 148-SM part: batch 8 on an 11008 x 4096 matrix needs 3.99 MB, which
- * fits; batch 1 or 2 on the same matrix 0.6 / 1.1 MB; a matrix with more than about 12 000 output rows at batch 3..8
- * (for instance 28672 x 8192) does not fit and is refused.
+ * before anything is launched.  For scale, on a 148-SM part: batch 8 on an 11008 x 4096 matrix needs 3.38 MB, batch 1
+ * or 2 on the same matrix 0.6 / 1.1 MB, batch 8 on 28672 x 8192 3.96 MB; a matrix with more than about 36 000 output
+ * rows at batch 3..8 does not fit and is refused.
  * The first call on each device looks up the array's device address (with that device current);
  * make that first call outside any stream capture.  All calls on a device share the one array:
  * it still holds the previous call's values when the next call starts (each call clears the part

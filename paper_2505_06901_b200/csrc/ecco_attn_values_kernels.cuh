@@ -243,7 +243,13 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
         }
         Block cur;                                         // fetched now, prefetched into L2 one unit earlier
         ldg_block(cur, block_ptr(u));
-        if (u + 1 < u1) prefetch_block_l2(block_ptr(u + 1));
+        if (u + 1 < u1) {
+            prefetch_block_l2(block_ptr(u + 1));
+            // the scores of this warp's tokens in the next unit, one 128-byte line per query head: into L2 now
+            const int nbh = static_cast<int>((u + 1) / chunks), nt = static_cast<int>((u + 1) % chunks) * kTokens + static_cast<int>(warp) * 32;
+            if (static_cast<int>(lane) < q_per_kv && nt < seq)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(d_scores + (static_cast<size_t>(nbh) * q_per_kv + lane) * seq + nt));
+        }
         // lanes past the end of the row decode the row's last token again (zeroed below)
         const GroupHeader h = open_group<kTabHalf>(cur, tb, ws, T);
         __syncwarp();                                      // the tiles of the previous token tile have been read
