@@ -27,12 +27,14 @@ __device__ __forceinline__ void softmax_merge(float& m, float& s, float m2, floa
     m = mn;
 }
 __global__ void __launch_bounds__(256)
-ecco_softmax_stats_kernel(const float* d_scores, int rows, int seq, float2* d_stats)
+ecco_softmax_stats_kernel(const float* d_scores, int rows, int seq, float2* d_stats, unsigned int* d_tickets, int n_tickets)
 {
     __shared__ float2 part[8];
     const int row = static_cast<int>(blockIdx.x), tid = static_cast<int>(threadIdx.x), lane = tid & 31, warp = tid >> 5;
     release_dependents();
     dependency_wait();                                     // the scores may come from the previous kernel of the stream
+    // also clears the ticket words of the call's workspace (the previous kernel, which may have used them, is complete)
+    for (int i = row * 256 + tid; i < n_tickets; i += static_cast<int>(gridDim.x) * 256) d_tickets[i] = 0u;
     if (row >= rows) return;
     const float* s = d_scores + static_cast<size_t>(row) * seq;
     float mx = -INFINITY, sum = 0.0f;

@@ -552,10 +552,9 @@ extern "C" int ecco_attn_values(const void* d_meta, const uint8_t* d_vblocks, in
     float2* stats = reinterpret_cast<float2*>(wsb);
     float* partial = reinterpret_cast<float*>(wsb + p.stats_bytes);
     unsigned int* tickets = reinterpret_cast<unsigned int*>(wsb + p.stats_bytes + p.partial_bytes);
-    rc = zero_tickets(tickets, p.ticket_bytes, s);
-    if (rc) return rc;
     const int heads = batch * n_kv_heads, rows = heads * q_per_kv;
-    rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>(rows), 256u, 0, s, d_scores, rows, seq, stats);
+    rc = launch_overlapped(ecco_softmax_stats_kernel, static_cast<unsigned>(rows), 256u, 0, s, d_scores, rows, seq, stats, tickets,
+                           static_cast<int>(p.ticket_bytes / sizeof(unsigned int)));
     if (rc) return rc;
     return launch_attn_values<kAvWarps>(di, p, d_meta, d_vblocks, heads, seq, q_per_kv, d_scores, stats, d_out, partial, tickets, s);
 }
