@@ -473,7 +473,7 @@ __device__ __forceinline__ uint32_t decode_symbols(const GroupHeader& h, const W
     return alive ? pos : 0u;
 }
 
-// Kernels that need the decoded ranks again (outlier fix-up, second pass) keep them in syms[16][32]: position n in
+// Kernels that need the decoded ranks again (the outlier fix-up of the scalar fused kernels) keep them in syms[16][32]: position n in
 // nibble n & 7 of word n >> 3.  put() takes the sink's pair byte at even n and stores a word when it is complete
 // (n mod 8 is a compile-time constant after unrolling).
 struct RankPacker {

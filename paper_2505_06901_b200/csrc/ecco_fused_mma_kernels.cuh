@@ -45,8 +45,8 @@ __host__ __device__ constexpr int tile_column(int i) { return 2 * (i >> 2) + (i 
 
 // vfrag[2c], vfrag[2c+1]: B fragments of chunk c (tile columns (lane%4)*2 + {0,1}, and + 8), vector lane/4
 // acc[0] / acc[1]: C fragments of rows 0..15 / 16..31 of the warp's 32 groups
-// fetch_vectors(vfrag) is called between the two passes: a caller whose vectors change with every group (the GEMV)
-// loads them there, so that they do not occupy sixteen registers during the first pass; one whose vectors stay
+// fetch_vectors(vfrag) is called after the decode: a caller whose vectors change with every group (the GEMV)
+// loads them there, so that they do not occupy sixteen registers during the decode; one whose vectors stay
 // (the scores) copies them.
 __device__ __forceinline__ void load_vfrag(uint32_t (&vfrag)[16], const __half* base, size_t col_stride, int n_cols);
 

@@ -10,12 +10,15 @@
 //   tables   pattern[64][16] fp16 | ID_KP table [4096] u16 | codebook records [256] x 16 B | shape tables
 //            [n_shapes][256] u8 | pair tables, brought in by three bulk copies (cp.async.bulk + mbarrier)
 //   per warp tab[16][32]  u32   per-lane dequantised centroids in rank order (the rank of the abs-max symbol
-//                               holds the abs-max)
+//                               holds the abs-max); fp32 in the scalar fused kernels, fp16 with two warps to an
+//                               array elsewhere
 //            bits[18][32] u32   the warp's 32 blocks, word-transposed: lane L's word w at
 //                               [w][L] -> bank L whatever w is (conflict-free refills);
 //                               rows 16 and 17 stay zero (stream bits past 512 read as 0)
-//            syms[16][32] u32   (fused kernels) decoded ranks, 8 nibbles per word, for the
+//            syms[16][32] u32   (scalar fused kernels) decoded ranks, 8 nibbles per word, for the
 //                               outlier fix-up
+//            tiles              ecco_decompress: one [32 groups][16 values] fp16 staging tile for the tensor stores;
+//                               tensor-core kernels: eight of them, the whole decoded group, as MMA operands
 //
 // Layout of the sources (one translation unit; the .cuh files are included here and nowhere else):
 //   ecco_device_core.cuh            shared-memory layout, PTX helpers, table staging, the per-group decoder
