@@ -358,7 +358,7 @@ def run_ours(args, workload=None, extras=True):
             kv["out"] = torch.empty(kt.n_groups * G, dtype=torch.float16, device="cuda")
             dec.append(kv)
 
-    dec_items = [(d["meta"], d["blocks"], d["n"], d["out"]) for d in dec]
+    dec_items = B.decompress_items([(d["meta"], d["blocks"], d["n"], d["out"]) for d in dec])      # marshalled once
 
     def seg_decompress_single():
         for d in dec:
@@ -392,7 +392,7 @@ def run_ours(args, workload=None, extras=True):
             xk, yk = ("x1", "y1") if b == 1 else ("x8", "y8")
             items = [(d["meta"], d["blocks"], d["n_out"], d["k"], g[0][xk], d[yk]) for d in g]      # one x for the group
             nb = B.ecco_gemv_batch_workspace_bytes(items, b)
-            calls.append((items, torch.empty(nb, dtype=torch.uint8, device="cuda"), nb))
+            calls.append((B.gemv_items(items), torch.empty(nb, dtype=torch.uint8, device="cuda"), nb))      # marshalled once
         grouped[b] = calls
 
     def seg_gemv(b):

@@ -269,12 +269,21 @@ def ecco_decompress(d_meta, d_blocks, n_groups: int, d_out_fp16, stream=None) ->
            "ecco_decompress")
 
 
-def ecco_decompress_batch(items, stream=None) -> None:
-    """items: sequence of (d_meta, d_blocks, n_groups, d_out_fp16); one call for all of them (see include/ecco.h)."""
+def decompress_items(items):
+    """The host array ecco_decompress_batch reads, from a sequence of (d_meta, d_blocks, n_groups, d_out_fp16).  A
+    caller that issues the same batch again and again builds it once and passes it instead of the sequence."""
     arr = (DecompressItem * max(len(items), 1))()
     for i, (d_meta, d_blocks, n_groups, d_out) in enumerate(items):
         arr[i].d_meta, arr[i].d_blocks, arr[i].n_groups, arr[i].d_out_fp16 = _ptr(d_meta), _ptr(d_blocks), n_groups, _ptr(d_out)
-    _check(lib().ecco_decompress_batch(arr, len(items), _stream(stream)), "ecco_decompress_batch")
+    arr.n_items = len(items)
+    return arr
+
+
+def ecco_decompress_batch(items, stream=None) -> None:
+    """items: sequence of (d_meta, d_blocks, n_groups, d_out_fp16), or what decompress_items made of one; one call
+    for all of them (see include/ecco.h)."""
+    arr = items if isinstance(items, C.Array) else decompress_items(items)
+    _check(lib().ecco_decompress_batch(arr, arr.n_items, _stream(stream)), "ecco_decompress_batch")
 
 
 def ecco_gemv_workspace_bytes(n_out: int, k: int, batch: int) -> int:
@@ -288,11 +297,14 @@ def ecco_gemv(d_meta, d_blocks, n_out: int, k: int, d_x_fp16, batch: int, d_y, d
            "ecco_gemv")
 
 
-def _gemv_items(items):
+def gemv_items(items):
+    """The host array ecco_gemv_batch reads, from a sequence of (d_meta, d_blocks, n_out, k, d_x_fp16, d_y).  A caller
+    that issues the same group again and again builds it once and passes it instead of the sequence."""
     arr = (GemvItem * max(len(items), 1))()
     for i, (d_meta, d_blocks, n_out, k, d_x, d_y) in enumerate(items):
         arr[i].d_meta, arr[i].d_blocks, arr[i].n_out, arr[i].k = _ptr(d_meta), _ptr(d_blocks), n_out, k
         arr[i].d_x_fp16, arr[i].d_y = _ptr(d_x), _ptr(d_y)
+    arr.n_items = len(items)
     return arr
 
 
@@ -305,8 +317,10 @@ def ecco_gemv_batch_workspace_bytes(items, batch: int) -> int:
 
 
 def ecco_gemv_batch(items, batch: int, d_workspace, workspace_bytes: int, stream=None) -> None:
-    """items: sequence of (d_meta, d_blocks, n_out, k, d_x_fp16, d_y); one call for all of them (see include/ecco.h)."""
-    _check(lib().ecco_gemv_batch(_gemv_items(items), len(items), batch, _ptr(d_workspace) if d_workspace is not None else None,
+    """items: sequence of (d_meta, d_blocks, n_out, k, d_x_fp16, d_y), or what gemv_items made of one; one call for
+    all of them (see include/ecco.h)."""
+    arr = items if isinstance(items, C.Array) else gemv_items(items)
+    _check(lib().ecco_gemv_batch(arr, arr.n_items, batch, _ptr(d_workspace) if d_workspace is not None else None,
                                  workspace_bytes, _stream(stream)), "ecco_gemv_batch")
 
 
