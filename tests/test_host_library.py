@@ -43,6 +43,19 @@ def test_argument_errors_without_a_gpu(binding, cfg1_small, eo):
     assert L.ecco_attn_scores(16, 32, 1, 1, 8, 9, 64, ctypes.c_float(1.0), 128, None) == binding.ERR_INVALID_ARG
     assert L.ecco_gemv_workspace_bytes(4096, 4096, 1) >= 4096 * 4 * 32
     assert L.ecco_gemv_workspace_bytes(4096, 100, 1) == 0
+    # several matrices in one call: the same checks per item, at most eight items, all before any CUDA call
+    good = (16, 32, 100, 128, 64, 128)
+    items = lambda seq: binding.gemv_items(seq)
+    assert L.ecco_gemv_batch(items([]), 0, 1, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.ecco_gemv_batch(items([good] * 9), 9, 1, None, 0, None) == binding.ERR_INVALID_ARG
+    assert L.ecco_gemv_batch(items([good, (16, 32, 100, 100, 64, 128)]), 2, 1, None, 0, None) == binding.ERR_INVALID_ARG     # k % 128
+    assert L.ecco_gemv_batch(items([good, (16, 32 + 4, 100, 128, 64, 128)]), 2, 1, None, 0, None) == binding.ERR_ALIGNMENT   # blocks
+    assert L.ecco_gemv_batch(items([good]), 1, 9, None, 0, None) == binding.ERR_INVALID_ARG                                   # batch > 8
+    one = binding.ecco_gemv_batch_workspace_bytes([good], 3)
+    assert one == binding.ecco_gemv_workspace_bytes(100, 128, 3) > 0
+    assert binding.ecco_gemv_batch_workspace_bytes([good, (0, 0, 4096, 4096, 0, 0)], 3) > one
+    assert binding.ecco_gemv_batch_workspace_bytes([good] * 9, 1) == 0
+    assert binding.ecco_gemv_batch_workspace_bytes([(0, 0, 100, 100, 0, 0)], 1) == 0
     # bad metadata tables are refused
     pat, cb, kp = cfg1_small["meta"].patterns(), cfg1_small["meta"].cb_lengths(), cfg1_small["meta"].kp_lengths()
     bad_cb = cb.copy(); bad_cb[3, 1, 0] = 9
