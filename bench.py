@@ -595,7 +595,9 @@ def run_ours(args, workload=None, extras=True):
     # clock); the per-symbol costs are ncu counters of this kernel, the symbol rate is this run's.
     sm_limits = None
     if "decompress_sm" in ncu_consts and dec_ms > 0:
-        c, m = ncu_consts["decompress_sm"], ncu_consts["measured_sm_rates"]
+        # weights and KV caches cost differently per symbol (a KV cache has more code shapes, hence more escapes)
+        c = ncu_consts.get("decompress_sm_weights", ncu_consts["decompress_sm"]) if wname in ("cfg2", "cfg4", "small") else ncu_consts["decompress_sm"]
+        m = ncu_consts["measured_sm_rates"]
         props = torch.cuda.get_device_properties(local)
         sms, ghz = props.multi_processor_count, ((clocks or {}).get("sm_mhz") or 0) / 1e3
         if ghz > 0:
@@ -605,7 +607,8 @@ def run_ours(args, workload=None, extras=True):
                           "achieved": warp_symbols_per_s * c["warp_instructions_per_warp_symbol"] / 1e9},
                 "lsu": {"bound": "lsu", "unit": "G wavefronts/s", "peak": sms * m["lsu_wavefronts_per_clk_sm"] * ghz,
                         "achieved": warp_symbols_per_s * c["lsu_wavefronts_per_warp_symbol"] / 1e9},
-                "per_warp_symbol": {"instructions": c["warp_instructions_per_warp_symbol"], "wavefronts": c["lsu_wavefronts_per_warp_symbol"]},
+                "per_warp_symbol": {"instructions": c["warp_instructions_per_warp_symbol"], "wavefronts": c["lsu_wavefronts_per_warp_symbol"],
+                                    "captured_on": c["workload"]},
                 "measured_rates": m,
                 "source": "per-symbol costs: ncu capture of this kernel (paper_2505_06901_b200/ncu_constants.json); peaks = SMs x measured rate x sampled SM clock",
             }
