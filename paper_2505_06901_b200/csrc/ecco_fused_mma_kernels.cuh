@@ -14,7 +14,10 @@ namespace {
 // accumulate (fp16 x fp16 products are exact in fp32).  A warp is independent of the others: no
 // vector slice in shared memory, no block barrier.
 // ---------------------------------------------------------------------------------------------
-constexpr uint32_t kMmaValueBytes = 8 * 1024;                               // eight [32 rows][16 k] fp16 tiles
+// Eight [32 rows][16 k] fp16 tiles per warp, the last of which lies over rows 0..7 of the warp's bit-stream array: it
+// is written when symbol 127 has been decoded, and by then every lane is past stream bit 256 (22 header bits at least
+// and two bits per symbol), while the outlier fields sit in bits 272..511, rows 8..15.
+constexpr uint32_t kMmaValueBytes = 7 * 1024;
 constexpr uint32_t kMmaWarpBytes = kTabBytes / 2 + kMmaValueBytes + kBitsBytes;   // half a value table (two warps share one), tiles, bit stream
 // value tables first, then per warp the tiles and the bit-stream array; *vals = the warp's first tile
 __device__ __forceinline__ WarpSmem mma_warp_smem(const Tables& tb, uint32_t nw, uint32_t* vals)
@@ -56,8 +59,8 @@ __device__ __forceinline__ void row_dot_mma(const Block& blk, const Tables& tb, 
 {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t swz = ((lane >> 2) & 1u) << 4, my_row = vals + lane * 32;
-    const GroupHeader h = open_group<kTabHalf>(blk, tb, ws, T);
-    __syncwarp();                                          // the tiles of the previous group have been read
+    __syncwarp();                                          // the tiles of the previous group have been read (the last one is
+    const GroupHeader h = open_group<kTabHalf>(blk, tb, ws, T);     // about to be overwritten by this group's stream)
     uint32_t r8[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree, kTabHalf>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t) {
         const int col = tile_column(n & 15);               // see load_vfrag; clipped positions arrive as +0
