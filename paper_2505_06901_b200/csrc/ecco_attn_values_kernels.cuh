@@ -89,7 +89,8 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-constexpr uint32_t kAvValueBytes = 8 * 1024;                                // eight [32 tokens][16 dims] fp16 tiles
+// eight [32 tokens][16 dims] fp16 tiles, the last of which lies over rows 0..7 of the warp's bit-stream array (see K2m)
+constexpr uint32_t kAvValueBytes = 7 * 1024;
 constexpr uint32_t kAvWarpBytes = kTabBytes / 2 + kAvValueBytes + kBitsBytes;   // half a value table (two warps share one), tiles, bit stream
 constexpr uint32_t kAvSlots = 4;                                            // reduction slots: see flush
 
@@ -253,8 +254,8 @@ ecco_attn_values_kernel(const uint8_t* __restrict__ d_meta, const uint8_t* __res
                 asm volatile("prefetch.global.L2 [%0];" ::"l"(d_scores + (static_cast<size_t>(nbh) * q_per_kv + lane) * seq + nt));
         }
         // lanes past the end of the row decode the row's last token again (zeroed below)
-        const GroupHeader h = open_group<kTabHalf>(cur, tb, ws, T);
         __syncwarp();                                      // the tiles of the previous token tile have been read
+        const GroupHeader h = open_group<kTabHalf>(cur, tb, ws, T);
         uint32_t r[8] = {0, 0, 0, 0, 0, 0, 0, 0};
         const uint32_t end = decode_symbols<true, 16, kBlockBits, kFusedFree, kTabHalf>(h, ws, tb.pairs, [&](int n, uint32_t v, uint32_t, bool, uint32_t) {
             const int slot = (n & 15) >> 1;                // clipped positions arrive as +0
