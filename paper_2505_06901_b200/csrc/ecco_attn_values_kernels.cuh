@@ -92,7 +92,7 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], const uint32_t (&a)[4],
 // eight [32 tokens][16 dims] fp16 tiles, the last of which lies over rows 0..7 of the warp's bit-stream array (see K2m)
 constexpr uint32_t kAvValueBytes = 7 * 1024;
 constexpr uint32_t kAvWarpBytes = kTabBytes / 2 + kAvValueBytes + kBitsBytes;   // half a value table (two warps share one), tiles, bit stream
-constexpr uint32_t kAvSlots = 4;                                            // reduction slots: see flush
+constexpr uint32_t kAvSlots = 8;                                            // reduction slots: see flush
 
 constexpr float kProbScale = 32768.0f, kProbUnscale = 1.0f / 32768.0f;      // powers of two: exact
 
