@@ -25,6 +25,9 @@
  * d_meta must be 16-byte aligned.  The library refuses to run on a device that is not
  * compute capability 10.x (ECCO_ERR_UNSUPPORTED_ARCH); there is no CPU fallback.
  *
+ * Graph capture: a chain of device calls may be captured into a CUDA graph and replayed, once every entry point in
+ * it has been called eagerly on that device (the first call sets its kernels' attributes).
+ *
  * Stream order: the usual one.  Internally the kernels are launched so that one may become
  * resident while the previous kernel of the stream is still draining, but each waits for that
  * kernel to complete before its first access to memory, so only launch latency overlaps.  The

@@ -863,6 +863,60 @@ def test_var_decompress_config2_gate_full_size(B, eo, W, synth):
     assert total / n < 512                                                  # on average the stream is shorter than the blocks
 
 
+# ------------------------------------------------------------------ capture into a CUDA graph
+def test_calls_can_be_captured_into_a_cuda_graph(B, eo, kv_small, cfg1_small, synth):
+    """The device calls neither synchronise nor allocate, so a chain of them can be captured into a CUDA graph
+    (after one eager call of each, which sets the kernels' attributes) and replayed; the replay gives the eager
+    results bit for bit, also after the inputs have changed in place."""
+    wm, km = B.meta_to_device(lib_meta_from_oracle(B, cfg1_small["meta"])), B.meta_to_device(lib_meta_from_oracle(B, kv_small["meta"]))
+    wb, kb = dev(cfg1_small["blocks"]), dev(kv_small["blocks"])                 # 256 x 1024 weights, K cache [2][4][256]
+    n_out, k, heads, seq, qpk = 256, 1024, 8, 256, 2
+    x = dev(synth.activations(8, k, 3))
+    q = dev(synth.queries(1, heads * qpk, 4))
+    out = torch.empty(2048 * 128, dtype=torch.float16, device="cuda")
+    y1, y8 = torch.empty((1, n_out), dtype=torch.float32, device="cuda"), torch.empty((8, n_out), dtype=torch.float32, device="cuda")
+    sc = torch.empty((1, heads * qpk, seq), dtype=torch.float32, device="cuda")
+    av = torch.empty((1, heads * qpk, 128), dtype=torch.float32, device="cuda")
+    items1, items8 = [(wm, wb, n_out, k, x, y1)], [(wm, wb, n_out, k, x, y8)]
+    nb1, nb8 = B.ecco_gemv_batch_workspace_bytes(items1, 1), B.ecco_gemv_batch_workspace_bytes(items8, 8)
+    ws1, ws8 = torch.empty(nb1, dtype=torch.uint8, device="cuda"), torch.empty(nb8, dtype=torch.uint8, device="cuda")
+    nbv = B.ecco_attn_values_workspace_bytes(1, heads, seq, qpk)
+    wsv = torch.empty(nbv, dtype=torch.uint8, device="cuda")
+    a1, a8 = B.gemv_items(items1), B.gemv_items(items8)
+
+    def chain(st):
+        B.ecco_decompress(wm, wb, 2048, out, st)
+        B.ecco_gemv_batch(a1, 1, ws1, nb1, st)
+        B.ecco_gemv_batch(a8, 8, ws8, nb8, st)
+        B.ecco_attn_scores(km, kb, 1, heads, seq, qpk, q, 0.0884, sc, st)
+        B.ecco_attn_values(km, kb, 1, heads, seq, qpk, sc, av, wsv, nbv, st)
+
+    results = lambda: [t.clone() for t in (out, y1, y8, sc, av)]
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        chain(st)                                          # eager: also the first call of every kernel
+        st.synchronize()
+        want = results()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            chain(st)
+        for t in (out, y1, y8, sc, av):
+            t.fill_(float("nan"))
+        g.replay()
+        st.synchronize()
+        assert B.ecco_device_status() == 0
+        assert all(torch.equal(a, b) for a, b in zip(want, results()))
+        x.mul_(0.5)                                        # new inputs in the same buffers
+        q.mul_(2.0)
+        g.replay()
+        st.synchronize()
+        replayed = results()
+        chain(st)
+        st.synchronize()
+        assert all(torch.equal(a, b) for a, b in zip(replayed, results()))
+        assert not torch.equal(replayed[1], want[1])
+
+
 # ------------------------------------------------------------------ stream order of back-to-back calls
 def test_back_to_back_calls_keep_stream_order(B, eo, kv_small, cfg1_small, synth):
     """The kernels are launched so that one may start while its predecessor in the stream drains.  Calls that
