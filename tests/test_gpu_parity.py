@@ -517,6 +517,24 @@ def test_config2_llama7b_layer_full_size(B, eo, W, synth):
     assert B.ecco_device_status() == 0
     for (om, t), (_, _, n, d_out) in zip(metas, items):
         assert_device_equals_oracle(eo, om, t.blocks, d_out)
+    # the fused GEMV in the launch configuration bench.py times: matrices that share x in one ecco_gemv_batch call
+    # (here q with itself standing in for k and v, and gate twice for gate + up), every output row against the oracle
+    (oq, tq), (og, tg) = metas[0], metas[1]
+    for batch in (1, 8):
+        for om, t, (d_meta, d_blocks, _, _), copies in ((oq, tq, items[0], 3), (og, tg, items[1], 2)):
+            n_out, k = t.shape
+            x = synth.activations(batch, k, 90 + batch)
+            d_x = dev(x)
+            ys = [torch.full((batch, n_out), float("nan"), dtype=torch.float32, device="cuda") for _ in range(copies)]
+            call = [(d_meta, d_blocks, n_out, k, d_x, y) for y in ys]
+            wsb = B.ecco_gemv_batch_workspace_bytes(call, batch)
+            ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+            B.ecco_gemv_batch(call, batch, ws, wsb)
+            torch.cuda.synchronize()
+            assert B.ecco_device_status() == 0
+            ref, refabs = oracle_gemv_threads(eo, om, t.blocks, n_out, k, x, batch)
+            for y in ys:
+                check_fused(y.cpu().numpy().astype(np.float64), ref, refabs, f"gemv batch-call b{batch} full {n_out}x{k}")
 
 
 def check_full_attn(B, eo, synth, t, qpk):
