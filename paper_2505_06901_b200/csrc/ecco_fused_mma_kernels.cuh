@@ -130,7 +130,10 @@ ecco_gemv_mma_kernel(const __grid_constant__ GemvBatch batch, int n_cols, float*
     const int W = static_cast<int>(balanced_warps(static_cast<uint64_t>(U), gridDim.x * static_cast<uint32_t>(nw)));
     const int64_t u0 = wg < W ? unit_begin(U, W, wg) : 0, u1 = wg < W ? unit_begin(U, W, wg + 1) : 0;
     issue_tables(tb, d_meta);
-    if (!same_tables(batch, tb)) return;                   // images are host-written: readable before the wait
+    if (!same_tables(batch, tb)) {                         // images are host-written: readable before the wait
+        wait_tables(tb);                                   // the table copies into this CTA's shared memory must land first
+        return;
+    }
     dependency_wait();                                     // everything but the host-written tables: after the previous kernel of the stream
     GemvPos pos = {0, 0, 0};
     if (u0 < u1) { pos = gemv_pos_of(batch, u0); prefetch_block_l2(gemv_block_ptr(batch, pos, lane)); }
